@@ -1,0 +1,145 @@
+/*
+ * btc.h -- C ABI of the B200 (sm_100a) codebook-binary linear layer.
+ *
+ * The layer (BTC-LLM inference path) stores a weight matrix as indices into a
+ * binary codebook plus a row-wise scale:
+ *
+ *     W^[n, j*v:(j+1)*v] = alpha_n * C[idx[n, j]] (+ mu_n),   C in {+1,-1}^{Kc x v}
+ *     y[m, n]            = sum_k x[m, k] * W^[n, k]
+ *
+ * (storage rule and block-dot sum: paper appendix "Binary codebook LUT-GEMM";
+ * row-wise alpha / mu: Eq. 1-2 and the "Dequantize" step of Algorithm "Binary
+ * Transformation and Compression").  Rows of W^ are output features, blocks of
+ * length v run along the input dimension K, and v must divide K.
+ *
+ * Conventions for every entry point
+ *   - All array arguments are DEVICE pointers owned by the caller unless a
+ *     parameter is explicitly called "host".  The library allocates no device
+ *     memory, never synchronises, and enqueues its work on `stream` (a
+ *     cudaStream_t passed as void*, NULL = the legacy default stream).
+ *   - Returns a btc_status; never aborts, traps or prints.  Argument errors are
+ *     detected on the host before anything is launched.
+ *   - idx values must be < Kc; this is the caller's contract (kernels do not
+ *     check it).  btc_validate_indices checks it on the device.
+ *   - Ranges: 1 <= v <= 32, K % v == 0, 1 <= Kc <= 65536 (Kc need not be a power
+ *     of two), N >= 1, M >= 1.
+ *   - Alignment: x, idx, y and C_packed 16-byte aligned; alpha / mu 2-byte.
+ */
+#ifndef BTC_H_
+#define BTC_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#if defined(__GNUC__)
+#define BTC_API __attribute__((visibility("default")))
+#else
+#define BTC_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    BTC_OK = 0,
+    BTC_ERR_NULL = 1,        /* a required pointer is NULL                              */
+    BTC_ERR_SHAPE = 2,       /* v, Kc, M, N, K out of range, or v does not divide K     */
+    BTC_ERR_ALIGN = 3,       /* a pointer misses its alignment                          */
+    BTC_ERR_UNSUPPORTED = 4, /* dtype / option not implemented by this entry point      */
+    BTC_ERR_WORKSPACE = 5,   /* workspace missing or smaller than ..._workspace_bytes() */
+    BTC_ERR_CUDA = 6,        /* a CUDA runtime / driver call failed                     */
+    BTC_ERR_TIMEOUT = 7      /* a bounded device-side wait ran out (status word)        */
+} btc_status;
+
+typedef enum { BTC_F16 = 0, BTC_BF16 = 1, BTC_F32 = 2 } btc_dtype;
+
+/* Optional online activation transform x' = x * D * (P1 (x) P2), D = diag(sigma) with
+ * sigma in {+1,-1} (paper Section 4.2 "Transformation Pair", applied at inference as
+ * X <- X T).  With x viewed row-major as a k1 x k2 matrix X:  X' = P1^T (X o sigma) P2.
+ * sigma_bits: device uint32[ceil(K/32)], bit k set = -1 (flip channel k).
+ * P1 [k1*k1], P2 [k2*k2]: device fp32, row-major.  k1 * k2 == K. */
+typedef struct {
+    const uint32_t *sigma_bits;
+    const float *P1;
+    const float *P2;
+    int k1;
+    int k2;
+} btc_transform;
+
+/* Library version (major*10000 + minor*100 + patch) and a static description of a status. */
+BTC_API int btc_version(void);
+BTC_API const char *btc_status_string(int status);
+
+/* Last CUDA error code (cudaError_t as int) recorded by a call that returned BTC_ERR_CUDA
+ * on this host thread; 0 if none. */
+BTC_API int btc_last_cuda_error(void);
+
+/* ---- codebook packing (offline, once per layer) --------------------------------------------
+ * Bit map b = (c + 1) / 2 (Algorithm "Efficient Binary Vector Packing and Unpacking"): bit t
+ * (LSB first) of C_packed[k] is 1 where C_pm1[k][t] >= 0 (sign(0) = +1, Section 4.1 M-step),
+ * bits >= v are 0.  C_pm1: int8 [Kc][v] row-major.
+ * C_packed is a buffer of btc_codebook_packed_bytes(Kc, v) bytes, 16-byte aligned: the first Kc
+ * uint32 words are the public form just described (the interchange format); the rest is a
+ * kernel-private re-arrangement of the same bits that the linear kernels read, so the whole
+ * buffer must be passed to them unchanged.  btc_codebook_packed_bytes returns 0 for an invalid
+ * shape. */
+BTC_API size_t btc_codebook_packed_bytes(int Kc, int v);
+BTC_API int btc_codebook_pack(const int8_t *C_pm1, int Kc, int v, uint32_t *C_packed, void *stream);
+/* Same mapping with both pointers in HOST memory; runs on the calling thread, no GPU work. */
+BTC_API int btc_codebook_pack_host(const int8_t *C_pm1_host, int Kc, int v, uint32_t *C_packed_host);
+
+/* ---- the layer ---------------------------------------------------------------------------
+ * y[m, n] = alpha_n * sum_j <x[m, j*v:(j+1)*v], C[idx[n, j]]>  (+ mu_n * sum_k x[m, k])
+ *
+ *   x        [M, K] row-major, x_dtype = BTC_F16 or BTC_BF16
+ *   idx      uint16 [N, K/v] row-major
+ *   C_packed the buffer written by btc_codebook_pack (btc_codebook_packed_bytes(Kc, v) bytes)
+ *   alpha    fp16 [N]; mu fp16 [N] or NULL (NULL = no mean term)
+ *   T        NULL, or an activation transform applied to x first (see btc_transform)
+ *   y        [M, N] row-major, y_dtype = BTC_F32 (also BTC_F16 / BTC_BF16, rounded to nearest)
+ *   workspace / workspace_bytes: scratch of at least btc_linear_workspace_bytes(...) bytes,
+ *            256-byte aligned; may be NULL when that function returns 0.  Contents are
+ *            undefined afterwards; concurrent calls need distinct workspaces.
+ *
+ * btc_linear_gemv: the memory-bound decode path, 1 <= M <= 8, fp32 accumulation of the
+ *   identity <x, c> = 2 * sum_{bit=1} x - sum x  (or its signed-sum equivalent).
+ * btc_linear_gemm: any M >= 1, built for M >= 128: index tiles are decoded to +-1 bf16 tiles in
+ *   shared memory and multiplied on the tcgen05 tensor cores with fp32 accumulation in
+ *   tensor memory; alpha (and mu) are applied in fp32 in the epilogue.  fp16 x is accepted and
+ *   multiplied as fp16.
+ * Errors: NULL / SHAPE / ALIGN / UNSUPPORTED / WORKSPACE as above; BTC_ERR_CUDA if a launch
+ * fails.  Both are asynchronous: a device-side failure shows up at the caller's next sync.
+ */
+BTC_API size_t btc_linear_workspace_bytes(int M, int N, int K, int v, int Kc);
+
+BTC_API int btc_linear_gemv(const void *x, int x_dtype, const uint16_t *idx, const uint32_t *C_packed,
+                    const void *alpha, const void *mu, const btc_transform *T, void *y, int y_dtype,
+                    int M, int N, int K, int v, int Kc, void *workspace, size_t workspace_bytes,
+                    void *stream);
+
+BTC_API int btc_linear_gemm(const void *x, int x_dtype, const uint16_t *idx, const uint32_t *C_packed,
+                    const void *alpha, const void *mu, const btc_transform *T, void *y, int y_dtype,
+                    int M, int N, int K, int v, int Kc, void *workspace, size_t workspace_bytes,
+                    void *stream);
+
+/* ---- helpers (not on the hot path) --------------------------------------------------------- */
+
+/* B^[n, j*v + t] = +1 / -1 as int8 [N, K]: the decoded sign matrix, for bit-exact checks. */
+BTC_API int btc_decode_pm1(const uint16_t *idx, const uint32_t *C_packed, int N, int K, int v, int Kc,
+                   int8_t *B_out, void *stream);
+
+/* Counts entries of idx[0..count) that are >= Kc into *bad_count (device int32, zeroed by the
+ * call before counting). */
+BTC_API int btc_validate_indices(const uint16_t *idx, size_t count, int Kc, int *bad_count, void *stream);
+
+/* Bits per weight.  mode 0: log2(Kc)/v; 1: ceil(log2 Kc)/v (the paper's accounting, Section 4.3);
+ * 2: 16/v (uint16 containers as stored here).  Adds scale_bits_per_row/K, and v*Kc/(N*K) for the
+ * codebook when with_codebook != 0.  Host arithmetic only; returns -1 for an invalid shape. */
+BTC_API double btc_bits_per_weight(int N, int K, int v, int Kc, int scale_bits_per_row, int mode,
+                           int with_codebook);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* BTC_H_ */

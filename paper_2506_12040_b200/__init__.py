@@ -1,0 +1,14 @@
+"""B200 (sm_100a) codebook-binary linear layer: Python names for the C ABI in include/btc.h."""
+from .binding import (  # noqa: F401
+    BtcError,
+    bits_per_weight,
+    codebook_pack,
+    codebook_pack_host,
+    decode_pm1,
+    lib,
+    linear,
+    linear_gemm,
+    linear_gemv,
+    linear_workspace_bytes,
+    validate_indices,
+)

@@ -1,0 +1,212 @@
+"""ctypes binding of libbtc_b200.so: argument marshalling only.
+
+Every step of the layer runs in the library's CUDA kernels; torch supplies device memory
+and the current stream.  There is no CPU or eager-PyTorch fallback: if the shared library
+cannot be loaded, importing this module raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+import torch
+
+from . import build as _build
+
+BTC_F16, BTC_BF16, BTC_F32 = 0, 1, 2
+_DT = {torch.float16: BTC_F16, torch.bfloat16: BTC_BF16, torch.float32: BTC_F32}
+
+EXPORTS = (
+    "btc_version", "btc_status_string", "btc_last_cuda_error", "btc_codebook_packed_bytes",
+    "btc_codebook_pack", "btc_codebook_pack_host", "btc_linear_workspace_bytes", "btc_linear_gemv",
+    "btc_linear_gemm", "btc_decode_pm1", "btc_validate_indices", "btc_bits_per_weight",
+)
+
+
+class BtcTransform(ctypes.Structure):
+    _fields_ = [("sigma_bits", ctypes.c_void_p), ("P1", ctypes.c_void_p), ("P2", ctypes.c_void_p),
+                ("k1", ctypes.c_int), ("k2", ctypes.c_int)]
+
+
+class BtcError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        msg = lib.btc_status_string(status).decode()
+        if status == 6:
+            msg += f" [cudaError {lib.btc_last_cuda_error()}]"
+        super().__init__(f"{where}: {msg} (status {status})")
+
+
+def _load() -> ctypes.CDLL:
+    path = _build.LIB
+    if not os.path.exists(path) or _build.is_stale():
+        # The library travels with the source tree; build it in place if it is absent or older
+        # than its sources.  No nvcc means no library, and that is an error, not a fallback.
+        _build.build_library()
+    L = ctypes.CDLL(path)
+    vp, ci, sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_size_t
+    L.btc_version.restype = ci
+    L.btc_status_string.restype = ctypes.c_char_p
+    L.btc_status_string.argtypes = [ci]
+    L.btc_last_cuda_error.restype = ci
+    L.btc_codebook_packed_bytes.restype = sz
+    L.btc_codebook_packed_bytes.argtypes = [ci, ci]
+    L.btc_codebook_pack.argtypes = [vp, ci, ci, vp, vp]
+    L.btc_codebook_pack_host.argtypes = [vp, ci, ci, vp]
+    L.btc_linear_workspace_bytes.restype = sz
+    L.btc_linear_workspace_bytes.argtypes = [ci] * 5
+    lin = [vp, ci, vp, vp, vp, vp, ctypes.POINTER(BtcTransform), vp, ci, ci, ci, ci, ci, ci, vp, sz, vp]
+    L.btc_linear_gemv.argtypes = lin
+    L.btc_linear_gemm.argtypes = lin
+    L.btc_decode_pm1.argtypes = [vp, vp, ci, ci, ci, ci, vp, vp]
+    L.btc_validate_indices.argtypes = [vp, sz, ci, vp, vp]
+    L.btc_bits_per_weight.restype = ctypes.c_double
+    L.btc_bits_per_weight.argtypes = [ci] * 7
+    return L
+
+
+lib = _load()
+
+
+def _stream() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
+    return None if t is None else t.data_ptr()
+
+
+def _dev(t: torch.Tensor, name: str):
+    if not t.is_cuda:
+        raise ValueError(f"{name} must be a CUDA tensor")
+    if not t.is_contiguous():
+        raise ValueError(f"{name} must be contiguous")
+
+
+def packed_words(Kc: int, v: int) -> int:
+    n = int(lib.btc_codebook_packed_bytes(Kc, v))
+    if n == 0:
+        raise ValueError("invalid codebook shape")
+    return n // 4
+
+
+def codebook_pack(C_pm1: torch.Tensor) -> torch.Tensor:
+    """int8 [Kc, v] of +-1 (device) -> packed codebook buffer (int32 words).  The first Kc words are
+    the public form (bit t = element t); the rest is kernel-private.  Pass the whole tensor on."""
+    _dev(C_pm1, "C_pm1")
+    if C_pm1.dtype != torch.int8 or C_pm1.dim() != 2:
+        raise ValueError("C_pm1 must be int8 [Kc, v]")
+    Kc, v = C_pm1.shape
+    out = torch.empty(packed_words(Kc, v), dtype=torch.int32, device=C_pm1.device)
+    st = lib.btc_codebook_pack(C_pm1.data_ptr(), Kc, v, out.data_ptr(), _stream())
+    if st:
+        raise BtcError(st, "btc_codebook_pack")
+    return out
+
+
+def codebook_pack_host(C_pm1: torch.Tensor) -> torch.Tensor:
+    """Host-memory variant (CPU tensors in and out); no GPU work."""
+    if C_pm1.is_cuda or C_pm1.dtype != torch.int8 or C_pm1.dim() != 2 or not C_pm1.is_contiguous():
+        raise ValueError("C_pm1 must be a contiguous CPU int8 [Kc, v] tensor")
+    Kc, v = C_pm1.shape
+    out = torch.empty(packed_words(Kc, v), dtype=torch.int32)
+    st = lib.btc_codebook_pack_host(C_pm1.data_ptr(), Kc, v, out.data_ptr())
+    if st:
+        raise BtcError(st, "btc_codebook_pack_host")
+    return out
+
+
+def linear_workspace_bytes(M: int, N: int, K: int, v: int, Kc: int) -> int:
+    return int(lib.btc_linear_workspace_bytes(M, N, K, v, Kc))
+
+
+def _linear(fn, name, x, idx, C_packed, alpha, v, Kc, mu, out, out_dtype, workspace, transform):
+    for t, n in ((x, "x"), (idx, "idx"), (C_packed, "C_packed"), (alpha, "alpha")):
+        _dev(t, n)
+    if x.dim() != 2 or idx.dim() != 2:
+        raise ValueError("x must be [M, K] and idx [N, K/v]")
+    if x.dtype not in (torch.float16, torch.bfloat16):
+        raise ValueError("x must be fp16 or bf16")
+    if idx.element_size() != 2 or alpha.dtype != torch.float16 or C_packed.element_size() != 4:
+        raise ValueError("idx must be 16-bit integers, alpha fp16, C_packed 32-bit words")
+    M, K = x.shape
+    N, Kb = idx.shape
+    if C_packed.numel() != packed_words(Kc, v):
+        raise ValueError("C_packed is not the buffer codebook_pack wrote for this (Kc, v)")
+    if Kb * v != K or alpha.numel() != N:
+        raise ValueError("shape mismatch between x, idx, v and alpha")
+    if mu is not None:
+        _dev(mu, "mu")
+        if mu.dtype != torch.float16 or mu.numel() != N:
+            raise ValueError("mu must be fp16 [N]")
+    if out is None:
+        out = torch.empty((M, N), dtype=out_dtype, device=x.device)
+    else:
+        _dev(out, "out")
+        if tuple(out.shape) != (M, N):
+            raise ValueError("out must be [M, N]")
+    tr = None
+    extra = 0
+    if transform is not None:
+        sig, P1, P2 = transform
+        tr = BtcTransform(sig.data_ptr(), P1.data_ptr(), P2.data_ptr(), P1.shape[0], P2.shape[0])
+        extra = (M * K * 2 + 255) // 256 * 256
+    need = linear_workspace_bytes(M, N, K, v, Kc) + extra
+    ws_ptr, ws_bytes = None, 0
+    if need:
+        if workspace is None:
+            workspace = torch.empty(need, dtype=torch.uint8, device=x.device)
+        ws_ptr, ws_bytes = workspace.data_ptr(), workspace.numel() * workspace.element_size()
+    st = fn(x.data_ptr(), _DT[x.dtype], idx.data_ptr(), C_packed.data_ptr(), alpha.data_ptr(), _ptr(mu),
+            ctypes.byref(tr) if tr is not None else None, out.data_ptr(), _DT[out.dtype],
+            M, N, K, v, Kc, ws_ptr, ws_bytes, _stream())
+    if st:
+        raise BtcError(st, name)
+    return out
+
+
+def linear_gemv(x, idx, C_packed, alpha, v, Kc, mu=None, out=None, out_dtype=torch.float32, workspace=None,
+                transform=None):
+    """Decode path (M <= 8): y[M, N] = x * W^T with W^ = alpha * C[idx] (+ mu)."""
+    return _linear(lib.btc_linear_gemv, "btc_linear_gemv", x, idx, C_packed, alpha, v, Kc, mu, out, out_dtype,
+                   workspace, transform)
+
+
+def linear_gemm(x, idx, C_packed, alpha, v, Kc, mu=None, out=None, out_dtype=torch.float32, workspace=None,
+                transform=None):
+    """Tensor-core path (any M, built for large M)."""
+    return _linear(lib.btc_linear_gemm, "btc_linear_gemm", x, idx, C_packed, alpha, v, Kc, mu, out, out_dtype,
+                   workspace, transform)
+
+
+def linear(x, idx, C_packed, alpha, v, Kc, **kw):
+    """Routes by M the way a caller would: decode path up to 8 rows, tensor-core path above."""
+    return (linear_gemv if x.shape[0] <= 8 else linear_gemm)(x, idx, C_packed, alpha, v, Kc, **kw)
+
+
+def decode_pm1(idx, C_packed, v, Kc) -> torch.Tensor:
+    """Decoded sign matrix int8 [N, K]."""
+    _dev(idx, "idx"); _dev(C_packed, "C_packed")
+    N, Kb = idx.shape
+    out = torch.empty((N, Kb * v), dtype=torch.int8, device=idx.device)
+    st = lib.btc_decode_pm1(idx.data_ptr(), C_packed.data_ptr(), N, Kb * v, v, Kc,
+                            out.data_ptr(), _stream())
+    if st:
+        raise BtcError(st, "btc_decode_pm1")
+    return out
+
+
+def validate_indices(idx, Kc: int) -> int:
+    """Number of indices >= Kc (synchronises to read the count back)."""
+    _dev(idx, "idx")
+    bad = torch.empty(1, dtype=torch.int32, device=idx.device)
+    st = lib.btc_validate_indices(idx.data_ptr(), idx.numel(), Kc, bad.data_ptr(), _stream())
+    if st:
+        raise BtcError(st, "btc_validate_indices")
+    return int(bad.item())
+
+
+def bits_per_weight(N, K, v, Kc, scale_bits_per_row=0, mode="container", with_codebook=False) -> float:
+    m = {"nominal": 0, "container": 1, "stored": 2}[mode]
+    return float(lib.btc_bits_per_weight(N, K, v, Kc, scale_bits_per_row, m, int(with_codebook)))

@@ -1,0 +1,144 @@
+// Host side of the C ABI: argument validation, variant selection, launch.
+#include <cmath>
+#include "btc_internal.cuh"
+
+namespace btc {
+
+static thread_local int g_last_cuda_error = 0;
+
+int cuda_fail(cudaError_t e)
+{
+    g_last_cuda_error = (int)e;
+    return BTC_ERR_CUDA;
+}
+
+static bool aligned(const void *p, size_t a) { return reinterpret_cast<uintptr_t>(p) % a == 0; }
+
+static int validate(const void *x, int x_dt, const uint16_t *idx, const uint32_t *Cp, const void *alpha,
+                    void *y, int y_dt, int M, int N, int K, int v, int Kc)
+{
+    if (!x || !idx || !Cp || !alpha || !y) return BTC_ERR_NULL;
+    if (v < 1 || v > 32 || Kc < 1 || Kc > 65536 || M < 1 || N < 1 || K < 1 || K % v) return BTC_ERR_SHAPE;
+    if (x_dt != BTC_F16 && x_dt != BTC_BF16) return BTC_ERR_UNSUPPORTED;
+    if (y_dt != BTC_F32 && y_dt != BTC_F16 && y_dt != BTC_BF16) return BTC_ERR_UNSUPPORTED;
+    if (!aligned(x, 16) || !aligned(idx, 16) || !aligned(y, 16) || !aligned(Cp, 16) || !aligned(alpha, 2))
+        return BTC_ERR_ALIGN;
+    return BTC_OK;
+}
+
+enum Path { PATH_GEMV, PATH_GEMM };
+
+static int run_linear(Path path, const void *x, int x_dt, const uint16_t *idx, const uint32_t *Cp,
+                      const void *alpha, const void *mu, const btc_transform *T, void *y, int y_dt, int M,
+                      int N, int K, int v, int Kc, void *ws, size_t ws_bytes, void *stream)
+{
+    int rc = validate(x, x_dt, idx, Cp, alpha, y, y_dt, M, N, K, v, Kc);
+    if (rc != BTC_OK) return rc;
+    if (mu && !aligned(mu, 2)) return BTC_ERR_ALIGN;
+    if (path == PATH_GEMV && M > 8) return BTC_ERR_SHAPE;
+    const size_t need = btc_linear_workspace_bytes(M, N, K, v, Kc);
+    const size_t xt_bytes = T ? (((size_t)M * K * 2 + 255) / 256) * 256 : 0;
+    if (need + xt_bytes > 0) {
+        if (!ws || ws_bytes < need + xt_bytes) return BTC_ERR_WORKSPACE;
+        if (!aligned(ws, 256)) return BTC_ERR_ALIGN;
+    }
+    cudaStream_t s = (cudaStream_t)stream;
+
+    LinearArgs a;
+    a.x = x; a.idx = idx; a.Cp = Cp;
+    a.alpha = reinterpret_cast<const __half *>(alpha);
+    a.mu = reinterpret_cast<const __half *>(mu);
+    a.y = y; a.workspace = ws; a.workspace_bytes = ws_bytes;
+    a.x_dt = x_dt; a.y_dt = y_dt;
+    a.M = M; a.N = N; a.K = K; a.v = v; a.Kc = Kc; a.Kb = K / v;
+
+    if (T) {
+        // The transformed activations live at the front of the workspace; the kernels' own
+        // scratch follows.
+        if (!T->sigma_bits || !T->P1 || !T->P2) return BTC_ERR_NULL;
+        if (T->k1 < 1 || T->k2 < 1 || (long long)T->k1 * T->k2 != K) return BTC_ERR_SHAPE;
+        rc = launch_transform(x, x_dt, *T, ws, M, K, s);
+        if (rc != BTC_OK) return rc;
+        a.x = ws;
+        a.workspace = static_cast<char *>(ws) + xt_bytes;
+        a.workspace_bytes = ws_bytes - xt_bytes;
+    }
+
+    rc = BTC_ERR_UNSUPPORTED;
+    if (path == PATH_GEMV) rc = launch_gemv_decode(a, s);
+    else rc = launch_gemm_tcgen05(a, s);
+    if (rc == BTC_ERR_UNSUPPORTED) {
+        if (path == PATH_GEMM && M <= 8) rc = launch_gemv_decode(a, s);
+        if (rc == BTC_ERR_UNSUPPORTED) rc = launch_linear_generic(a, s);
+    }
+    return rc;
+}
+
+}  // namespace btc
+
+using namespace btc;
+
+extern "C" int btc_version(void) { return 100; }
+
+extern "C" const char *btc_status_string(int st)
+{
+    switch (st) {
+    case BTC_OK: return "ok";
+    case BTC_ERR_NULL: return "a required pointer is NULL";
+    case BTC_ERR_SHAPE: return "shape out of range (1<=v<=32, v divides K, 1<=Kc<=65536, M,N,K>=1; gemv needs M<=8)";
+    case BTC_ERR_ALIGN: return "pointer alignment (x, idx, y, C_packed: 16 bytes; workspace: 256 bytes)";
+    case BTC_ERR_UNSUPPORTED: return "dtype or option not supported";
+    case BTC_ERR_WORKSPACE: return "workspace missing or too small";
+    case BTC_ERR_CUDA: return "CUDA call failed (see btc_last_cuda_error)";
+    case BTC_ERR_TIMEOUT: return "a bounded device-side wait ran out";
+    default: return "unknown status";
+    }
+}
+
+extern "C" int btc_last_cuda_error(void) { return g_last_cuda_error; }
+
+extern "C" size_t btc_codebook_packed_bytes(int Kc, int v)
+{
+    if (v < 1 || v > 32 || Kc < 1 || Kc > 65536) return 0;
+    return (size_t)((Kc + 3) / 4 * 4) * 8;
+}
+
+extern "C" size_t btc_linear_workspace_bytes(int M, int N, int K, int v, int Kc)
+{
+    if (v < 1 || v > 32 || Kc < 1 || Kc > 65536 || M < 1 || N < 1 || K < 1 || K % v) return 0;
+    size_t a = (M <= 8) ? gemv_decode_workspace_bytes(M, N, K, v, Kc) : 0;
+    size_t b = gemm_tcgen05_workspace_bytes(M, N, K, v, Kc);
+    size_t w = a > b ? a : b;
+    return (w + 255) / 256 * 256;
+}
+
+extern "C" int btc_linear_gemv(const void *x, int x_dtype, const uint16_t *idx, const uint32_t *C_packed,
+                               const void *alpha, const void *mu, const btc_transform *T, void *y, int y_dtype,
+                               int M, int N, int K, int v, int Kc, void *workspace, size_t workspace_bytes,
+                               void *stream)
+{
+    return run_linear(PATH_GEMV, x, x_dtype, idx, C_packed, alpha, mu, T, y, y_dtype, M, N, K, v, Kc,
+                      workspace, workspace_bytes, stream);
+}
+
+extern "C" int btc_linear_gemm(const void *x, int x_dtype, const uint16_t *idx, const uint32_t *C_packed,
+                               const void *alpha, const void *mu, const btc_transform *T, void *y, int y_dtype,
+                               int M, int N, int K, int v, int Kc, void *workspace, size_t workspace_bytes,
+                               void *stream)
+{
+    return run_linear(PATH_GEMM, x, x_dtype, idx, C_packed, alpha, mu, T, y, y_dtype, M, N, K, v, Kc,
+                      workspace, workspace_bytes, stream);
+}
+
+extern "C" double btc_bits_per_weight(int N, int K, int v, int Kc, int scale_bits_per_row, int mode,
+                                      int with_codebook)
+{
+    if (v < 1 || v > 32 || Kc < 1 || Kc > 65536 || N < 1 || K < 1 || mode < 0 || mode > 2) return -1.0;
+    double ib;
+    if (mode == 0) ib = std::log2((double)Kc);
+    else if (mode == 1) { int b = 0; while ((1 << b) < Kc) ++b; ib = b; }
+    else ib = 16.0;
+    double r = ib / v + (double)scale_bits_per_row / K;
+    if (with_codebook) r += (double)v * Kc / ((double)N * K);
+    return r;
+}

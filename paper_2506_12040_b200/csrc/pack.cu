@@ -1,0 +1,108 @@
+// Codebook packing, sign-matrix decode and index validation kernels (offline / checking helpers).
+#include "btc_internal.cuh"
+
+namespace btc {
+
+// Kernel-private word of one centroid for the decode path ("MMA layout"): the bit of weight t sits
+// at (t & 1) * 16 + P0 + (t >> 1) with P0 = 12 - v/2, so that `word & mask` with one bit kept per
+// 16-bit half is a pair of fp16 numbers {0, 2^(pos-24)}.  Defined for v % 4 == 0, v <= 24; 0 otherwise.
+__host__ __device__ inline uint32_t mma_layout_word(uint32_t pub, int v)
+{
+    if (v % 4 != 0 || v > 24) return 0u;
+    const int p0 = 12 - v / 2;
+    uint32_t w = 0;
+    for (int t = 0; t < v; ++t)
+        if ((pub >> t) & 1u) w |= 1u << ((t & 1) * 16 + p0 + (t >> 1));
+    return w;
+}
+
+// bit t of out[k] = (C[k][t] + 1) / 2, with C >= 0 read as +1; private words at out[Kc4 + k].
+__global__ void pack_codebook_kernel(const int8_t *__restrict__ C, int Kc, int v, uint32_t *__restrict__ out)
+{
+    const int k = blockIdx.x * blockDim.x + threadIdx.x;
+    const int Kc4 = (Kc + 3) / 4 * 4;
+    if (k >= Kc4) return;
+    uint32_t w = 0;
+    if (k < Kc)
+        for (int t = 0; t < v; ++t)
+            if (C[(size_t)k * v + t] >= 0) w |= 1u << t;
+    out[k] = w;
+    out[Kc4 + k] = mma_layout_word(w, v);
+}
+
+// One thread per (row, block): expands the centroid word into v int8 signs.
+__global__ void decode_pm1_kernel(const uint16_t *__restrict__ idx, const uint32_t *__restrict__ Cp,
+                                  size_t blocks, int Kb, int v, int8_t *__restrict__ B)
+{
+    const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= blocks) return;
+    const uint32_t w = Cp[idx[i]];
+    int8_t *dst = B + i * (size_t)v;   // row n = i / Kb, block j = i % Kb: offset n*K + j*v = i*v
+    for (int t = 0; t < v; ++t) dst[t] = ((w >> t) & 1u) ? 1 : -1;
+    (void)Kb;
+}
+
+__global__ void validate_indices_kernel(const uint16_t *__restrict__ idx, size_t count, int Kc, int *bad)
+{
+    size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const size_t stride = (size_t)gridDim.x * blockDim.x;
+    int local = 0;
+    for (; i < count; i += stride) local += (idx[i] >= Kc) ? 1 : 0;
+    for (int o = 16; o > 0; o >>= 1) local += __shfl_xor_sync(0xffffffffu, local, o);
+    if ((threadIdx.x & 31) == 0 && local) atomicAdd(bad, local);
+}
+
+}  // namespace btc
+
+using namespace btc;
+
+extern "C" int btc_codebook_pack(const int8_t *C_pm1, int Kc, int v, uint32_t *C_packed, void *stream)
+{
+    if (!C_pm1 || !C_packed) return BTC_ERR_NULL;
+    if (v < 1 || v > 32 || Kc < 1 || Kc > 65536) return BTC_ERR_SHAPE;
+    if (reinterpret_cast<uintptr_t>(C_packed) % 16) return BTC_ERR_ALIGN;
+    pack_codebook_kernel<<<(Kc + 3 + 127) / 128, 128, 0, (cudaStream_t)stream>>>(C_pm1, Kc, v, C_packed);
+    return cuda_check_launch();
+}
+
+extern "C" int btc_codebook_pack_host(const int8_t *C, int Kc, int v, uint32_t *out)
+{
+    if (!C || !out) return BTC_ERR_NULL;
+    if (v < 1 || v > 32 || Kc < 1 || Kc > 65536) return BTC_ERR_SHAPE;
+    const int Kc4 = (Kc + 3) / 4 * 4;
+    for (int k = 0; k < Kc4; ++k) {
+        uint32_t w = 0;
+        if (k < Kc)
+            for (int t = 0; t < v; ++t)
+                if (C[(size_t)k * v + t] >= 0) w |= 1u << t;
+        out[k] = w;
+        out[Kc4 + k] = mma_layout_word(w, v);
+    }
+    return BTC_OK;
+}
+
+extern "C" int btc_decode_pm1(const uint16_t *idx, const uint32_t *C_packed, int N, int K, int v, int Kc,
+                              int8_t *B_out, void *stream)
+{
+    if (!idx || !C_packed || !B_out) return BTC_ERR_NULL;
+    if (v < 1 || v > 32 || Kc < 1 || Kc > 65536 || N < 1 || K < 1 || K % v) return BTC_ERR_SHAPE;
+    const size_t blocks = (size_t)N * (K / v);
+    const size_t grid = (blocks + 255) / 256;
+    if (grid > 0x7fffffffull) return BTC_ERR_SHAPE;
+    decode_pm1_kernel<<<(unsigned)grid, 256, 0, (cudaStream_t)stream>>>(idx, C_packed, blocks, K / v, v, B_out);
+    return cuda_check_launch();
+}
+
+extern "C" int btc_validate_indices(const uint16_t *idx, size_t count, int Kc, int *bad_count, void *stream)
+{
+    if (!idx || !bad_count) return BTC_ERR_NULL;
+    if (Kc < 1 || Kc > 65536) return BTC_ERR_SHAPE;
+    cudaStream_t s = (cudaStream_t)stream;
+    cudaError_t e = cudaMemsetAsync(bad_count, 0, sizeof(int), s);
+    if (e != cudaSuccess) return cuda_fail(e);
+    if (count == 0) return BTC_OK;
+    size_t grid = (count + 255) / 256;
+    if (grid > 148 * 16) grid = 148 * 16;
+    validate_indices_kernel<<<(unsigned)grid, 256, 0, s>>>(idx, count, Kc, bad_count);
+    return cuda_check_launch();
+}

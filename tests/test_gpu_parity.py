@@ -1,0 +1,177 @@
+"""GPU parity: the CUDA path (through the C ABI) against the fp64 CPU oracle, element by element,
+on the same seeded inputs.  Tolerances: decode bit-exact; outputs max-rel-err <= 2e-3 for the
+decode path (fp32 accumulate, M <= 8) and <= 1e-2 for the tensor-core path."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2506_12040_b200 as btc
+import workloads as wl
+from util import TOL_GEMM, TOL_GEMV, errors, oracle_y, run_layer, to_device
+
+pytestmark = pytest.mark.gpu
+
+
+def _spec(N, K, v, Kc, **kw):
+    return wl.LayerSpec("t", N, K, v, Kc, **kw)
+
+
+# ------------------------------------------------------------------ packing / decode: bit exact
+
+@pytest.mark.parametrize("v,Kc", [(1, 2), (4, 9), (8, 85), (13, 500), (16, 4096), (16, 7132), (20, 65536), (32, 1000)])
+def test_pack_and_decode_bit_exact(v, Kc):
+    N, Kb = 37, 11
+    L = wl.make_layer(_spec(N, Kb * v, v, Kc), 1, seed=100 + v)
+    d = to_device(L)
+    assert np.array_equal(d["Cp"].cpu().numpy().view(np.uint32)[:Kc], oracle.pack_codebook(L.C_pm1))
+    B = btc.decode_pm1(d["idx"], d["Cp"], v, Kc).cpu().numpy()
+    assert np.array_equal(B, oracle.decode_pm1(L.idx, L.C_pm1))
+
+
+def test_validate_indices_counts():
+    idx = torch.arange(0, 5000, dtype=torch.int32).to(torch.int16).cuda()
+    assert btc.validate_indices(idx, 65536) == 0
+    assert btc.validate_indices(idx, 4096) == 5000 - 4096
+    assert btc.validate_indices(idx, 1) == 4999
+
+
+# ------------------------------------------------------------------ one-hot probes: decode through the real kernels
+
+@pytest.mark.parametrize("N,K,v,Kc", [(200, 256, 16, 300), (130, 320, 20, 65536), (64, 96, 12, 777)])
+@pytest.mark.parametrize("path", ["gemv", "gemm"])
+def test_one_hot_probe_is_exact(N, K, v, Kc, path):
+    """x = e_k  =>  y[m, n] = alpha_n * B^[n, k] exactly (one non-zero term), so the production kernels'
+    decode is checked bit for bit without materialising the weight."""
+    M = 8 if path == "gemv" else 160
+    L = wl.make_layer(_spec(N, K, v, Kc), M, seed=7)
+    ks = (np.arange(M) * 37 + 5) % K
+    xb = np.zeros((M, K), dtype=np.float16)
+    xb[np.arange(M), ks] = 1.0
+    L.x_bits = xb.view(np.uint16)
+    y, _ = run_layer(L, path)
+    B = oracle.decode_pm1(L.idx, L.C_pm1)
+    want = L.alpha.astype(np.float32)[None, :] * B[:, ks].T.astype(np.float32)
+    assert np.array_equal(y.cpu().numpy(), want)
+
+
+# ------------------------------------------------------------------ decode path parity (M <= 8)
+
+SMALL = [
+    # N, K, v, Kc, M, dist, mu
+    (1, 16, 16, 1, 1, "uniform", False),
+    (5, 64, 16, 7, 3, "uniform", True),
+    (257, 1040, 16, 4096, 8, "uniform", False),
+    (300, 2000, 20, 65536, 4, "zipf", False),
+    (129, 4096, 16, 8192, 1, "uniform", True),
+    (70, 11008, 16, 8192, 2, "uniform", False),
+    (1000, 640, 20, 21619, 5, "zipf", True),
+    (33, 72, 4, 9, 7, "uniform", False),
+    (96, 512, 8, 85, 6, "uniform", False),
+    (40, 126, 18, 21619, 1, "uniform", False),
+    (64, 960, 32, 5000, 8, "uniform", True),
+]
+
+
+@pytest.mark.parametrize("N,K,v,Kc,M,dist,mu", SMALL)
+def test_gemv_parity_small(N, K, v, Kc, M, dist, mu):
+    L = wl.make_layer(_spec(N, K, v, Kc, idx_dist=dist, with_mu=mu, outlier_frac=0.01), M, seed=N + K + M)
+    y, _ = run_layer(L, "gemv")
+    rel, fwd = errors(y, oracle_y(L), L)
+    assert rel <= TOL_GEMV and fwd <= TOL_GEMV, (rel, fwd)
+
+
+@pytest.mark.parametrize("config", [1, 2, 3])
+def test_gemv_parity_benchmark_configs(config):
+    """Full-size layers of the benchmark configs, every output compared (the oracle needs seconds)."""
+    cfg = wl.CONFIGS[config]
+    seen = set()
+    for lid, spec in enumerate(cfg["layers"]):
+        if (spec.N, spec.K) in seen:
+            continue
+        seen.add((spec.N, spec.K))
+        for M in cfg["M"]:
+            L = wl.make_layer(spec, M, cfg["seed"], lid)
+            y, _ = run_layer(L, "gemv")
+            rel, fwd = errors(y, oracle_y(L), L)
+            assert rel <= TOL_GEMV and fwd <= TOL_GEMV, (spec, M, rel, fwd)
+
+
+def test_gemv_is_deterministic_and_respects_bounds():
+    L = wl.make_layer(_spec(517, 4096, 16, 8192), 8, seed=3)
+    d = to_device(L)
+    M, N = 8, 517
+    guard = torch.full((M * N + 512,), 12345.0, dtype=torch.float32, device="cuda")
+    out = guard[256:256 + M * N].view(M, N)
+    btc.linear_gemv(d["x"], d["idx"], d["Cp"], d["alpha"], 16, 8192, out=out)
+    first = out.clone()
+    btc.linear_gemv(d["x"], d["idx"], d["Cp"], d["alpha"], 16, 8192, out=out)
+    torch.cuda.synchronize()
+    assert torch.equal(first, out)
+    assert bool((guard[:256] == 12345.0).all()) and bool((guard[256 + M * N:] == 12345.0).all())
+
+
+@pytest.mark.parametrize("dt", [torch.float16, torch.bfloat16])
+def test_gemv_half_outputs(dt):
+    L = wl.make_layer(_spec(300, 1024, 16, 4096), 2, seed=9)
+    y32, _ = run_layer(L, "gemv")
+    y16, _ = run_layer(L, "gemv", out_dtype=dt)
+    assert torch.equal(y16, y32.to(dt))
+
+
+def test_gemv_bf16_activations():
+    L = wl.make_layer(_spec(260, 2048, 16, 8192, x_dtype="bf16"), 4, seed=12)
+    y, _ = run_layer(L, "gemv")
+    rel, fwd = errors(y, oracle_y(L), L)
+    assert rel <= TOL_GEMV and fwd <= TOL_GEMV
+
+
+# ------------------------------------------------------------------ tensor-core path parity
+
+GEMM_SMALL = [
+    # N, K, v, Kc, M, xdt, mu
+    (128, 64, 16, 100, 128, "bf16", False),
+    (256, 256, 16, 8192, 256, "bf16", False),
+    (200, 320, 16, 4096, 130, "bf16", True),
+    (384, 1024, 16, 8192, 512, "f16", False),
+    (130, 640, 20, 65536, 300, "bf16", False),
+    (1000, 512, 8, 85, 9, "bf16", True),
+    (512, 2048, 16, 7132, 1024, "bf16", False),
+]
+
+
+@pytest.mark.parametrize("N,K,v,Kc,M,xdt,mu", GEMM_SMALL)
+def test_gemm_parity_small(N, K, v, Kc, M, xdt, mu):
+    L = wl.make_layer(_spec(N, K, v, Kc, x_dtype=xdt, with_mu=mu), M, seed=N + K + M)
+    y, _ = run_layer(L, "gemm")
+    rel, fwd = errors(y, oracle_y(L), L)
+    assert rel <= TOL_GEMM and fwd <= TOL_GEMM, (rel, fwd)
+
+
+@pytest.mark.parametrize("M", [512, 2048])
+def test_gemm_parity_benchmark_config_sampled(M):
+    """Config 4 at full size in the launch configuration the bench times; the oracle recomputes 24
+    sampled rows of y (every column of those rows), because a full fp64 product would take minutes."""
+    cfg = wl.CONFIGS[4]
+    for lid, spec in enumerate(cfg["layers"]):
+        L = wl.make_layer(spec, M, cfg["seed"], lid)
+        y, _ = run_layer(L, "gemm")
+        rows = np.unique(np.concatenate([[0, 1, 127, 128, M - 1], (np.arange(19) * 977 + 31) % M]))
+        sub = wl.LayerData(spec, len(rows), L.C_pm1, L.idx, L.alpha, L.x_bits[rows].copy(), L.mu)
+        rel, fwd = errors(y[torch.from_numpy(rows).cuda()], oracle_y(sub), sub)
+        assert rel <= TOL_GEMM and fwd <= TOL_GEMM, (spec, M, rel, fwd)
+        assert bool(torch.isfinite(y).all())
+
+
+def test_gemm_deterministic_and_bounded():
+    L = wl.make_layer(_spec(300, 1024, 16, 8192, x_dtype="bf16"), 200, seed=5)
+    d = to_device(L)
+    M, N = 200, 300
+    guard = torch.full((M * N + 512,), 777.0, dtype=torch.float32, device="cuda")
+    out = guard[256:256 + M * N].view(M, N)
+    btc.linear_gemm(d["x"], d["idx"], d["Cp"], d["alpha"], 16, 8192, out=out)
+    first = out.clone()
+    btc.linear_gemm(d["x"], d["idx"], d["Cp"], d["alpha"], 16, 8192, out=out)
+    torch.cuda.synchronize()
+    assert torch.equal(first, out)
+    assert bool((guard[:256] == 777.0).all()) and bool((guard[256 + M * N:] == 777.0).all())
