@@ -133,6 +133,11 @@ BTC_API int btc_decode_pm1(const uint16_t *idx, const uint32_t *C_packed, int N,
  * call before counting). */
 BTC_API int btc_validate_indices(const uint16_t *idx, size_t count, int Kc, int *bad_count, void *stream);
 
+/* Reads the library's device-side status word into *status_host (host pointer): BTC_OK, or
+ * BTC_ERR_TIMEOUT if a bounded wait inside a tensor-core kernel ran out since the library was
+ * loaded (the output of that launch is undefined).  This helper SYNCHRONISES the device. */
+BTC_API int btc_device_status(int *status_host);
+
 /* Bits per weight.  mode 0: log2(Kc)/v; 1: ceil(log2 Kc)/v (the paper's accounting, Section 4.3);
  * 2: 16/v (uint16 containers as stored here).  Adds scale_bits_per_row/K, and v*Kc/(N*K) for the
  * codebook when with_codebook != 0.  Host arithmetic only; returns -1 for an invalid shape. */

@@ -5,6 +5,7 @@ from .binding import (  # noqa: F401
     codebook_pack,
     codebook_pack_host,
     decode_pm1,
+    device_status,
     lib,
     linear,
     linear_gemm,

@@ -20,7 +20,7 @@ _DT = {torch.float16: BTC_F16, torch.bfloat16: BTC_BF16, torch.float32: BTC_F32}
 EXPORTS = (
     "btc_version", "btc_status_string", "btc_last_cuda_error", "btc_codebook_packed_bytes",
     "btc_codebook_pack", "btc_codebook_pack_host", "btc_linear_workspace_bytes", "btc_linear_gemv",
-    "btc_linear_gemm", "btc_decode_pm1", "btc_validate_indices", "btc_bits_per_weight",
+    "btc_linear_gemm", "btc_decode_pm1", "btc_validate_indices", "btc_bits_per_weight", "btc_device_status",
 )
 
 
@@ -61,6 +61,7 @@ def _load() -> ctypes.CDLL:
     L.btc_linear_gemm.argtypes = lin
     L.btc_decode_pm1.argtypes = [vp, vp, ci, ci, ci, ci, vp, vp]
     L.btc_validate_indices.argtypes = [vp, sz, ci, vp, vp]
+    L.btc_device_status.argtypes = [ctypes.POINTER(ctypes.c_int)]
     L.btc_bits_per_weight.restype = ctypes.c_double
     L.btc_bits_per_weight.argtypes = [ci] * 7
     return L
@@ -205,6 +206,15 @@ def validate_indices(idx, Kc: int) -> int:
     if st:
         raise BtcError(st, "btc_validate_indices")
     return int(bad.item())
+
+
+def device_status() -> int:
+    """Device-side status word (0 = ok, 7 = a bounded wait ran out).  Synchronises the device."""
+    out = ctypes.c_int(0)
+    st = lib.btc_device_status(ctypes.byref(out))
+    if st:
+        raise BtcError(st, "btc_device_status")
+    return int(out.value)
 
 
 def bits_per_weight(N, K, v, Kc, scale_bits_per_row=0, mode="container", with_codebook=False) -> float:

@@ -1,5 +1,365 @@
+// Tensor-core path: y[M,N] = x[M,K] * W^[N,K]^T with W^ = alpha * C[idx] (+ mu), for large M.
+//
+// The contraction runs on the 5th-generation tensor cores (tcgen05.mma, kind::f16, fp32 accumulators
+// in tensor memory).  Roles inside one CTA (one 128 x BM output tile, BM in {128, 256}):
+//   warp 0     TMA producer: x tiles [BM rows x 64 k] -> shared memory (128-byte swizzle)
+//   warp 1     MMA issuer: one elected thread issues tcgen05.mma for every 64-wide k step
+//   warp 2     allocates / frees tensor memory
+//   warps 4-7  decode producers: thread r expands the indices of weight row n0+r for the current
+//              64-wide k step into +-1 bf16 (or fp16) in the same swizzled K-major layout the MMA
+//              reads (A operand); afterwards the same warps run the epilogue: tcgen05.ld, scale by
+//              alpha_n in fp32 (+ mu_n * sum_k x[m,k]), store y.
+// The weight tile is the A operand (128 rows = UMMA M), x is the B operand (BM rows = UMMA N), so the
+// accumulator holds y^T: tensor-memory lane = output feature n, column = activation row m, and a warp
+// stores 32 consecutive n for one m (coalesced).  Keeping the decoded tile pure +-1 and applying the
+// row scale in the fp32 epilogue is exact for a row-wise alpha.
+//
+// Every mbarrier wait is bounded: after ~2 s of polling the CTA raises a status word, stops waiting
+// and runs to completion (the output is then undefined and btc_device_status reports the timeout).
+#include <cuda.h>
 #include "btc_internal.cuh"
+
 namespace btc {
-int launch_gemm_tcgen05(const LinearArgs &, cudaStream_t) { return BTC_ERR_UNSUPPORTED; }
-size_t gemm_tcgen05_workspace_bytes(int, int, int, int, int) { return 0; }
+
+constexpr int G_BN = 128;          // weight rows per tile (UMMA M)
+constexpr int G_BK = 64;           // k per stage: 64 x 2 bytes = one 128-byte swizzle row
+constexpr int G_THREADS = 256;
+constexpr uint32_t G_A_BYTES = G_BN * G_BK * 2;
+
+__device__ int g_gemm_status = 0;  // 0 = ok, 7 = a bounded wait ran out
+
+// ------------------------------------------------------------------------------------ PTX wrappers
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Bounded wait.  Returns false (and latches *abort_flag) when the deadline passes.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag) {
+    if (*abort_flag) return false;
+    if (mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    int spins = 0;
+    while (!mbar_try_wait(bar, parity)) {
+        if ((++spins & 63) == 0) {
+            if (*abort_flag) return false;
+            if (clock64() - t0 > 4000000000LL) {   // ~2 s at 2 GHz
+                *abort_flag = 1;
+                atomicExch(&g_gemm_status, (int)BTC_ERR_TIMEOUT);
+                return false;
+            }
+        }
+    }
+    return true;
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, int c0, int c1, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void tmem_alloc(uint32_t smem_dst, uint32_t ncols) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_dst), "r"(ncols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void umma_f16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
+        "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// K-major, 128-byte-swizzled operand tile whose rows are 128 bytes: 8-row groups are 1024 bytes apart.
+__device__ __forceinline__ uint64_t make_smem_desc(uint32_t saddr) {
+    uint64_t d = 0;
+    d |= (uint64_t)((saddr & 0x3FFFF) >> 4);          // start address, 16-byte units
+    d |= (uint64_t)1 << 16;                            // leading byte offset (unused for swizzled K-major)
+    d |= (uint64_t)(1024 >> 4) << 32;                  // stride byte offset between 8-row groups
+    d |= (uint64_t)1 << 46;                            // descriptor version for sm_100
+    d |= (uint64_t)2 << 61;                            // SWIZZLE_128B
+    return d;
+}
+
+struct GemmParams {
+    LinearArgs a;
+    const float *sumx;       // [M] row sums of x (only read when mu != nullptr)
+    int k_tiles;             // ceil(K / 64)
+};
+
+// sum_k x[m,k] in fp32, one warp per row (needed only for the mean term).
+__global__ void rowsum_kernel(const void *x, int x_dt, int M, int K, float *out)
+{
+    const int m = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    if (m >= M) return;
+    float s = 0.f;
+    for (int k = threadIdx.x & 31; k < K; k += 32) s += load_as_float(x, x_dt, (size_t)m * K + k);
+    s = warp_sum(s);
+    if ((threadIdx.x & 31) == 0) out[m] = s;
+}
+
+template <int BM, int STAGES>
+__global__ void __launch_bounds__(G_THREADS, 1)
+gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_x, const GemmParams p)
+{
+    constexpr uint32_t B_BYTES = BM * G_BK * 2;
+    constexpr uint32_t STAGE_BYTES = G_A_BYTES + B_BYTES;
+    extern __shared__ __align__(1024) unsigned char smem_raw[];
+    // carve: stages (1024-byte aligned), then barriers
+    const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    unsigned char *smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
+    uint64_t *bars = reinterpret_cast<uint64_t *>(smem_gen + (size_t)STAGES * STAGE_BYTES);
+    // bars: [0,S) full_x, [S,2S) full_w, [2S,3S) empty, [3S] accum
+    uint32_t *s_tmem = reinterpret_cast<uint32_t *>(bars + 3 * STAGES + 1);
+    volatile int *s_abort = reinterpret_cast<volatile int *>(s_tmem + 1);
+
+    const LinearArgs &a = p.a;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int n0 = blockIdx.x * G_BN;
+    const int m0 = blockIdx.y * BM;
+    const int KT = p.k_tiles;
+    const bool is_bf16 = (a.x_dt == BTC_BF16);
+
+    auto bar_full_x = [&](int s) { return smem_u32(bars + s); };
+    auto bar_full_w = [&](int s) { return smem_u32(bars + STAGES + s); };
+    auto bar_empty = [&](int s) { return smem_u32(bars + 2 * STAGES + s); };
+    const uint32_t bar_accum = smem_u32(bars + 3 * STAGES);
+
+    if (tid == 0) {
+        for (int s = 0; s < STAGES; ++s) {
+            mbar_init(bar_full_x(s), 1);
+            mbar_init(bar_full_w(s), 128);
+            mbar_init(bar_empty(s), 1);
+        }
+        mbar_init(bar_accum, 1);
+        *s_abort = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 2) tmem_alloc(smem_u32(s_tmem), BM);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_d = *s_tmem;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------ TMA producer (x tiles)
+        if (lane == 0) {
+            for (int kt = 0; kt < KT; ++kt) {
+                const int s = kt % STAGES;
+                const uint32_t ph = (kt / STAGES) & 1;
+                if (kt >= STAGES) mbar_wait(bar_empty(s), ph ^ 1, s_abort);
+                mbar_expect_tx(bar_full_x(s), B_BYTES);
+                const uint32_t dst = smem_base + s * STAGE_BYTES + G_A_BYTES;
+                tma_load_2d(dst, &tmap_x, kt * G_BK, m0, bar_full_x(s));
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            // kind::f16 instruction descriptor: D = f32, A/B = bf16 or f16, both K-major, M = 128, N = BM
+            uint32_t idesc = (1u << 4) | ((uint32_t)(BM >> 3) << 17) | ((uint32_t)(G_BN >> 4) << 24);
+            if (is_bf16) idesc |= (1u << 7) | (1u << 10);
+            for (int kt = 0; kt < KT; ++kt) {
+                const int s = kt % STAGES;
+                const uint32_t ph = (kt / STAGES) & 1;
+                mbar_wait(bar_full_x(s), ph, s_abort);
+                mbar_wait(bar_full_w(s), ph, s_abort);
+                tc_fence_after();
+                const uint32_t a_addr = smem_base + s * STAGE_BYTES;
+                const uint64_t adesc = make_smem_desc(a_addr);
+                const uint64_t bdesc = make_smem_desc(a_addr + G_A_BYTES);
+#pragma unroll
+                for (int k = 0; k < G_BK / 16; ++k)      // +32 bytes per 16-wide k step inside the swizzle row
+                    umma_f16(tmem_d, adesc + 2 * k, bdesc + 2 * k, idesc, (kt | k) ? 1u : 0u);
+                umma_commit(bar_empty(s));               // frees the stage when these MMAs have read it
+            }
+            umma_commit(bar_accum);                      // accumulator complete
+        }
+    } else if (warp >= 4) {
+        // ------------------------------------------------------------ decode producers (weights -> A tile)
+        const int r = tid - 128;                          // row inside the tile, also the TMEM lane
+        const int n = min(n0 + r, a.N - 1);
+        const uint16_t *irow = a.idx + (size_t)n * a.Kb;
+        const uint32_t one2 = is_bf16 ? 0x3F803F80u : 0x3C003C00u;
+        const int v = a.v;
+        for (int kt = 0; kt < KT; ++kt) {
+            const int s = kt % STAGES;
+            const uint32_t ph = (kt / STAGES) & 1;
+            // 64 weight bits of this row for k in [k0, k0+64), gathered from the public codeword words
+            const int k0 = kt * G_BK;
+            const int jf = k0 / v;
+            const int jl = min((k0 + G_BK - 1) / v, a.Kb - 1);
+            uint64_t win = 0;
+            for (int j = jf; j <= jl; ++j) {
+                const uint64_t w = __ldg(a.Cp + __ldg(irow + j));
+                const int off = j * v - k0;
+                win |= (off >= 0) ? (w << off) : (w >> (-off));
+            }
+            const uint64_t neg = ~win;                    // sign bit set where the weight is -1
+            if (kt >= STAGES) mbar_wait(bar_empty(s), ph ^ 1, s_abort);
+            unsigned char *arow = smem_gen + (size_t)s * STAGE_BYTES + (size_t)r * 128;
+#pragma unroll
+            for (int c = 0; c < 8; ++c) {
+                const uint32_t b = (uint32_t)(neg >> (8 * c)) & 0xFFu;
+                uint4 q;
+                q.x = one2 | ((b & 1u) << 15) | ((b & 2u) << 30);
+                q.y = one2 | ((b & 4u) << 13) | ((b & 8u) << 28);
+                q.z = one2 | ((b & 16u) << 11) | ((b & 32u) << 26);
+                q.w = one2 | ((b & 64u) << 9) | ((b & 128u) << 24);
+                *reinterpret_cast<uint4 *>(arow + ((c ^ (r & 7)) << 4)) = q;   // 128-byte swizzle
+            }
+            fence_proxy_async_smem();                     // make the generic-proxy writes visible to the MMA
+            mbar_arrive(bar_full_w(s));
+        }
+        // ------------------------------------------------------------ epilogue
+        mbar_wait(bar_accum, 0, s_abort);
+        tc_fence_after();
+        const int nrow = n0 + r;
+        const float al = __half2float(a.alpha[n]);
+        const float mu = a.mu ? __half2float(a.mu[n]) : 0.f;
+        const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
+#pragma unroll 1
+        for (int c0 = 0; c0 < BM; c0 += 32) {
+            uint32_t rr[32];
+            tmem_ld32(tmem_d + lane_base + c0, rr);
+            tmem_ld_wait();
+            if (nrow < a.N) {
+#pragma unroll
+                for (int i = 0; i < 32; ++i) {
+                    const int m = m0 + c0 + i;
+                    if (m < a.M) {
+                        float y = al * __uint_as_float(rr[i]);
+                        if (a.mu) y += mu * p.sumx[m];
+                        store_from_float(a.y, a.y_dt, (size_t)m * a.N + nrow, y);
+                    }
+                }
+            }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (*s_abort) {
+        // give copies that may still be in flight time to land before shared memory is released
+        for (int i = 0; i < 200; ++i) __nanosleep(1000);
+        __syncthreads();
+    }
+    if (warp == 2) tmem_dealloc(tmem_d, BM);
+}
+
+// ------------------------------------------------------------------------------------ host side
+typedef CUresult (*encode_tiled_fn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                    const cuuint64_t *, const cuuint32_t *, const cuuint32_t *,
+                                    CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                    CUtensorMapFloatOOBfill);
+
+static encode_tiled_fn get_encode()
+{
+    static encode_tiled_fn fn = nullptr;
+    if (!fn) {
+        void *ptr = nullptr;
+        cudaDriverEntryPointQueryResult qr;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qr) == cudaSuccess &&
+            qr == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<encode_tiled_fn>(ptr);
+    }
+    return fn;
+}
+
+template <int BM, int STAGES>
+static int launch_cfg(const CUtensorMap &tm, const GemmParams &p, cudaStream_t s)
+{
+    constexpr size_t smem = (size_t)STAGES * (G_A_BYTES + BM * G_BK * 2) + 1024 + (3 * STAGES + 1) * 8 + 16;
+    auto kern = gemm_tcgen05_kernel<BM, STAGES>;
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return cuda_fail(e);
+    dim3 grid((p.a.N + G_BN - 1) / G_BN, (p.a.M + BM - 1) / BM);
+    kern<<<grid, G_THREADS, smem, s>>>(tm, p);
+    return cuda_check_launch();
+}
+
+size_t gemm_tcgen05_workspace_bytes(int M, int, int, int, int)
+{
+    return M > 8 ? (size_t)M * sizeof(float) : 0;   // row sums of x for the mean term
+}
+
+int launch_gemm_tcgen05(const LinearArgs &a, cudaStream_t s)
+{
+    if (a.M <= 8) return BTC_ERR_UNSUPPORTED;                  // the decode path is the better kernel there
+    if (a.K % 8) return BTC_ERR_UNSUPPORTED;                   // TMA row pitch must be a multiple of 16 bytes
+    encode_tiled_fn enc = get_encode();
+    if (!enc) return BTC_ERR_UNSUPPORTED;
+    const int BM = (a.M > 128 && (long long)((a.M + 255) / 256) * ((a.N + 127) / 128) >= 120) ? 256 : 128;
+
+    CUtensorMap tm;
+    const cuuint64_t dims[2] = {(cuuint64_t)a.K, (cuuint64_t)a.M};
+    const cuuint64_t strides[1] = {(cuuint64_t)a.K * 2};
+    const cuuint32_t box[2] = {(cuuint32_t)G_BK, (cuuint32_t)BM};
+    const cuuint32_t estr[2] = {1, 1};
+    const CUtensorMapDataType dt = a.x_dt == BTC_BF16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT16;
+    CUresult r = enc(&tm, dt, 2, const_cast<void *>(a.x), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                     CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return cuda_fail(cudaErrorInvalidValue);
+
+    GemmParams p;
+    p.a = a;
+    p.k_tiles = (a.K + G_BK - 1) / G_BK;
+    p.sumx = nullptr;
+    if (a.mu) {
+        if (!a.workspace || a.workspace_bytes < (size_t)a.M * sizeof(float)) return BTC_ERR_WORKSPACE;
+        float *sx = reinterpret_cast<float *>(a.workspace);
+        rowsum_kernel<<<(a.M + 7) / 8, 256, 0, s>>>(a.x, a.x_dt, a.M, a.K, sx);
+        int rc = cuda_check_launch();
+        if (rc != BTC_OK) return rc;
+        p.sumx = sx;
+    }
+    if (BM == 256) return launch_cfg<256, 4>(tm, p, s);
+    return launch_cfg<128, 6>(tm, p, s);
+}
+
+}  // namespace btc
+
+extern "C" BTC_API int btc_device_status(int *status_host)
+{
+    if (!status_host) return BTC_ERR_NULL;
+    int v = 0;
+    cudaError_t e = cudaMemcpyFromSymbol(&v, btc::g_gemm_status, sizeof(int));
+    if (e != cudaSuccess) return btc::cuda_fail(e);
+    *status_host = v;
+    return BTC_OK;
 }
