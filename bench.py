@@ -1,0 +1,418 @@
+#!/usr/bin/env python
+"""Benchmark of the codebook-binary linear hot path on B200.
+
+One "step" = one pass of the LLaMA-2-7B-shaped decode layer set (q,k,v,o 4096x4096; gate,up
+11008x4096; down 4096x11008; v=16, Kc=8192, uniform indices, fp16 x with 0.1% outlier channels)
+at M=1 through the decode kernel: 7 launches.  Steps rotate over R distinct weight sets whose
+total size exceeds twice the L2, so every step streams its indices from HBM.  The headline value
+is effective HBM GB/s = algorithmic bytes per step / device time per step; microseconds per
+layer, the M=8 decode numbers and the tensor-core path's TFLOP/s at M=512/2048 (with a cuBLAS
+fp16 GEMM of the same shape as context) ride along in "details".
+
+  python bench.py [--gpus N] [--steps K] [--warmup W]      one JSON line on stdout
+  python bench.py --impl reference ...                      the CPU oracle on the same metric
+
+With N > 1 (torchrun) every rank runs an independent replica on its own GPU (the path has no
+exchange step); value is the sum over ranks of the work divided by the slowest rank's time.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import workloads as wl  # noqa: E402
+
+METRIC = "effective HBM GB/s at M=1 (us/layer and TFLOP/s at M=2048 in details)"
+UNIT = "GB/s"
+CONFIG_ID = 2
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return {"hbm_gbs": float(d["hbm_gbs"]), "bf16_tflops": float(d["bf16_tflops"]),
+                "bf16_tflops_sustained": float(d.get("bf16_tflops_sustained", d["bf16_tflops"])),
+                "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+def algorithmic_bytes(spec, M: int) -> int:
+    """bytes(M) = 2*N*K/v [idx] + 4*Kc [packed C] + 2*N [alpha] + 2*M*K [x] + 4*M*N [y]."""
+    return 2 * spec.N * spec.Kb + 4 * spec.Kc + 2 * spec.N + 2 * M * spec.K + 4 * M * spec.N
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.idx = gpu_index
+        self.samples = []
+        self._stop = threading.Event()
+        self._t = None
+
+    def _run(self):
+        while not self._stop.is_set():
+            try:
+                out = subprocess.run(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                      "-i", str(self.idx)], capture_output=True, text=True, timeout=5).stdout
+                parts = [p.strip() for p in out.strip().split(",")]
+                if len(parts) >= 7:
+                    self.samples.append(parts)
+            except Exception:
+                pass
+            self._stop.wait(0.05)
+
+    def __enter__(self):
+        self._t = threading.Thread(target=self._run, daemon=True)
+        self._t.start()
+        return self
+
+    def __exit__(self, *a):
+        self._stop.set()
+        self._t.join(timeout=6)
+
+    def summary(self):
+        if not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["unsampled"]}
+        mhz = sorted(int(float(s[0])) for s in self.samples)
+        reasons = set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for s in self.samples:
+            for name, val in zip(names, s[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": mhz[len(mhz) // 2], "sm_max_mhz": int(float(self.samples[0][1])),
+                "reasons": sorted(reasons), "samples": len(self.samples)}
+
+
+# ----------------------------------------------------------------------------------------------
+REF_ROW_FRACTION = 8      # the reference arm's step covers the first N/8 output rows of every layer
+
+
+def run_reference(args):
+    """The CPU oracle as it stands, timed on the host cores.  One step = the M=1 layer set restricted
+    to the first N/8 output rows of each of the 7 layers (a bounded sample: rows are independent, so
+    bytes and time both scale with the row count)."""
+    import oracle
+    cfg = wl.CONFIGS[CONFIG_ID]
+    layers = [wl.make_layer(s, 1, cfg["seed"], i) for i, s in enumerate(cfg["layers"])]
+    xs = [L.x_f64() for L in layers]
+    rows = [L.spec.N // REF_ROW_FRACTION for L in layers]
+    total_bytes = sum(2 * n * L.spec.Kb + 4 * L.spec.Kc + 2 * n + 2 * L.spec.K + 4 * n for n, L in zip(rows, layers))
+    subs = [(np.ascontiguousarray(L.idx[:n]), L.alpha[:n].copy()) for n, L in zip(rows, layers)]
+
+    def step():
+        for L, x, (idx, al) in zip(layers, xs, subs):
+            oracle.linear(x, idx, L.C_pm1, al, None)
+
+    for _ in range(min(args.warmup, 2)):
+        step()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        step()
+    dt = (time.perf_counter() - t0) / args.steps
+    val = total_bytes / dt * 1e-9
+    cores = oracle.threads()
+    line = {"impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": "config 2: LLaMA-2-7B decode layer set, M=1, 7 projections per step"},
+            "cpu_baseline": {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle",
+                             "sample": f"{args.steps} steps, each the first 1/{REF_ROW_FRACTION} of the output rows of the 7 layers "
+                                       "(fp64 dense decode + naive matmul)"},
+            "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+
+
+# ----------------------------------------------------------------------------------------------
+def run_gpu(args):
+    import torch
+    import paper_2506_12040_b200 as btc
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+        dist = dist_mod
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    peaks = measured_peaks()
+    cfg = wl.CONFIGS[CONFIG_ID]
+    specs = cfg["layers"]
+
+    def dev_layer(L):
+        dt = torch.float16 if L.spec.x_dtype == "f16" else torch.bfloat16
+        d = {"x": torch.from_numpy(L.x_bits.view(np.int16).copy()).to(dev).view(dt),
+             "idx": torch.from_numpy(L.idx.view(np.int16).copy()).to(dev),
+             "alpha": torch.from_numpy(L.alpha.view(np.int16).copy()).to(dev).view(torch.float16),
+             "Cp": btc.codebook_pack(torch.from_numpy(L.C_pm1.copy()).to(dev))}
+        return d
+
+    # ---- weight sets: R distinct copies of the 7 layers (indices re-drawn per set), > 2x L2 in total
+    step_idx_bytes = sum(2 * s.N * s.Kb for s in specs)
+    l2 = torch.cuda.get_device_properties(dev).L2_cache_size
+    R = max(2, int(np.ceil(2.2 * l2 / step_idx_bytes)))
+    base = [wl.make_layer(s, 8, cfg["seed"], i) for i, s in enumerate(specs)]
+    sets = []
+    for r in range(R):
+        layers = []
+        for i, (s, L) in enumerate(zip(specs, base)):
+            d = dev_layer(L) if r == 0 else dict(sets[0][i])
+            if r > 0:
+                idx = wl.make_indices(s.N, s.Kb, s.Kc, s.idx_dist, cfg["seed"] + 7919 * r, 16 * i + 1)
+                d["idx"] = torch.from_numpy(idx.view(np.int16)).to(dev)
+            layers.append(d)
+        sets.append(layers)
+
+    def make_runner(M):
+        outs = [[torch.empty((M, s.N), dtype=torch.float32, device=dev) for s in specs] for _ in range(R)]
+        xs = [sets[0][i]["x"][:M].contiguous() for i in range(len(specs))]
+
+        def step(r):
+            for i, s in enumerate(specs):
+                d = sets[r][i]
+                btc.linear_gemv(xs[i], d["idx"], d["Cp"], d["alpha"], s.v, s.Kc, out=outs[r][i])
+        return step, outs, xs
+
+    def time_steps(step, steps, warmup):
+        stream = torch.cuda.Stream(device=dev)
+        with torch.cuda.stream(stream):
+            for w in range(max(warmup, 3)):
+                step(w % R)
+            stream.synchronize()
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=stream):
+                for k in range(steps):
+                    step(k % R)
+            g.replay()                      # one untimed replay (graph upload)
+            stream.synchronize()
+            if dist is not None:
+                dist.barrier()
+            torch.cuda.synchronize()
+            e0 = torch.cuda.Event(enable_timing=True)
+            e1 = torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            g.replay()
+            e1.record(stream)
+            stream.synchronize()
+            torch.cuda.synchronize()
+        return e0.elapsed_time(e1) * 1e-3   # seconds for `steps` steps
+
+    # ---- headline: M = 1
+    step1, outs1, xs1 = make_runner(1)
+    bytes_step = sum(algorithmic_bytes(s, 1) for s in specs)
+    with ClockSampler(local) as clk:
+        t_total = time_steps(step1, args.steps, args.warmup)
+        # keep the sampler busy for at least a few samples on very short runs
+        t_end = time.time() + 0.3
+        while time.time() < t_end:
+            step1(0)
+        torch.cuda.synchronize()
+    clocks = clk.summary()
+    t_max = t_total
+    if dist is not None:
+        tt = torch.tensor([t_total], device=dev, dtype=torch.float64)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        t_max = float(tt.item())
+    ms_per_step = t_max / args.steps * 1e3
+    value = world * bytes_step / (t_max / args.steps) * 1e-9
+    launches = args.steps * len(specs)
+    avg_launch_s = t_total / launches
+    bytes_per_launch = bytes_step / len(specs)
+    achieved = bytes_per_launch / avg_launch_s * 1e-9
+
+    details = {"us_per_layer_M1": avg_launch_s * 1e6, "weight_sets": R,
+               "per_shape_M1": {}, "hbm_nominal_gbs": 8000.0,
+               "frac_of_nominal": achieved / 8000.0}
+
+    if rank == 0 and not args.quick:
+        # ---- per shape, M in {1, 8}, each over its own rotating sets
+        def time_shape(i, M, reps=200):
+            s = specs[i]
+            x = sets[0][i]["x"][:M].contiguous()
+            outs = [torch.empty((M, s.N), dtype=torch.float32, device=dev) for _ in range(R)]
+            rr = [r for r in range(R)]
+            # same-shape layers of other slots double the number of distinct index copies
+            same = [j for j, t in enumerate(specs) if (t.N, t.K) == (s.N, s.K)]
+
+            def one(k):
+                d = sets[rr[k % R]][same[(k // R) % len(same)]]
+                btc.linear_gemv(x, d["idx"], d["Cp"], d["alpha"], s.v, s.Kc, out=outs[k % R])
+            stream = torch.cuda.Stream(device=dev)
+            with torch.cuda.stream(stream):
+                for k in range(5):
+                    one(k)
+                stream.synchronize()
+                g = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(g, stream=stream):
+                    for k in range(reps):
+                        one(k)
+                g.replay()
+                stream.synchronize()
+                e0 = torch.cuda.Event(enable_timing=True)
+                e1 = torch.cuda.Event(enable_timing=True)
+                e0.record(stream)
+                g.replay()
+                e1.record(stream)
+                stream.synchronize()
+            us = e0.elapsed_time(e1) * 1e3 / reps
+            b = algorithmic_bytes(s, M)
+            return {"us": us, "GBps": b / us * 1e-3, "frac_measured": b / us * 1e-3 / peaks["hbm_gbs"]}
+        seen = set()
+        for i, s in enumerate(specs):
+            if (s.N, s.K) in seen:
+                continue
+            seen.add((s.N, s.K))
+            for M in (1, 8):
+                details.setdefault(f"per_shape_M{M}", {})[f"{s.N}x{s.K}"] = time_shape(i, M)
+
+        # ---- tensor-core path, config 4 shapes, with a cuBLAS fp16 GEMM of the same shape as context
+        gem = {}
+        c4 = wl.CONFIGS[4]
+        flush = torch.empty(int(1.5 * l2), dtype=torch.uint8, device=dev)
+        ws = torch.empty(1 << 20, dtype=torch.uint8, device=dev)
+        for li, s in enumerate(c4["layers"]):
+            L = wl.make_layer(s, 1, c4["seed"], li)
+            d = dev_layer(L)
+            for M in c4["M"]:
+                xb = torch.from_numpy(wl.make_x(M, s.K, "bf16", c4["seed"], 16 * li + 3).view(np.int16)).to(dev).view(torch.bfloat16)
+                y = torch.empty((M, s.N), dtype=torch.float32, device=dev)
+                wd = torch.randn(s.N, s.K, device=dev, dtype=torch.float16)
+                xh = xb.to(torch.float16)
+
+                def ours():
+                    btc.linear_gemm(xb, d["idx"], d["Cp"], d["alpha"], s.v, s.Kc, out=y, workspace=ws)
+
+                def cublas():
+                    torch.matmul(xh, wd.t())
+                res = {}
+                for name, fn in (("btc", ours), ("cublas_fp16", cublas)):
+                    for _ in range(3):
+                        fn()
+                    ts = []
+                    for _ in range(7):
+                        flush.zero_()
+                        e0 = torch.cuda.Event(enable_timing=True)
+                        e1 = torch.cuda.Event(enable_timing=True)
+                        e0.record()
+                        fn()
+                        e1.record()
+                        torch.cuda.synchronize()
+                        ts.append(e0.elapsed_time(e1) * 1e3)
+                    us = float(np.median(ts))
+                    res[name] = {"us": us, "TFLOPs": 2.0 * M * s.N * s.K / us * 1e-6}
+                res["frac_bf16_peak_measured"] = res["btc"]["TFLOPs"] / peaks["bf16_tflops"]
+                gem[f"M{M}_{s.N}x{s.K}"] = res
+        details["gemm"] = gem
+        details["device_status"] = btc.device_status()
+
+    # ---- end to end: host buffers in, host buffers out, through the same calls
+    e2e = None
+    if rank == 0 or world > 1:
+        xh = [x.cpu().pin_memory() for x in xs1]
+        yh = [torch.empty((1, s.N), dtype=torch.float32).pin_memory() for s in specs]
+        xd = [torch.empty_like(x) for x in xs1]
+        stream = torch.cuda.Stream(device=dev)
+        n_e2e = max(20, min(args.steps, 200))
+
+        def e2e_step(r):
+            for i, s in enumerate(specs):
+                xd[i].copy_(xh[i], non_blocking=True)
+                d = sets[r][i]
+                btc.linear_gemv(xd[i], d["idx"], d["Cp"], d["alpha"], s.v, s.Kc, out=outs1[r][i])
+                yh[i].copy_(outs1[r][i], non_blocking=True)
+        with torch.cuda.stream(stream):
+            for w in range(3):
+                e2e_step(w % R)
+            stream.synchronize()
+            e0 = torch.cuda.Event(enable_timing=True)
+            e1 = torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            for k in range(n_e2e):
+                e2e_step(k % R)
+            e1.record(stream)
+            stream.synchronize()
+        te = e0.elapsed_time(e1) * 1e-3 / n_e2e
+        if dist is not None:
+            tt = torch.tensor([te], device=dev, dtype=torch.float64)
+            dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+            te = float(tt.item())
+        e2e = {"value": world * bytes_step / te * 1e-9, "unit": UNIT,
+               "h2d_bytes_per_step": int(sum(x.numel() * 2 for x in xs1)),
+               "d2h_bytes_per_step": int(sum(4 * s.N for s in specs)),
+               "note": "x from pinned host memory and y back to host every layer; weights resident on the device"}
+
+    # ---- CPU oracle on the host cores (rank 0, N = 1 only): one full M=1 step, repeated for ~10 s
+    cpu = None
+    if rank == 0 and world == 1:
+        import oracle
+        layers = [wl.make_layer(s, 1, cfg["seed"], i) for i, s in enumerate(specs)]
+        xs64 = [L.x_f64() for L in layers]
+        oracle.linear(xs64[0], layers[0].idx, layers[0].C_pm1, layers[0].alpha)
+        n_rep, t0 = 0, time.perf_counter()
+        while True:
+            for L, x in zip(layers, xs64):
+                oracle.linear(x, L.idx, L.C_pm1, L.alpha)
+            n_rep += 1
+            if time.perf_counter() - t0 > 10.0 or n_rep >= 50:
+                break
+        dt = (time.perf_counter() - t0) / n_rep
+        cpu = {"value": bytes_step / dt * 1e-9, "unit": UNIT, "cores": oracle.threads(), "kind": "oracle",
+               "sample": f"{n_rep} full M=1 steps (7 layers each), fp64 dense decode + naive matmul"}
+
+    if rank == 0:
+        peak = peaks["hbm_gbs"]
+        line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+                "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
+                "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+                "config": {"workload": "config 2: LLaMA-2-7B decode layer set (7 projections, v=16, Kc=8192), M=1",
+                           "cold_l2": f"inputs larger than L2: {R} weight sets x {step_idx_bytes / 1e6:.1f} MB of indices",
+                           "timing": "one CUDA graph of all steps, CUDA events on the launching stream",
+                           "multi_gpu": "replicas only"},
+                "clocks": clocks, "e2e": e2e, "gpu_launches": launches,
+                "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                             "frac": achieved / peak, "traffic": None, "peak_source": f"of {peaks['source']}",
+                             "kernel": "gemv_decode_kernel", "bytes_per_launch": bytes_per_launch,
+                             "avg_launch_us": avg_launch_s * 1e6},
+                "cpu_baseline": cpu, "details": details}
+        print(json.dumps(line))
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="btc", choices=["btc", "reference"])
+    ap.add_argument("--quick", action="store_true", help="headline only (skip per-shape and GEMM details)")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        if int(os.environ.get("RANK", "0")) == 0:
+            run_reference(args)
+        return
+    run_gpu(args)
+
+
+if __name__ == "__main__":
+    main()
