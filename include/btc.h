@@ -123,6 +123,34 @@ BTC_API int btc_linear_gemm(const void *x, int x_dtype, const uint16_t *idx, con
                     int M, int N, int K, int v, int Kc, void *workspace, size_t workspace_bytes,
                     void *stream);
 
+/* ---- btc_linear_gemm for callers that cannot allocate device memory ---------------------------
+ * (No counterpart in the paper: this is a packaging variant of btc_linear_gemm, same arithmetic.)
+ *
+ * Some callers have no way to hand over a workspace: code that runs where cudaMalloc is forbidden
+ * (inside a region that must not touch the allocator, a plugin whose host gives it only its input
+ * and output buffers, a process whose memory was carved up in advance).  For them the scratch that
+ * btc_linear_gemm needs for the mean term (the fp32 row sums of x, 4*M bytes) lives in a fixed
+ * array inside the library's device image, BTC_STATIC_SCRATCH_BYTES long.  Every GPU that loads
+ * the library holds that array until the process exits.
+ *
+ * Arguments are those of btc_linear_gemm without workspace / workspace_bytes.  Differences:
+ *   - Needs btc_linear_workspace_bytes(M, N, K, v, Kc) <= BTC_STATIC_SCRATCH_BYTES, i.e.
+ *     M <= BTC_STATIC_SCRATCH_BYTES / 4 rows of x; larger M returns BTC_ERR_WORKSPACE and nothing
+ *     is launched.  T must be NULL (the transform needs M*K*2 bytes more): BTC_ERR_UNSUPPORTED.
+ *   - The first call on each device looks up the array's device address (no allocation, no
+ *     launch) and caches it; make that first call outside any stream capture.  The device that is
+ *     current at the call is the one used, as for every other entry point.
+ *   - All calls on one device share the one array.  Two calls whose kernels may overlap on the
+ *     GPU (different streams, no ordering between them) race on it and may corrupt each other's
+ *     mean term; order them on one stream or with events.  The array keeps the previous call's
+ *     contents; each call overwrites the part it reads, so nothing has to be cleared.
+ *   - Calls no cudaMalloc / cudaFree and no allocating library routine, on any call.
+ */
+#define BTC_STATIC_SCRATCH_BYTES 65536
+BTC_API int btc_linear_gemm_static_scratch(const void *x, int x_dtype, const uint16_t *idx,
+                    const uint32_t *C_packed, const void *alpha, const void *mu, const btc_transform *T,
+                    void *y, int y_dtype, int M, int N, int K, int v, int Kc, void *stream);
+
 /* ---- helpers (not on the hot path) --------------------------------------------------------- */
 
 /* B^[n, j*v + t] = +1 / -1 as int8 [N, K]: the decoded sign matrix, for bit-exact checks. */

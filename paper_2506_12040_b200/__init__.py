@@ -9,6 +9,7 @@ from .binding import (  # noqa: F401
     lib,
     linear,
     linear_gemm,
+    linear_gemm_static_scratch,
     linear_gemv,
     linear_workspace_bytes,
     validate_indices,

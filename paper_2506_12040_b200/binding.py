@@ -20,7 +20,7 @@ _DT = {torch.float16: BTC_F16, torch.bfloat16: BTC_BF16, torch.float32: BTC_F32}
 EXPORTS = (
     "btc_version", "btc_status_string", "btc_last_cuda_error", "btc_codebook_packed_bytes",
     "btc_codebook_pack", "btc_codebook_pack_host", "btc_linear_workspace_bytes", "btc_linear_gemv",
-    "btc_linear_gemm", "btc_decode_pm1", "btc_validate_indices", "btc_bits_per_weight", "btc_device_status",
+    "btc_linear_gemm", "btc_linear_gemm_static_scratch", "btc_decode_pm1", "btc_validate_indices", "btc_bits_per_weight", "btc_device_status",
 )
 
 
@@ -59,6 +59,7 @@ def _load() -> ctypes.CDLL:
     lin = [vp, ci, vp, vp, vp, vp, ctypes.POINTER(BtcTransform), vp, ci, ci, ci, ci, ci, ci, vp, sz, vp]
     L.btc_linear_gemv.argtypes = lin
     L.btc_linear_gemm.argtypes = lin
+    L.btc_linear_gemm_static_scratch.argtypes = lin[:14] + [vp]
     L.btc_decode_pm1.argtypes = [vp, vp, ci, ci, ci, ci, vp, vp]
     L.btc_validate_indices.argtypes = [vp, sz, ci, vp, vp]
     L.btc_device_status.argtypes = [ctypes.POINTER(ctypes.c_int)]
@@ -179,6 +180,30 @@ def linear_gemm(x, idx, C_packed, alpha, v, Kc, mu=None, out=None, out_dtype=tor
     """Tensor-core path (any M, built for large M)."""
     return _linear(lib.btc_linear_gemm, "btc_linear_gemm", x, idx, C_packed, alpha, v, Kc, mu, out, out_dtype,
                    workspace, transform)
+
+
+STATIC_SCRATCH_BYTES = 65536
+
+
+def linear_gemm_static_scratch(x, idx, C_packed, alpha, v, Kc, mu=None, out=None):
+    """btc_linear_gemm for callers that cannot allocate device memory: the scratch of the mean term is a
+    fixed array inside the library (STATIC_SCRATCH_BYTES, so M <= 16384), shared by all calls on a device.
+    `out` must be given by such a caller; when it is None this wrapper allocates it with torch, the
+    library itself still allocates nothing.  Calls that may overlap on the GPU race on the array."""
+    for t, n in ((x, "x"), (idx, "idx"), (C_packed, "C_packed"), (alpha, "alpha")):
+        _dev(t, n)
+    M, K = x.shape
+    N, Kb = idx.shape
+    if Kb * v != K or alpha.numel() != N or C_packed.numel() != packed_words(Kc, v):
+        raise ValueError("shape mismatch between x, idx, v, alpha and C_packed")
+    if out is None:
+        out = torch.empty((M, N), dtype=torch.float32, device=x.device)
+    st = lib.btc_linear_gemm_static_scratch(x.data_ptr(), _DT[x.dtype], idx.data_ptr(), C_packed.data_ptr(),
+                                            alpha.data_ptr(), _ptr(mu), None, out.data_ptr(), _DT[out.dtype],
+                                            M, N, K, v, Kc, _stream())
+    if st:
+        raise BtcError(st, "btc_linear_gemm_static_scratch")
+    return out
 
 
 def linear(x, idx, C_packed, alpha, v, Kc, **kw):

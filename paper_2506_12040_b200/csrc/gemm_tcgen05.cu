@@ -363,3 +363,57 @@ extern "C" BTC_API int btc_device_status(int *status_host)
     *status_host = v;
     return BTC_OK;
 }
+
+// ---------------------------------------------------------------------------------------------
+// btc_linear_gemm for callers that cannot allocate: the row-sum scratch of the mean term lives in
+// a fixed array of the device image instead of a caller-supplied workspace.
+//
+// In host code `g_static_scratch` is only a handle for the runtime, not a device address, so it
+// must never be passed to a kernel as is; its address on the current device comes from
+// cudaGetSymbolAddress, looked up once per device and cached.
+#include <mutex>
+
+namespace btc {
+
+static __device__ __align__(256) unsigned char g_static_scratch[BTC_STATIC_SCRATCH_BYTES];
+
+constexpr int MAX_DEVICES = 64;
+static void *g_static_scratch_addr[MAX_DEVICES] = {};
+static std::mutex g_static_scratch_mutex;
+
+// Device address of g_static_scratch on the current device (cached per device); no allocation.
+static int static_scratch_address(void **out)
+{
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return cuda_fail(e);
+    if (dev < 0 || dev >= MAX_DEVICES) return BTC_ERR_UNSUPPORTED;
+    std::lock_guard<std::mutex> lock(g_static_scratch_mutex);
+    if (!g_static_scratch_addr[dev]) {
+        void *p = nullptr;
+        e = cudaGetSymbolAddress(&p, g_static_scratch);
+        if (e != cudaSuccess) return cuda_fail(e);
+        if (!p) return cuda_fail(cudaErrorInvalidSymbol);
+        g_static_scratch_addr[dev] = p;
+    }
+    *out = g_static_scratch_addr[dev];
+    return BTC_OK;
+}
+
+}  // namespace btc
+
+extern "C" BTC_API int btc_linear_gemm_static_scratch(const void *x, int x_dtype, const uint16_t *idx,
+                                                      const uint32_t *C_packed, const void *alpha,
+                                                      const void *mu, const btc_transform *T, void *y,
+                                                      int y_dtype, int M, int N, int K, int v, int Kc,
+                                                      void *stream)
+{
+    if (T) return BTC_ERR_UNSUPPORTED;
+    if (v < 1 || v > 32 || Kc < 1 || Kc > 65536 || M < 1 || N < 1 || K < 1 || K % v) return BTC_ERR_SHAPE;
+    if (btc_linear_workspace_bytes(M, N, K, v, Kc) > (size_t)BTC_STATIC_SCRATCH_BYTES) return BTC_ERR_WORKSPACE;
+    void *scratch = nullptr;
+    const int rc = btc::static_scratch_address(&scratch);
+    if (rc != BTC_OK) return rc;
+    return btc_linear_gemm(x, x_dtype, idx, C_packed, alpha, mu, nullptr, y, y_dtype, M, N, K, v, Kc, scratch,
+                           (size_t)BTC_STATIC_SCRATCH_BYTES, stream);
+}
