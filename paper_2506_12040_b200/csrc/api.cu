@@ -65,7 +65,10 @@ static int run_linear(Path path, const void *x, int x_dt, const uint16_t *idx, c
     }
 
     rc = BTC_ERR_UNSUPPORTED;
-    if (path == PATH_GEMV) rc = launch_gemv_decode(a, s);
+    if (path == PATH_GEMV || M <= 8) {
+        rc = launch_gemv_imma(&a, 1, s);
+        if (rc == BTC_ERR_UNSUPPORTED) rc = launch_gemv_decode(a, s);
+    }
     else rc = launch_gemm_tcgen05(a, s);
     if (rc == BTC_ERR_UNSUPPORTED) {
         if (path == PATH_GEMM && M <= 8) rc = launch_gemv_decode(a, s);
@@ -100,7 +103,7 @@ extern "C" int btc_last_cuda_error(void) { return g_last_cuda_error; }
 extern "C" size_t btc_codebook_packed_bytes(int Kc, int v)
 {
     if (v < 1 || v > 32 || Kc < 1 || Kc > 65536) return 0;
-    return (size_t)((Kc + 3) / 4 * 4) * 8;
+    return (size_t)((Kc + 3) / 4 * 4) * 12;
 }
 
 extern "C" size_t btc_linear_workspace_bytes(int M, int N, int K, int v, int Kc)

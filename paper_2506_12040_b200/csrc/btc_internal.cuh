@@ -40,6 +40,12 @@ size_t gemv_decode_workspace_bytes(int M, int N, int K, int v, int Kc);
 int launch_gemm_tcgen05(const LinearArgs &a, cudaStream_t s);
 size_t gemm_tcgen05_workspace_bytes(int M, int N, int K, int v, int Kc);
 
+// gemv_imma.cu: integer-MMA decode path; runs up to IM_MAXP independent layers (M <= 8 each) in one launch.
+// Returns BTC_ERR_UNSUPPORTED when a shape is outside what it covers (nothing is launched then).
+constexpr int IM_MAXP = 8;
+int launch_gemv_imma(const LinearArgs *problems, int count, cudaStream_t s);
+int imma_status_read(int *out);
+
 // transform.cu: x' = x * D * (P1 (x) P2) into xt (same dtype/shape as x).
 int launch_transform(const void *x, int x_dt, const btc_transform &T, void *xt, int M, int K,
                      cudaStream_t s);

@@ -360,7 +360,10 @@ extern "C" BTC_API int btc_device_status(int *status_host)
     int v = 0;
     cudaError_t e = cudaMemcpyFromSymbol(&v, btc::g_gemm_status, sizeof(int));
     if (e != cudaSuccess) return btc::cuda_fail(e);
-    *status_host = v;
+    int v2 = 0;
+    const int rc = btc::imma_status_read(&v2);
+    if (rc != BTC_OK) return rc;
+    *status_host = v ? v : v2;
     return BTC_OK;
 }
 

@@ -16,6 +16,17 @@ __host__ __device__ inline uint32_t mma_layout_word(uint32_t pub, int v)
     return w;
 }
 
+// Kernel-private word of one centroid for the integer-MMA decode path ("byte-lane layout"): the bit of
+// weight t sits at bit (t >> 2) of byte (t & 3), so `word & (0x01010101 << c)` is four unsigned bytes
+// {0 or 2^c} for the weights 4c .. 4c+3.
+__host__ __device__ inline uint32_t byte_lane_word(uint32_t pub, int v)
+{
+    uint32_t w = 0;
+    for (int t = 0; t < v; ++t)
+        if ((pub >> t) & 1u) w |= 1u << (8 * (t & 3) + (t >> 2));
+    return w;
+}
+
 // bit t of out[k] = (C[k][t] + 1) / 2, with C >= 0 read as +1; private words at out[Kc4 + k].
 __global__ void pack_codebook_kernel(const int8_t *__restrict__ C, int Kc, int v, uint32_t *__restrict__ out)
 {
@@ -28,6 +39,7 @@ __global__ void pack_codebook_kernel(const int8_t *__restrict__ C, int Kc, int v
             if (C[(size_t)k * v + t] >= 0) w |= 1u << t;
     out[k] = w;
     out[Kc4 + k] = mma_layout_word(w, v);
+    out[2 * Kc4 + k] = byte_lane_word(w, v);
 }
 
 // One thread per (row, block): expands the centroid word into v int8 signs.
@@ -77,6 +89,7 @@ extern "C" int btc_codebook_pack_host(const int8_t *C, int Kc, int v, uint32_t *
                 if (C[(size_t)k * v + t] >= 0) w |= 1u << t;
         out[k] = w;
         out[Kc4 + k] = mma_layout_word(w, v);
+        out[2 * Kc4 + k] = byte_lane_word(w, v);
     }
     return BTC_OK;
 }
