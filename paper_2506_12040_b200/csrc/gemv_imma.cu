@@ -147,11 +147,16 @@ __host__ __device__ inline ImSmem im_smem_layout(int tab_bytes, int part_ints)
     return L;
 }
 
-// Balanced base-256 digit d (of D) of X: X = sum_d dig_d * 256^d, dig_d in [-128, 127] for d < D-1.
-__device__ __forceinline__ int im_digit(int X, int d, int D)
+// Two packed fp16 (dt = BTC_F16) or bf16 numbers -> two floats.
+__device__ __forceinline__ void im_unpack2(uint32_t w, int dt, float &lo, float &hi)
 {
-    for (int i = 0; i < d; ++i) X = (X - (int)(signed char)(X & 0xff)) >> 8;
-    return (d == D - 1) ? X : (int)(signed char)(X & 0xff);
+    if (dt == BTC_F16) {
+        const float2 f = __half22float2(*reinterpret_cast<const __half2 *>(&w));
+        lo = f.x; hi = f.y;
+    } else {
+        lo = __uint_as_float(w << 16);
+        hi = __uint_as_float(w & 0xffff0000u);
+    }
 }
 
 template <int NCLS, int NQ, int NM>
@@ -322,13 +327,26 @@ gemv_imma_kernel(const __grid_constant__ ImBatch batch)
             const int cmax = P.ncls - 1;
             const int PBITS = 8 * D - 2 - cmax;                // |X| <= 2^PBITS
 
-            // ---- quantisation of x: per-row scale, integer row sums
-            for (int m = 0; m < M; ++m) {
-                float a = 0.f;
-                for (int k = ctid; k < K; k += CT) a = fmaxf(a, fabsf(load_as_float(P.x, P.x_dt, (size_t)m * K + k)));
+            // ---- quantisation of x, step 1: per-row scale from the largest magnitude (16-byte loads)
+            {
+                const int nvec = K >> 3;                        // K % 16 == 0 (checked on the host)
+                for (int m = 0; m < M; ++m) {
+                    float a = 0.f;
+                    const uint4 *xr = reinterpret_cast<const uint4 *>(reinterpret_cast<const uint16_t *>(P.x) + (size_t)m * K);
+                    for (int i = ctid; i < nvec; i += CT) {
+                        const uint4 q4 = __ldg(xr + i);
+                        const uint32_t wds[4] = {q4.x, q4.y, q4.z, q4.w};
 #pragma unroll
-                for (int o = 16; o > 0; o >>= 1) a = fmaxf(a, __shfl_xor_sync(0xffffffffu, a, o));
-                if (lane == 0) s_redf[warp * 8 + m] = a;
+                        for (int j = 0; j < 4; ++j) {
+                            float lo, hi;
+                            im_unpack2(wds[j], P.x_dt, lo, hi);
+                            a = fmaxf(a, fmaxf(fabsf(lo), fabsf(hi)));
+                        }
+                    }
+#pragma unroll
+                    for (int o = 16; o > 0; o >>= 1) a = fmaxf(a, __shfl_xor_sync(0xffffffffu, a, o));
+                    if (lane == 0) s_redf[warp * 8 + m] = a;
+                }
             }
             im_named_bar(1, CT);
             if (ctid < M) {
@@ -339,17 +357,65 @@ gemv_imma_kernel(const __grid_constant__ ImBatch batch)
                 slot[ctid] = (a > 0.f) ? ldexp(1.0, e - PBITS) : 1.0;
             }
             im_named_bar(1, CT);
-            float scale[MAXM];
+
+            // ---- step 2: B fragments of this lane (blocks wbase + 16 q + 4 t + e, classes c, column
+            //      g + 8 nm = m * D + d) and the integer row sums, from 8-byte loads of x
+            const int wbase = warp * 16 * nq;
+            uint32_t breg[NQ][4][NCLS][NM];
+            long long xsum[NM];
 #pragma unroll
-            for (int m = 0; m < MAXM; ++m) scale[m] = (m < M) ? (float)(1.0 / slot[m]) : 0.f;
-            for (int m = 0; m < M; ++m) {
-                double sacc = 0.0;
-                const float sc = (float)(1.0 / slot[m]);
-                for (int k = ctid; k < K; k += CT)
-                    sacc += (double)__float2int_rn(load_as_float(P.x, P.x_dt, (size_t)m * K + k) * sc);
+            for (int nm = 0; nm < NM; ++nm) {
+                xsum[nm] = 0;
+                const int col = g + 8 * nm;
+                const int m = col / D, d = col - m * D;
+                const bool colvalid = m < M;
+                const float sc = colvalid ? (float)(1.0 / slot[colvalid ? m : 0]) : 0.f;
+                const uint16_t *xrow = reinterpret_cast<const uint16_t *>(P.x) + (size_t)(colvalid ? m : 0) * K;
+                const uint32_t sel = (uint32_t)d | ((uint32_t)(4 + d) << 4);
+                const uint32_t flip = (d < D - 1) ? 0x80808080u : 0u;
+                constexpr int BIAS = (D == 4) ? 0x00808080 : 0x00008080;
 #pragma unroll
-                for (int o = 16; o > 0; o >>= 1) sacc += __shfl_xor_sync(0xffffffffu, sacc, o);
-                if (lane == 0) s_redd[warp * 8 + m] = sacc;
+                for (int q = 0; q < NQ; ++q) {
+                    uint2 raw[4][NCLS];
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const int jb = wbase + 16 * q + 4 * t + e;
+                        const bool bvalid = colvalid && (q < nq) && (jb < Kb);
+#pragma unroll
+                        for (int c = 0; c < NCLS; ++c) {
+                            raw[e][c] = make_uint2(0u, 0u);
+                            if (bvalid && c <= cmax)
+                                raw[e][c] = __ldg(reinterpret_cast<const uint2 *>(xrow + (size_t)jb * v + 4 * c));
+                        }
+                    }
+#pragma unroll
+                    for (int e = 0; e < 4; ++e)
+#pragma unroll
+                        for (int c = 0; c < NCLS; ++c) {
+                            float f0, f1, f2, f3;
+                            im_unpack2(raw[e][c].x, P.x_dt, f0, f1);
+                            im_unpack2(raw[e][c].y, P.x_dt, f2, f3);
+                            const int X0 = __float2int_rn(f0 * sc), X1 = __float2int_rn(f1 * sc);
+                            const int X2 = __float2int_rn(f2 * sc), X3 = __float2int_rn(f3 * sc);
+                            if (d == 0) xsum[nm] += (long long)(X0 + X1) + (long long)(X2 + X3);
+                            const int sh = 1 << ((c <= cmax) ? (cmax - c) : 0);
+                            // balanced digit d of Y: byte d of (Y + BIAS), with 0x80 flipped back below the top digit
+                            const uint32_t y01 = __byte_perm((uint32_t)(X0 * sh + BIAS), (uint32_t)(X1 * sh + BIAS), sel);
+                            const uint32_t y23 = __byte_perm((uint32_t)(X2 * sh + BIAS), (uint32_t)(X3 * sh + BIAS), sel);
+                            const bool on = colvalid && (c <= cmax);
+                            breg[q][e][c][nm] = on ? (__byte_perm(y01, y23, 0x5410) ^ flip) : 0u;
+                        }
+                }
+            }
+            // integer row sums: the four lanes (t) of column m * D hold disjoint blocks of row m
+#pragma unroll
+            for (int nm = 0; nm < NM; ++nm) {
+                const int col = g + 8 * nm;
+                const int m = col / D, d = col - m * D;
+                long long sacc = xsum[nm];
+                sacc += __shfl_xor_sync(0xffffffffu, sacc, 1);
+                sacc += __shfl_xor_sync(0xffffffffu, sacc, 2);
+                if (t == 0 && d == 0 && m < M) s_redd[warp * 8 + m] = (double)sacc;
             }
             im_named_bar(1, CT);
             if (ctid < M) {
@@ -359,40 +425,6 @@ gemv_imma_kernel(const __grid_constant__ ImBatch batch)
             }
             // (the epilogue warp reads the slot only after a partial-sum barrier that follows this point)
 
-            // ---- B fragments of this lane: blocks wbase + 16 q + 4 t + e, classes c, column group nm
-            const int wbase = warp * 16 * nq;
-            uint32_t breg[NQ][4][NCLS][NM];
-#pragma unroll
-            for (int q = 0; q < NQ; ++q) {
-#pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    const int jb = wbase + 16 * q + 4 * t + e;
-                    const bool bvalid = (q < nq) && (jb < Kb);
-#pragma unroll
-                    for (int c = 0; c < NCLS; ++c) {
-#pragma unroll
-                        for (int nm = 0; nm < NM; ++nm) {
-                            const int col = g + 8 * nm;
-                            const int m = col / D, d = col - m * D;
-                            uint32_t packed = 0;
-                            if (bvalid && m < M && c <= cmax) {
-                                float sc = 0.f;
-#pragma unroll
-                                for (int mm = 0; mm < MAXM; ++mm) if (mm == m) sc = scale[mm];
-#pragma unroll
-                                for (int b = 0; b < 4; ++b) {
-                                    const int k = jb * v + 4 * c + b;
-                                    int X = 0;
-                                    if (4 * c + b < v) X = __float2int_rn(load_as_float(P.x, P.x_dt, (size_t)m * K + k) * sc);
-                                    const int dig = im_digit(X * (1 << (cmax - c)), d, D);
-                                    packed |= (uint32_t)(dig & 0xff) << (8 * b);
-                                }
-                            }
-                            breg[q][e][c][nm] = packed;
-                        }
-                    }
-                }
-            }
             if (tab_smem && !im_mbar_wait(bar_tabfull, seg & 1, s_abort)) break;
             const uint32_t *tab = tab_smem ? s_tab : P.tab;
 
@@ -556,7 +588,7 @@ int launch_gemv_imma(const LinearArgs *problems, int count, cudaStream_t s)
     for (int i = 0; i < count; ++i) {
         const LinearArgs &a = problems[i];
         ImProblem &p = b.p[i];
-        if (a.M < 1 || a.M > 8 || a.Kb % 4 != 0 || a.v > 20) return BTC_ERR_UNSUPPORTED;
+        if (a.M < 1 || a.M > 8 || a.Kb % 4 != 0 || a.v % 4 != 0 || a.v > 20) return BTC_ERR_UNSUPPORTED;
         if ((long long)a.Kb * 32 > IM_STAGE_BYTES) return BTC_ERR_UNSUPPORTED;      // one 16-row tile must fit a stage
         p.x = a.x; p.idx = a.idx; p.alpha = a.alpha; p.mu = a.mu; p.y = a.y;
         const int Kc4 = (a.Kc + 3) / 4 * 4;
