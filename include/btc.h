@@ -123,6 +123,35 @@ BTC_API int btc_linear_gemm(const void *x, int x_dtype, const uint16_t *idx, con
                     int M, int N, int K, int v, int Kc, void *workspace, size_t workspace_bytes,
                     void *stream);
 
+/* ---- several independent layers in one launch (decode path) ---------------------------------
+ * A decode step is a handful of small layers (the q/k/v projections share one x; gate/up likewise),
+ * each only a few MB of indices: launched one by one, launch latency and pipeline ramp-up cost more
+ * than the index stream itself.  btc_linear_gemv_batch runs `count` independent layers
+ *     y_i[m, n] = alpha_i[n] * sum_j <x_i[m, j*v:(j+1)*v], C_i[idx_i[n, j]]>  (+ mu_i[n] * sum_k x_i[m, k])
+ * (same definition as btc_linear_gemv: paper appendix "Binary codebook LUT-GEMM", second display,
+ * with the row-wise dequantisation of Eq. 1-2) as one persistent kernel over the concatenated
+ * work, up to BTC_BATCH_MAX layers per launch; longer lists and layers the fused kernel does not
+ * cover are run by further launches on the same stream, so the call never fails for that reason.
+ *   problems  HOST array of `count` descriptors; it is read before the call returns.  Every pointer
+ *             inside a descriptor is a DEVICE pointer with the layout, alignment and ranges stated
+ *             for btc_linear_gemv; 1 <= M <= 8 for every layer.  No transform argument.
+ *   The layers must be independent: no y_i may alias an x_j, idx_j or another y_j of the same call.
+ * Errors: as btc_linear_gemv; the first failing layer's status is returned and later layers of the
+ * list may not have been enqueued.
+ */
+#define BTC_BATCH_MAX 8
+typedef struct {
+    const void *x;
+    const uint16_t *idx;
+    const uint32_t *C_packed;
+    const void *alpha;
+    const void *mu;        /* NULL = no mean term */
+    void *y;
+    int x_dtype, y_dtype;
+    int M, N, K, v, Kc;
+} btc_linear_problem;
+BTC_API int btc_linear_gemv_batch(const btc_linear_problem *problems, int count, void *stream);
+
 /* ---- btc_linear_gemm for callers that cannot allocate device memory ---------------------------
  * (No counterpart in the paper: this is a packaging variant of btc_linear_gemm, same arithmetic.)
  *

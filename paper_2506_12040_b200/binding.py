@@ -20,13 +20,20 @@ _DT = {torch.float16: BTC_F16, torch.bfloat16: BTC_BF16, torch.float32: BTC_F32}
 EXPORTS = (
     "btc_version", "btc_status_string", "btc_last_cuda_error", "btc_codebook_packed_bytes",
     "btc_codebook_pack", "btc_codebook_pack_host", "btc_linear_workspace_bytes", "btc_linear_gemv",
-    "btc_linear_gemm", "btc_linear_gemm_static_scratch", "btc_decode_pm1", "btc_validate_indices", "btc_bits_per_weight", "btc_device_status",
+    "btc_linear_gemm", "btc_linear_gemv_batch", "btc_linear_gemm_static_scratch", "btc_decode_pm1", "btc_validate_indices", "btc_bits_per_weight", "btc_device_status",
 )
 
 
 class BtcTransform(ctypes.Structure):
     _fields_ = [("sigma_bits", ctypes.c_void_p), ("P1", ctypes.c_void_p), ("P2", ctypes.c_void_p),
                 ("k1", ctypes.c_int), ("k2", ctypes.c_int)]
+
+
+class BtcLinearProblem(ctypes.Structure):
+    _fields_ = [("x", ctypes.c_void_p), ("idx", ctypes.c_void_p), ("C_packed", ctypes.c_void_p),
+                ("alpha", ctypes.c_void_p), ("mu", ctypes.c_void_p), ("y", ctypes.c_void_p),
+                ("x_dtype", ctypes.c_int), ("y_dtype", ctypes.c_int),
+                ("M", ctypes.c_int), ("N", ctypes.c_int), ("K", ctypes.c_int), ("v", ctypes.c_int), ("Kc", ctypes.c_int)]
 
 
 class BtcError(RuntimeError):
@@ -59,6 +66,7 @@ def _load() -> ctypes.CDLL:
     lin = [vp, ci, vp, vp, vp, vp, ctypes.POINTER(BtcTransform), vp, ci, ci, ci, ci, ci, ci, vp, sz, vp]
     L.btc_linear_gemv.argtypes = lin
     L.btc_linear_gemm.argtypes = lin
+    L.btc_linear_gemv_batch.argtypes = [ctypes.POINTER(BtcLinearProblem), ci, vp]
     L.btc_linear_gemm_static_scratch.argtypes = lin[:14] + [vp]
     L.btc_decode_pm1.argtypes = [vp, vp, ci, ci, ci, ci, vp, vp]
     L.btc_validate_indices.argtypes = [vp, sz, ci, vp, vp]
@@ -180,6 +188,47 @@ def linear_gemm(x, idx, C_packed, alpha, v, Kc, mu=None, out=None, out_dtype=tor
     """Tensor-core path (any M, built for large M)."""
     return _linear(lib.btc_linear_gemm, "btc_linear_gemm", x, idx, C_packed, alpha, v, Kc, mu, out, out_dtype,
                    workspace, transform)
+
+
+class GemvBatch:
+    """A fixed list of independent decode-path layers (M <= 8 each) marshalled once, run with one
+    btc_linear_gemv_batch call per `run()`: each entry is a dict with x, idx, C_packed, alpha, v, Kc,
+    and optionally mu, out (fp32 [M, N] is allocated when absent)."""
+
+    def __init__(self, layers):
+        self.layers = []
+        arr = (BtcLinearProblem * len(layers))()
+        for i, L in enumerate(layers):
+            x, idx, Cp, alpha = L["x"], L["idx"], L["C_packed"], L["alpha"]
+            for t, n in ((x, "x"), (idx, "idx"), (Cp, "C_packed"), (alpha, "alpha")):
+                _dev(t, n)
+            M, K = x.shape
+            N, Kb = idx.shape
+            v, Kc = int(L["v"]), int(L["Kc"])
+            if Kb * v != K or alpha.numel() != N or Cp.numel() != packed_words(Kc, v):
+                raise ValueError("shape mismatch between x, idx, v, alpha and C_packed")
+            if x.dtype not in (torch.float16, torch.bfloat16) or alpha.dtype != torch.float16 or idx.element_size() != 2:
+                raise ValueError("x must be fp16/bf16, alpha fp16, idx 16-bit")
+            mu = L.get("mu")
+            out = L.get("out")
+            if out is None:
+                out = torch.empty((M, N), dtype=torch.float32, device=x.device)
+            arr[i] = BtcLinearProblem(x.data_ptr(), idx.data_ptr(), Cp.data_ptr(), alpha.data_ptr(), _ptr(mu),
+                                      out.data_ptr(), _DT[x.dtype], _DT[out.dtype], M, N, K, v, Kc)
+            self.layers.append((x, idx, Cp, alpha, mu, out))          # keeps the tensors alive
+        self._arr = arr
+        self.outs = [t[5] for t in self.layers]
+
+    def run(self):
+        st = lib.btc_linear_gemv_batch(self._arr, len(self.layers), _stream())
+        if st:
+            raise BtcError(st, "btc_linear_gemv_batch")
+        return self.outs
+
+
+def linear_gemv_batch(layers):
+    """One btc_linear_gemv_batch call over `layers` (see GemvBatch); returns the list of outputs."""
+    return GemvBatch(layers).run()
 
 
 STATIC_SCRATCH_BYTES = 65536

@@ -133,6 +133,47 @@ extern "C" int btc_linear_gemm(const void *x, int x_dtype, const uint16_t *idx, 
                       workspace, workspace_bytes, stream);
 }
 
+extern "C" int btc_linear_gemv_batch(const btc_linear_problem *problems, int count, void *stream)
+{
+    if (!problems) return BTC_ERR_NULL;
+    if (count < 1) return BTC_ERR_SHAPE;
+    cudaStream_t s = (cudaStream_t)stream;
+    LinearArgs group[IM_MAXP];
+    int i = 0;
+    while (i < count) {
+        // longest run of layers (at most IM_MAXP) starting at i
+        int n = 0;
+        for (; n < IM_MAXP && i + n < count; ++n) {
+            const btc_linear_problem &p = problems[i + n];
+            int rc = validate(p.x, p.x_dtype, p.idx, p.C_packed, p.alpha, p.y, p.y_dtype, p.M, p.N, p.K, p.v, p.Kc);
+            if (rc != BTC_OK) return rc;
+            if (p.mu && !aligned(p.mu, 2)) return BTC_ERR_ALIGN;
+            if (p.M > 8) return BTC_ERR_SHAPE;
+            LinearArgs &a = group[n];
+            a.x = p.x; a.idx = p.idx; a.Cp = p.C_packed;
+            a.alpha = reinterpret_cast<const __half *>(p.alpha);
+            a.mu = reinterpret_cast<const __half *>(p.mu);
+            a.y = p.y; a.workspace = nullptr; a.workspace_bytes = 0;
+            a.x_dt = p.x_dtype; a.y_dt = p.y_dtype;
+            a.M = p.M; a.N = p.N; a.K = p.K; a.v = p.v; a.Kc = p.Kc; a.Kb = p.K / p.v;
+        }
+        int rc = launch_gemv_imma(group, n, s);
+        if (rc == BTC_ERR_UNSUPPORTED) {
+            // some layer of the run is outside the fused kernel: one launch per layer instead
+            for (int k = 0; k < n; ++k) {
+                rc = launch_gemv_imma(&group[k], 1, s);
+                if (rc == BTC_ERR_UNSUPPORTED) rc = launch_gemv_decode(group[k], s);
+                if (rc == BTC_ERR_UNSUPPORTED) rc = launch_linear_generic(group[k], s);
+                if (rc != BTC_OK) return rc;
+            }
+        } else if (rc != BTC_OK) {
+            return rc;
+        }
+        i += n;
+    }
+    return BTC_OK;
+}
+
 extern "C" double btc_bits_per_weight(int N, int K, int v, int Kc, int scale_bits_per_row, int mode,
                                       int with_codebook)
 {

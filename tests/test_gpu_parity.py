@@ -175,3 +175,27 @@ def test_gemm_deterministic_and_bounded():
     torch.cuda.synchronize()
     assert torch.equal(first, out)
     assert bool((guard[:256] == 777.0).all()) and bool((guard[256 + M * N:] == 777.0).all())
+
+
+# ------------------------------------------------------------------ several layers in one launch
+
+def test_gemv_batch_matches_oracle_and_single_calls():
+    """Seven layers of mixed shape (the decode layer set scaled down, ragged N, one with mu, one bf16) in one
+    btc_linear_gemv_batch call: every output against the oracle, and bit-identical to the per-layer call."""
+    shapes = [(272, 1024, 16, 4096, False, "f16"), (272, 1024, 16, 4096, True, "f16"), (100, 1024, 16, 8192, False, "f16"),
+              (1000, 1024, 16, 8192, False, "bf16"), (688, 2752, 16, 8192, False, "f16"), (37, 320, 20, 65536, False, "f16"),
+              (513, 640, 20, 21619, True, "f16"), (64, 96, 12, 777, False, "f16"), (300, 2048, 16, 8192, False, "f16")]
+    for M in (1, 2, 8):
+        Ls = [wl.make_layer(_spec(N, K, v, Kc, with_mu=mu, x_dtype=dt, outlier_frac=0.01), M, seed=50 + i)
+              for i, (N, K, v, Kc, mu, dt) in enumerate(shapes)]
+        ds = [to_device(L) for L in Ls]
+        layers = [dict(x=d["x"], idx=d["idx"], C_packed=d["Cp"], alpha=d["alpha"], mu=d["mu"], v=L.spec.v, Kc=L.spec.Kc)
+                  for L, d in zip(Ls, ds)]
+        outs = btc.linear_gemv_batch(layers)
+        torch.cuda.synchronize()
+        for L, d, y in zip(Ls, ds, outs):
+            rel, fwd = errors(y, oracle_y(L), L)
+            assert rel <= TOL_GEMV and fwd <= TOL_GEMV, (L.spec, M, rel, fwd)
+            single = btc.linear_gemv(d["x"], d["idx"], d["Cp"], d["alpha"], L.spec.v, L.spec.Kc, mu=d["mu"])
+            assert torch.equal(single, y), (L.spec, M)
+    assert btc.device_status() == 0
