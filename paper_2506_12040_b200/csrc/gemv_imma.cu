@@ -135,18 +135,18 @@ __device__ __forceinline__ void im_unpack2(uint32_t w, int dt, float &lo, float 
 // Shared-memory layout (dynamic), offsets computed identically on host and device.
 struct ImSmem {
     uint32_t bars;        // mbarriers: full[S], empty[S], part_full[2], part_empty[2], tab_full, tab_free
-    uint32_t misc;        // abort flag, per-layer scale slots, reduction scratch
+    uint32_t misc;        // abort flag, per-part scale slots
     uint32_t planes;      // per compute warp: digit planes of its K-slice of one row of x
     uint32_t tab;         // codeword table
     uint32_t ring;        // index stages
     uint32_t part;        // partial sums [2][16 warps][rows][cols]
-    uint32_t acc;         // sums over warps (and K-parts) [IM_RC][rows][cols]
+    uint32_t acc;         // dot products summed over K-parts, double [IM_RC][rows][cols / 2]
     uint32_t total;
 };
 constexpr int IM_NBARS = 2 * IM_STAGES + 6;
-constexpr int IM_SLOTS = 3;                      // scale slots, one per layer a CTA is working on
-struct ImSlot { double inv[8]; double sx[8]; float sc[8]; };          // 1/scale, sum_k X, scale per row m
-constexpr int IM_MISC_BYTES = 16 + IM_SLOTS * (int)sizeof(ImSlot) + IM_CWARPS * 8 * 4 + IM_CWARPS * 8 * 8;
+constexpr int IM_SLOTS = 4;                      // scale slots: K-parts whose partial sums may still be in flight
+struct ImScale { double inv; double sx; };       // per (slot, compute warp, row m of x): 1/scale, and sum_k x over the slice
+constexpr int IM_MISC_BYTES = 16 + IM_SLOTS * IM_CWARPS * 8 * (int)sizeof(ImScale);
 constexpr int IM_PLANE_WORDS = 3 * 16 * 8;       // 3 digits x 16 blocks x (v / 4 <= 8) words
 
 __host__ __device__ inline ImSmem im_smem_layout(int tab_bytes, int tile_ints)
@@ -194,14 +194,13 @@ gemv_imma_kernel(const __grid_constant__ ImBatch batch)
     const ImSmem L = im_smem_layout(batch.tab_smem_bytes, TILE_INTS);
     uint64_t *bars = reinterpret_cast<uint64_t *>(smem + L.bars);
     volatile int *s_abort = reinterpret_cast<volatile int *>(smem + L.misc);
-    ImSlot *s_slot = reinterpret_cast<ImSlot *>(smem + L.misc + 16);
-    float *s_redf = reinterpret_cast<float *>(smem + L.misc + 16 + IM_SLOTS * sizeof(ImSlot));            // [16][8]
-    double *s_redd = reinterpret_cast<double *>(smem + L.misc + 16 + IM_SLOTS * sizeof(ImSlot) + IM_CWARPS * 32);   // [16][8]
+    ImScale *s_scale = reinterpret_cast<ImScale *>(smem + L.misc + 16);           // [IM_SLOTS][16 warps][8]
     uint32_t *s_planes = reinterpret_cast<uint32_t *>(smem + L.planes);
     uint32_t *s_tab = reinterpret_cast<uint32_t *>(smem + L.tab);
     unsigned char *s_ring = smem + L.ring;
     int *s_part = reinterpret_cast<int *>(smem + L.part);
-    int *s_acc = reinterpret_cast<int *>(smem + L.acc);
+    double *s_acc = reinterpret_cast<double *>(smem + L.acc);
+    constexpr int ACC_M = COLS / 2;                      // doubles per row of s_acc (>= MAXM)
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     auto bar_full = [&](int s) { return im_smem_u32(bars + s); };
@@ -224,7 +223,8 @@ gemv_imma_kernel(const __grid_constant__ ImBatch batch)
     const bool tab_smem = batch.tab_smem_bytes > 0;
 
     // All three roles walk the same sequence: layers pi (those with row groups for this CTA, counted
-    // by ps), chunks [c0, c1) of at most IM_RC row groups, K-parts j, row groups r; li counts iterations.
+    // by ps), chunks [c0, c1) of at most IM_RC row groups, K-parts j (counted by pc), row groups r; li
+    // counts iterations.
     if (warp == IM_CWARPS) {
         // ============================================================ producer
         int li = 0, ps = 0;
@@ -276,71 +276,76 @@ gemv_imma_kernel(const __grid_constant__ ImBatch batch)
         }
     } else if (warp > IM_CWARPS) {
         // ============================================================ epilogue (two warps)
-        const int ew = warp - IM_CWARPS - 1;                   // 0 or 1
-        const int R = lane;                                    // row of the group
+        // 64 threads = ROWS rows x SPLIT groups of compute warps; the groups of a row sit in adjacent lanes.
+        constexpr int SPLIT = (IM_EWARPS * 32) / ROWS;         // 2 or 4
+        constexpr int WPG = IM_CWARPS / SPLIT;                 // compute warps per group
+        const int et = (warp - IM_CWARPS - 1) * 32 + lane;
+        const int R = et / SPLIT, grp = et % SPLIT;
         asm volatile("griddepcontrol.wait;" ::: "memory");
-        int li = 0, ps = 0;
+        int li = 0, pc = 0;
         bool ok = true;
         for (int pi = 0; pi < batch.count && ok; ++pi) {
             const ImProblem &P = batch.p[pi];
             int glo, ghi;
             im_group_range(P, batch.cost_total, blockIdx.x, gridDim.x, glo, ghi);
             if (glo >= ghi) continue;
-            const ImSlot *slot = s_slot + (ps % IM_SLOTS);
-            ++ps;
-            const double unshift = 1.0 / (double)(1 << (P.ncls - 1));
+            const double unshift2 = 2.0 / (double)(1 << (P.ncls - 1));
             for (int c0 = glo; c0 < ghi && ok; c0 += IM_RC) {
                 const int c1 = min(c0 + IM_RC, ghi);
-                for (int j = 0; j < P.parts && ok; ++j) {
+                double sxtot[MAXM];                              // sum_k x[m, k] over the parts seen so far
+#pragma unroll
+                for (int m = 0; m < MAXM; ++m) sxtot[m] = 0.0;
+                for (int j = 0; j < P.parts && ok; ++j, ++pc) {
                     const bool last = (j == P.parts - 1);
+                    const ImScale *sc = s_scale + (size_t)(pc % IM_SLOTS) * IM_CWARPS * 8;
                     for (int r = c0; r < c1; ++r, ++li) {
                         const int buf = li & 1;
                         const int n = r * ROWS + R;
-                        const bool live = (R < ROWS) && (n < P.N);
+                        const bool live = (n < P.N) && (grp == 0);
                         float al = 0.f, mu = 0.f;
-                        if (last && live && ew < P.M) {
+                        if (last && live) {
                             al = __half2float(P.alpha[n]);
                             if (P.mu) mu = __half2float(P.mu[n]);
                         }
                         if (!im_mbar_wait(bar_pfull(buf), (li >> 1) & 1, s_abort)) { ok = false; break; }
-                        int *accrow = s_acc + (size_t)(P.parts > 1 ? (r - c0) : buf) * TILE_INTS + (size_t)R * COLS;
-                        if (R < ROWS) {
+                        double *accrow = s_acc + ((size_t)(P.parts > 1 ? (r - c0) : 0) * ROWS + R) * ACC_M;
+                        const int *base = s_part + ((size_t)buf * IM_CWARPS + grp * WPG) * TILE_INTS + (size_t)R * COLS;
+                        double dots[MAXM], sxp[MAXM];
 #pragma unroll
-                            for (int qd = 0; qd < 2 * NM; ++qd) {
-                                if ((qd & 1) != ew) continue;                 // this warp's column quads
-                                int4 sum = make_int4(0, 0, 0, 0);
-                                const int *base = s_part + (size_t)buf * IM_CWARPS * TILE_INTS + (size_t)R * COLS + qd * 4;
+                        for (int m = 0; m < MAXM; ++m) {
+                            dots[m] = 0.0; sxp[m] = 0.0;
+                            if (m < P.M) {
 #pragma unroll
-                                for (int w = 0; w < IM_CWARPS; ++w) {
-                                    const int4 v4 = *reinterpret_cast<const int4 *>(base + (size_t)w * TILE_INTS);
-                                    sum.x += v4.x; sum.y += v4.y; sum.z += v4.z; sum.w += v4.w;
+                                for (int w = 0; w < WPG; ++w) {
+                                    const int *pw3 = base + (size_t)w * TILE_INTS + 3 * m;
+                                    const long long T = ((long long)pw3[2] * 256 + pw3[1]) * 256 + pw3[0];
+                                    const ImScale sw = sc[(grp * WPG + w) * 8 + m];
+                                    dots[m] += (double)T * sw.inv;
+                                    sxp[m] += sw.sx;
                                 }
-                                int4 *dst = reinterpret_cast<int4 *>(accrow + qd * 4);
-                                if (j > 0) { const int4 o = *dst; sum.x += o.x; sum.y += o.y; sum.z += o.z; sum.w += o.w; }
-                                *dst = sum;
                             }
                         }
                         __syncwarp();
                         if (lane == 0) im_mbar_arrive(bar_pempty(buf));
-                        if (last) {
-                            double inv[MAXM], sx[MAXM];
 #pragma unroll
-                            for (int m = 0; m < MAXM; ++m) { inv[m] = slot->inv[m]; sx[m] = slot->sx[m]; }
-                            im_named_bar(2, IM_EWARPS * 32);              // the other warp's column quads are in place
-                            if (live) {
+                        for (int m = 0; m < MAXM; ++m) {
+                            if (m < P.M) {
 #pragma unroll
-                                for (int m = 0; m < MAXM; ++m) {
-                                    if (m < P.M && (m & 1) == ew) {
-                                        const double T = ((double)accrow[3 * m + 2] * 256.0 + (double)accrow[3 * m + 1]) * 256.0
-                                                         + (double)accrow[3 * m];
-                                        const double sumx = sx[m] * inv[m];
-                                        const double dot = (2.0 * T * unshift - sx[m]) * inv[m];
-                                        const float yv = (float)((double)al * dot + (double)mu * sumx);
-                                        store_from_float(P.y, P.y_dt, (size_t)m * P.N + n, yv);
-                                    }
+                                for (int o = 1; o < SPLIT; o <<= 1) {
+                                    dots[m] += __shfl_xor_sync(0xffffffffu, dots[m], o);
+                                    sxp[m] += __shfl_xor_sync(0xffffffffu, sxp[m], o);
+                                }
+                                if (r == c0) sxtot[m] += sxp[m];
+                                double dot = dots[m] * unshift2 - sxp[m];       // 2 * sum_{bit=1} x - sum x over this part
+                                if (grp == 0) {
+                                    if (j > 0) dot += accrow[m];
+                                    if (!last) accrow[m] = dot;
+                                }
+                                if (last && live) {
+                                    const float yv = (float)((double)al * dot + (double)mu * sxtot[m]);
+                                    store_from_float(P.y, P.y_dt, (size_t)m * P.N + n, yv);
                                 }
                             }
-                            im_named_bar(2, IM_EWARPS * 32);              // reads done before the slot of s_acc is reused
                         }
                     }
                 }
@@ -354,86 +359,31 @@ gemv_imma_kernel(const __grid_constant__ ImBatch batch)
         constexpr int MAGIC_BITS = 0x4B400000;
         uint32_t *planes = s_planes + warp * IM_PLANE_WORDS;
         asm volatile("griddepcontrol.wait;" ::: "memory");
-        int li = 0, ps = 0;
+        int li = 0, ps = 0, pc = 0;
         bool ok = true;
         for (int pi = 0; pi < batch.count && ok; ++pi) {
             const ImProblem &P = batch.p[pi];
             int glo, ghi;
             im_group_range(P, batch.cost_total, blockIdx.x, gridDim.x, glo, ghi);
             if (glo >= ghi) continue;
-            ImSlot *slot = s_slot + (ps % IM_SLOTS);
             const int M = P.M, K = P.K, Kb = P.Kb, v = P.v;
             const int cmax = P.ncls - 1;
             const int PBITS = 22 - cmax;                       // |X| <= 2^PBITS
-            const int nvec = K >> 3;                           // 16-byte loads; K % 16 == 0 (host check)
-
-            // ---- per layer, step 1: scale of every row of x from its largest magnitude
-            for (int m = 0; m < M; ++m) {
-                float a = 0.f;
-                const uint4 *xr = reinterpret_cast<const uint4 *>(reinterpret_cast<const uint16_t *>(P.x) + (size_t)m * K);
-                for (int i = tid; i < nvec; i += CT) {
-                    const uint4 q4 = __ldg(xr + i);
-                    const uint32_t wds[4] = {q4.x, q4.y, q4.z, q4.w};
-#pragma unroll
-                    for (int jj = 0; jj < 4; ++jj) {
-                        float lo, hi;
-                        im_unpack2(wds[jj], P.x_dt, lo, hi);
-                        a = fmaxf(a, fmaxf(fabsf(lo), fabsf(hi)));
-                    }
-                }
-#pragma unroll
-                for (int o = 16; o > 0; o >>= 1) a = fmaxf(a, __shfl_xor_sync(0xffffffffu, a, o));
-                if (lane == 0) s_redf[warp * 8 + m] = a;
-            }
-            im_named_bar(1, CT);
-            if (tid < M) {
-                float a = 0.f;
-                for (int w = 0; w < IM_CWARPS; ++w) a = fmaxf(a, s_redf[w * 8 + tid]);
-                int e = 0;
-                if (a > 0.f) (void)frexpf(a, &e);              // a = f * 2^e, f in [0.5, 1)
-                slot->inv[tid] = (a > 0.f) ? ldexp(1.0, e - PBITS) : 1.0;
-                slot->sc[tid] = (a > 0.f) ? ldexpf(1.0f, PBITS - e) : 1.0f;
-            }
-            im_named_bar(1, CT);
-            // ---- step 2: integer row sums  sum_k X[m, k]
-            for (int m = 0; m < M; ++m) {
-                const float sc = slot->sc[m];
-                int xs = 0;
-                const uint4 *xr = reinterpret_cast<const uint4 *>(reinterpret_cast<const uint16_t *>(P.x) + (size_t)m * K);
-                for (int i = tid; i < nvec; i += CT) {
-                    const uint4 q4 = __ldg(xr + i);
-                    const uint32_t wds[4] = {q4.x, q4.y, q4.z, q4.w};
-#pragma unroll
-                    for (int jj = 0; jj < 4; ++jj) {
-                        float lo, hi;
-                        im_unpack2(wds[jj], P.x_dt, lo, hi);
-                        xs += (__float_as_int(lo * sc + MAGIC) - MAGIC_BITS) + (__float_as_int(hi * sc + MAGIC) - MAGIC_BITS);
-                    }
-                }
-                double sacc = (double)xs;                      // |xs| <= 8 * ceil(nvec / CT) * 2^PBITS, far below 2^31 for K <= 2^20
-#pragma unroll
-                for (int o = 16; o > 0; o >>= 1) sacc += __shfl_xor_sync(0xffffffffu, sacc, o);
-                if (lane == 0) s_redd[warp * 8 + m] = sacc;
-            }
-            im_named_bar(1, CT);
-            if (tid < M) {
-                double sacc = 0.0;
-                for (int w = 0; w < IM_CWARPS; ++w) sacc += s_redd[w * 8 + tid];
-                slot->sx[tid] = sacc;
-            }
-            // (the epilogue warps read the slot only after a partial-sum barrier that follows this point)
-            if (tab_smem && !im_mbar_wait(bar_tabfull, ps & 1, s_abort)) break;
-            ++ps;
+            const int nwords = 16 * P.ncls;                    // words per digit plane of a warp's slice
+            bool tab_ready = !tab_smem;
             const uint32_t *tab = tab_smem ? s_tab : P.tab;
 
             for (int c0 = glo; c0 < ghi && ok; c0 += IM_RC) {
                 const int c1 = min(c0 + IM_RC, ghi);
-                for (int j = 0; j < P.parts && ok; ++j) {
+                for (int j = 0; j < P.parts && ok; ++j, ++pc) {
                     const int pw = min(IM_PW, Kb - j * IM_PW);
                     const int jb0 = j * IM_PW + warp * 16;          // first block of this warp's slice
                     const bool wvalid = warp * 16 + 4 * t < pw;     // this lane's four blocks exist (pw % 4 == 0)
+                    const int kend = (j * IM_PW + pw) * v;          // end of the part in x
+                    ImScale *scale_out = s_scale + ((size_t)(pc % IM_SLOTS) * IM_CWARPS + warp) * 8;
 
-                    // ---- B fragments for this part: digit planes of the warp's slice, row by row of x
+                    // ---- B fragments for this part.  The warp's slice of each row of x (16 blocks) is
+                    //      quantised with its own scale: X = rint(x * 2^(PBITS - e)), 2^e > max |x| of the slice.
                     uint32_t breg[4][NCLS][NM];
 #pragma unroll
                     for (int e = 0; e < 4; ++e)
@@ -441,36 +391,69 @@ gemv_imma_kernel(const __grid_constant__ ImBatch batch)
                         for (int c = 0; c < NCLS; ++c)
 #pragma unroll
                             for (int nm = 0; nm < NM; ++nm) breg[e][c][nm] = 0u;
-                    const int nwords = 16 * P.ncls;                 // words per digit plane of the slice
                     for (int m = 0; m < M; ++m) {
-                        const float sc = slot->sc[m];
                         const uint16_t *xrow = reinterpret_cast<const uint16_t *>(P.x) + (size_t)m * K;
-                        for (int gi = lane; gi < 2 * v; gi += 32) {          // groups of 8 activations
-                            const int k0 = jb0 * v + 8 * gi;
-                            uint4 q4 = make_uint4(0u, 0u, 0u, 0u);
-                            if (k0 < K && k0 / v < j * IM_PW + pw) q4 = __ldg(reinterpret_cast<const uint4 *>(xrow + k0));
-                            const uint32_t wds[4] = {q4.x, q4.y, q4.z, q4.w};
+                        // groups of 8 activations: lane, lane + 32 (the slice has 2 v <= 64 groups)
+                        uint4 q4[2];
+                        float amax = 0.f;
 #pragma unroll
-                            for (int h = 0; h < 2; ++h) {
-                                const int c = ((k0 + 4 * h) % v) >> 2;
-                                const uint32_t sh = 1u << (cmax - c);
-                                const uint32_t off = 0x8080u - (uint32_t)MAGIC_BITS * sh;    // arithmetic modulo 2^32
-                                float f0, f1, f2, f3;
-                                im_unpack2(wds[2 * h], P.x_dt, f0, f1);
-                                im_unpack2(wds[2 * h + 1], P.x_dt, f2, f3);
-                                // Y = X * 2^(cmax - c) + 0x8080: byte d of Y is balanced digit d of X * 2^(cmax-c), + 0x80 for d < 2
-                                const uint32_t y0 = (uint32_t)__float_as_int(f0 * sc + MAGIC) * sh + off;
-                                const uint32_t y1 = (uint32_t)__float_as_int(f1 * sc + MAGIC) * sh + off;
-                                const uint32_t y2 = (uint32_t)__float_as_int(f2 * sc + MAGIC) * sh + off;
-                                const uint32_t y3 = (uint32_t)__float_as_int(f3 * sc + MAGIC) * sh + off;
-                                const int wi = 2 * gi + h;
+                        for (int u = 0; u < 2; ++u) {
+                            const int k0 = jb0 * v + 8 * (lane + 32 * u);
+                            q4[u] = make_uint4(0u, 0u, 0u, 0u);
+                            if (lane + 32 * u < 2 * v && k0 < kend) q4[u] = __ldg(reinterpret_cast<const uint4 *>(xrow + k0));
+                            const uint32_t wds[4] = {q4[u].x, q4[u].y, q4[u].z, q4[u].w};
 #pragma unroll
-                                for (int d = 0; d < 3; ++d) {
-                                    const uint32_t sel = (uint32_t)d | ((uint32_t)(4 + d) << 4);
-                                    const uint32_t lo2 = __byte_perm(y0, y1, sel), hi2 = __byte_perm(y2, y3, sel);
-                                    planes[d * nwords + wi] = __byte_perm(lo2, hi2, 0x5410) ^ (d < 2 ? 0x80808080u : 0u);
+                            for (int jj = 0; jj < 4; ++jj) {
+                                float lo, hi;
+                                im_unpack2(wds[jj], P.x_dt, lo, hi);
+                                amax = fmaxf(amax, fmaxf(fabsf(lo), fabsf(hi)));
+                            }
+                        }
+#pragma unroll
+                        for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+                        // amax = f * 2^e with f in [1, 2) (a float from fp16 / bf16 is normal or zero): |x| < 2^(e+1)
+                        const int ex = max((int)((__float_as_uint(amax) >> 23) & 0xffu) - 127 + 1, -100);   // (clamped: bf16 can be tinier)
+                        const float sc = (amax > 0.f) ? __uint_as_float((uint32_t)(127 + PBITS - ex) << 23) : 1.0f;
+                        const double inv = (amax > 0.f) ? __longlong_as_double((long long)(1023 - PBITS + ex) << 52) : 1.0;
+                        int xs = 0;
+#pragma unroll
+                        for (int u = 0; u < 2; ++u) {
+                            const int gi = lane + 32 * u;
+                            if (gi < 2 * v) {
+                                const uint32_t wds[4] = {q4[u].x, q4[u].y, q4[u].z, q4[u].w};
+                                int cpos = (8 * gi) % v;                 // position of the group's first activation in its block
+#pragma unroll
+                                for (int h = 0; h < 2; ++h) {
+                                    const int c = cpos >> 2;
+                                    cpos += 4;
+                                    if (cpos >= v) cpos -= v;
+                                    const uint32_t sh = 1u << (cmax - c);
+                                    const uint32_t off = 0x8080u - (uint32_t)MAGIC_BITS * sh;    // arithmetic modulo 2^32
+                                    float f0, f1, f2, f3;
+                                    im_unpack2(wds[2 * h], P.x_dt, f0, f1);
+                                    im_unpack2(wds[2 * h + 1], P.x_dt, f2, f3);
+                                    const uint32_t b0 = (uint32_t)__float_as_int(f0 * sc + MAGIC), b1 = (uint32_t)__float_as_int(f1 * sc + MAGIC);
+                                    const uint32_t b2 = (uint32_t)__float_as_int(f2 * sc + MAGIC), b3 = (uint32_t)__float_as_int(f3 * sc + MAGIC);
+                                    xs += (int)(b0 + b1 + b2 + b3 - 4u * (uint32_t)MAGIC_BITS);
+                                    // Y = X * 2^(cmax - c) + 0x8080: byte d of Y is balanced digit d of X * 2^(cmax-c), + 0x80 for d < 2
+                                    const uint32_t y0 = b0 * sh + off, y1 = b1 * sh + off, y2 = b2 * sh + off, y3 = b3 * sh + off;
+                                    const int wi = 2 * gi + h;
+#pragma unroll
+                                    for (int d = 0; d < 3; ++d) {
+                                        const uint32_t sel = (uint32_t)d | ((uint32_t)(4 + d) << 4);
+                                        const uint32_t lo2 = __byte_perm(y0, y1, sel), hi2 = __byte_perm(y2, y3, sel);
+                                        planes[d * nwords + wi] = __byte_perm(lo2, hi2, 0x5410) ^ (d < 2 ? 0x80808080u : 0u);
+                                    }
                                 }
                             }
+                        }
+#pragma unroll
+                        for (int o = 16; o > 0; o >>= 1) xs += __shfl_xor_sync(0xffffffffu, xs, o);
+                        if (lane == 0) {
+                            ImScale o2;
+                            o2.inv = inv;
+                            o2.sx = (double)xs * inv;
+                            scale_out[m] = o2;
                         }
                         __syncwarp();
 #pragma unroll
@@ -486,6 +469,10 @@ gemv_imma_kernel(const __grid_constant__ ImBatch batch)
                             }
                         }
                         __syncwarp();
+                    }
+                    if (!tab_ready) {
+                        if (!im_mbar_wait(bar_tabfull, ps & 1, s_abort)) { ok = false; break; }
+                        tab_ready = true;
                     }
 
                     // ---- the row groups of the chunk, for this part
@@ -564,6 +551,7 @@ gemv_imma_kernel(const __grid_constant__ ImBatch batch)
                     }
                 }
             }
+            ++ps;
             if (tab_smem && ok) {
                 __syncwarp();
                 if (lane == 0) im_mbar_arrive(bar_tabfree);
