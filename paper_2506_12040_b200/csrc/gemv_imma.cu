@@ -31,6 +31,7 @@
 //   warps 17,18  epilogue: add the 16 partial tiles in a fixed order, add the K-parts, recombine
 //                digits, apply alpha (and mu), store y.
 // Every mbarrier wait is bounded; when one runs out the CTA raises a status word and drains.
+#include <cuda.h>
 #include "btc_internal.cuh"
 
 namespace btc {
@@ -39,7 +40,8 @@ constexpr int IM_CWARPS = 16;                   // compute warps
 constexpr int IM_EWARPS = 2;                    // epilogue warps
 constexpr int IM_THREADS = (IM_CWARPS + 1 + IM_EWARPS) * 32;
 constexpr int IM_STAGES = 4;
-constexpr int IM_STAGE_BYTES = 16 * 1024;       // one iteration's indices: 32 rows x 256 blocks
+constexpr int IM_BOX_COLS = 64;                 // blocks per TMA box row: 128 bytes, the swizzle span
+constexpr int IM_STAGE_BYTES = 16 * 1024;       // one iteration's indices: 4 boxes of 32 rows x 128 bytes
 constexpr int IM_PW = 256;                      // blocks per K-part (16 per compute warp)
 constexpr int IM_RC = 16;                       // row groups a CTA walks part by part at a time
 
@@ -57,13 +59,16 @@ struct ImProblem {
     int parts;                // ceil(Kb / IM_PW)
     int groups;               // row groups: ceil(N / (16 * TRK))
     int ncls;                 // v / 4
-    long long cost_base;      // sum over earlier layers of groups * Kb
+    int cost_base;            // sum over earlier layers of groups * Kb
 };
 
 struct ImBatch {
+    CUtensorMap map[IM_MAXP]; // idx of each layer as a 2-D tensor {K/v, N} of 16-bit words, box {64, rows}, 128-byte swizzle
     ImProblem p[IM_MAXP];
     int count;
-    long long cost_total;
+    int cost_total;           // sum over layers of groups * Kb (host bookkeeping)
+    int cost_per, cost_rem;   // the launch's cost line (sum of groups * Kb) cut for the grid: CTA b gets
+                              // [per * b + min(b, rem), + per + (b < rem))
     int tab_smem_bytes;       // bytes reserved for the codeword table (0: gather from global memory)
 };
 
@@ -109,6 +114,11 @@ __device__ __forceinline__ void im_bulk_g2s(uint32_t dst, const void *src, uint3
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                  ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
 }
+__device__ __forceinline__ void im_tma_2d(uint32_t dst, const CUtensorMap *map, int c0, int c1, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(bar) : "memory");
+}
 __device__ __forceinline__ void im_mma_u8s8(int (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
                                             uint32_t b0, uint32_t b1) {
     asm volatile(
@@ -146,10 +156,10 @@ struct ImSmem {
 constexpr int IM_NBARS = 2 * IM_STAGES + 6;
 constexpr int IM_SLOTS = 4;                      // scale slots: K-parts whose partial sums may still be in flight
 struct ImScale { double inv; double sx; };       // per (slot, compute warp, row m of x): 1/scale, and sum_k x over the slice
-constexpr int IM_MISC_BYTES = 16 + IM_SLOTS * IM_CWARPS * 8 * (int)sizeof(ImScale);
-constexpr int IM_PLANE_WORDS = 3 * 16 * 8;       // 3 digits x 16 blocks x (v / 4 <= 8) words
+constexpr int IM_MISC_BYTES = 16 + IM_SLOTS * IM_CWARPS * 8 * (int)sizeof(ImScale) + IM_CWARPS * 4;
+constexpr int IM_PLANE_WORDS = 3 * IM_PW * 5;    // all K-slices together: 3 digits x 256 blocks x (v / 4 <= 5) words
 
-__host__ __device__ inline ImSmem im_smem_layout(int tab_bytes, int tile_ints)
+__host__ __device__ inline ImSmem im_smem_layout(int tab_bytes, int cols, int rows)
 {
     ImSmem L;
     uint32_t o = 0;
@@ -157,28 +167,26 @@ __host__ __device__ inline ImSmem im_smem_layout(int tab_bytes, int tile_ints)
     o = (o + 15u) & ~15u;
     L.misc = o; o += IM_MISC_BYTES;
     o = (o + 15u) & ~15u;
-    L.planes = o; o += IM_CWARPS * IM_PLANE_WORDS * 4;
+    L.planes = o; o += IM_PLANE_WORDS * 4;
     o = (o + 127u) & ~127u;
     L.tab = o; o += (uint32_t)tab_bytes;
-    o = (o + 127u) & ~127u;
+    o = (o + 1023u) & ~1023u;                     // swizzled TMA boxes want 1024-byte alignment
     L.ring = o; o += IM_STAGES * IM_STAGE_BYTES;
-    L.part = o; o += 2u * IM_CWARPS * (uint32_t)tile_ints * 4u;
-    L.acc = o; o += (uint32_t)IM_RC * (uint32_t)tile_ints * 4u;
+    L.part = o; o += 2u * IM_CWARPS * 16u * (uint32_t)cols * 4u;           // one 16-row tile per compute warp
+    L.acc = o; o += (uint32_t)IM_RC * (uint32_t)rows * (uint32_t)(cols / 2) * 8u;
     L.total = o;
     return L;
 }
 
-// Row groups [lo, hi) of layer P that fall to CTA `b` of `nb`: the launch's work is laid on a line of
-// length cost_total (a row group of a layer costs its Kb), cut into nb equal stretches; a row group
-// belongs to the stretch its first point lies in.
-__device__ __forceinline__ void im_group_range(const ImProblem &P, long long cost_total, int b, int nb, int &lo, int &hi)
+// Row groups [lo, hi) of layer P that fall to this CTA: the launch's work is laid on a line (a row
+// group of a layer costs its Kb), cut into one stretch [a0, a1) per CTA; a row group belongs to the
+// stretch its first point lies in.
+__device__ __forceinline__ void im_group_range(const ImProblem &P, int a0, int a1, int &lo, int &hi)
 {
-    const long long a0 = cost_total * b / nb, a1 = cost_total * (b + 1) / nb;
-    long long l = (a0 - P.cost_base + P.Kb - 1) / P.Kb, h = (a1 - P.cost_base + P.Kb - 1) / P.Kb;
-    if (a0 <= P.cost_base) l = 0;
-    if (a1 <= P.cost_base) h = 0;
-    lo = (int)(l < P.groups ? l : P.groups);
-    hi = (int)(h < P.groups ? h : P.groups);
+    const int l = (a0 <= P.cost_base) ? 0 : (a0 - P.cost_base + P.Kb - 1) / P.Kb;
+    const int h = (a1 <= P.cost_base) ? 0 : (a1 - P.cost_base + P.Kb - 1) / P.Kb;
+    lo = min(l, P.groups);
+    hi = min(h, P.groups);
 }
 
 template <int NCLS, int NM>
@@ -189,12 +197,16 @@ gemv_imma_kernel(const __grid_constant__ ImBatch batch)
     constexpr int TRK = (NM == 1) ? 2 : 1;               // 16-row tiles per row group
     constexpr int ROWS = TRK * 16;
     constexpr int COLS = 8 * NM;
-    constexpr int TILE_INTS = ROWS * COLS;
+    constexpr int TILE_INTS = 16 * COLS;                 // one compute warp's partial tile
+    constexpr int KS = 16 / TRK;                         // K-slices of a part; warp w: slice w % KS, tile w / KS
+    constexpr int SLICE = IM_PW / KS;                    // blocks per slice
+    constexpr int BPL = SLICE / 4;                       // blocks per lane
     constexpr int MAXM = (NM == 1) ? 2 : (NM == 2 ? 5 : 8);
-    const ImSmem L = im_smem_layout(batch.tab_smem_bytes, TILE_INTS);
+    const ImSmem L = im_smem_layout(batch.tab_smem_bytes, COLS, ROWS);
     uint64_t *bars = reinterpret_cast<uint64_t *>(smem + L.bars);
     volatile int *s_abort = reinterpret_cast<volatile int *>(smem + L.misc);
     ImScale *s_scale = reinterpret_cast<ImScale *>(smem + L.misc + 16);           // [IM_SLOTS][16 warps][8]
+    float *s_xmax = reinterpret_cast<float *>(smem + L.misc + 16 + IM_SLOTS * IM_CWARPS * 8 * sizeof(ImScale));   // [16 warps]
     uint32_t *s_planes = reinterpret_cast<uint32_t *>(smem + L.planes);
     uint32_t *s_tab = reinterpret_cast<uint32_t *>(smem + L.tab);
     unsigned char *s_ring = smem + L.ring;
@@ -221,6 +233,8 @@ gemv_imma_kernel(const __grid_constant__ ImBatch batch)
     __syncthreads();
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const bool tab_smem = batch.tab_smem_bytes > 0;
+    const int cost_a0 = batch.cost_per * (int)blockIdx.x + min((int)blockIdx.x, batch.cost_rem);
+    const int cost_a1 = cost_a0 + batch.cost_per + ((int)blockIdx.x < batch.cost_rem ? 1 : 0);
 
     // All three roles walk the same sequence: layers pi (those with row groups for this CTA, counted
     // by ps), chunks [c0, c1) of at most IM_RC row groups, K-parts j (counted by pc), row groups r; li
@@ -232,7 +246,7 @@ gemv_imma_kernel(const __grid_constant__ ImBatch batch)
         for (int pi = 0; pi < batch.count && ok; ++pi) {
             const ImProblem &P = batch.p[pi];
             int glo, ghi;
-            im_group_range(P, batch.cost_total, blockIdx.x, gridDim.x, glo, ghi);
+            im_group_range(P, cost_a0, cost_a1, glo, ghi);
             if (glo >= ghi) continue;
             if (tab_smem) {
                 if (ps > 0 && !im_mbar_wait(bar_tabfree, (ps - 1) & 1, s_abort)) break;
@@ -247,29 +261,17 @@ gemv_imma_kernel(const __grid_constant__ ImBatch batch)
                 const int c1 = min(c0 + IM_RC, ghi);
                 for (int j = 0; j < P.parts && ok; ++j) {
                     const int pw = min(IM_PW, P.Kb - j * IM_PW);          // blocks of this part
-                    const uint32_t row_bytes = (uint32_t)pw * 2u;
                     for (int r = c0; r < c1; ++r, ++li) {
                         const int s = li % IM_STAGES;
                         if (li >= IM_STAGES && !im_mbar_wait(bar_empty(s), ((li / IM_STAGES) & 1) ^ 1, s_abort)) { ok = false; break; }
-                        const int row0 = r * ROWS;
-                        const int rows = min(ROWS, P.N - row0);
-                        unsigned char *stage = s_ring + (size_t)s * IM_STAGE_BYTES;
-                        const uint16_t *src = P.idx + (size_t)row0 * P.Kb + (size_t)j * IM_PW;
-                        // rows past N: zeros (index 0 is always valid)
-                        if (rows < ROWS) {
-                            uint32_t *z = reinterpret_cast<uint32_t *>(stage + (size_t)rows * row_bytes);
-                            const int nz = (ROWS - rows) * pw / 2;
-                            for (int i = lane; i < nz; i += 32) z[i] = 0u;
-                        }
+                        // boxes of 64 blocks x ROWS rows; rows past N and blocks past K/v arrive as zeros
+                        const int nbox = (pw + IM_BOX_COLS - 1) / IM_BOX_COLS;
+                        constexpr uint32_t BOX_BYTES = ROWS * 128;
+                        if (lane == 0) im_mbar_expect_tx(bar_full(s), (uint32_t)nbox * BOX_BYTES);
                         __syncwarp();
-                        if (lane == 0) im_mbar_expect_tx(bar_full(s), (uint32_t)rows * row_bytes);
-                        __syncwarp();
-                        if (P.parts == 1) {
-                            // the rows of the group are contiguous in memory: one copy
-                            if (lane == 0) im_bulk_g2s(im_smem_u32(stage), src, (uint32_t)rows * row_bytes, bar_full(s));
-                        } else if (lane < rows) {
-                            im_bulk_g2s(im_smem_u32(stage + (size_t)lane * row_bytes), src + (size_t)lane * P.Kb, row_bytes, bar_full(s));
-                        }
+                        if (lane < nbox)
+                            im_tma_2d(im_smem_u32(s_ring + (size_t)s * IM_STAGE_BYTES + (size_t)lane * BOX_BYTES), &batch.map[pi],
+                                      j * IM_PW + lane * IM_BOX_COLS, r * ROWS, bar_full(s));
                     }
                 }
             }
@@ -278,7 +280,7 @@ gemv_imma_kernel(const __grid_constant__ ImBatch batch)
         // ============================================================ epilogue (two warps)
         // 64 threads = ROWS rows x SPLIT groups of compute warps; the groups of a row sit in adjacent lanes.
         constexpr int SPLIT = (IM_EWARPS * 32) / ROWS;         // 2 or 4
-        constexpr int WPG = IM_CWARPS / SPLIT;                 // compute warps per group
+        constexpr int WPG = KS / SPLIT;                        // compute warps (K-slices) per group: 4
         const int et = (warp - IM_CWARPS - 1) * 32 + lane;
         const int R = et / SPLIT, grp = et % SPLIT;
         asm volatile("griddepcontrol.wait;" ::: "memory");
@@ -287,7 +289,7 @@ gemv_imma_kernel(const __grid_constant__ ImBatch batch)
         for (int pi = 0; pi < batch.count && ok; ++pi) {
             const ImProblem &P = batch.p[pi];
             int glo, ghi;
-            im_group_range(P, batch.cost_total, blockIdx.x, gridDim.x, glo, ghi);
+            im_group_range(P, cost_a0, cost_a1, glo, ghi);
             if (glo >= ghi) continue;
             const double unshift2 = 2.0 / (double)(1 << (P.ncls - 1));
             for (int c0 = glo; c0 < ghi && ok; c0 += IM_RC) {
@@ -309,19 +311,32 @@ gemv_imma_kernel(const __grid_constant__ ImBatch batch)
                         }
                         if (!im_mbar_wait(bar_pfull(buf), (li >> 1) & 1, s_abort)) { ok = false; break; }
                         double *accrow = s_acc + ((size_t)(P.parts > 1 ? (r - c0) : 0) * ROWS + R) * ACC_M;
-                        const int *base = s_part + ((size_t)buf * IM_CWARPS + grp * WPG) * TILE_INTS + (size_t)R * COLS;
+                        // row R lies in tile R / 16, written by the compute warps (R / 16) * KS + slice
+                        const int *base = s_part + ((size_t)buf * IM_CWARPS + (R >> 4) * KS + grp * WPG) * TILE_INTS + (size_t)(R & 15) * COLS;
                         double dots[MAXM], sxp[MAXM];
 #pragma unroll
-                        for (int m = 0; m < MAXM; ++m) {
-                            dots[m] = 0.0; sxp[m] = 0.0;
-                            if (m < P.M) {
+                        for (int m = 0; m < MAXM; ++m) { dots[m] = 0.0; sxp[m] = 0.0; }
 #pragma unroll
-                                for (int w = 0; w < WPG; ++w) {
-                                    const int *pw3 = base + (size_t)w * TILE_INTS + 3 * m;
-                                    const long long T = ((long long)pw3[2] * 256 + pw3[1]) * 256 + pw3[0];
-                                    const ImScale sw = sc[(grp * WPG + w) * 8 + m];
-                                    dots[m] += (double)T * sw.inv;
+                        for (int w = 0; w < WPG; ++w) {
+                            int pv[COLS];
+#pragma unroll
+                            for (int c4 = 0; c4 < COLS / 4; ++c4) {
+                                if (c4 * 4 < 3 * P.M) {                     // columns 3 m + d, m < M
+                                    const int4 q = *reinterpret_cast<const int4 *>(base + (size_t)w * TILE_INTS + c4 * 4);
+                                    pv[c4 * 4] = q.x; pv[c4 * 4 + 1] = q.y; pv[c4 * 4 + 2] = q.z; pv[c4 * 4 + 3] = q.w;
+                                } else {
+                                    pv[c4 * 4] = pv[c4 * 4 + 1] = pv[c4 * 4 + 2] = pv[c4 * 4 + 3] = 0;
+                                }
+                            }
+#pragma unroll
+                            for (int m = 0; m < MAXM; ++m) {
+                                if (m < P.M) {
+                                    const double T = ((double)pv[3 * m + 2] * 256.0 + (double)pv[3 * m + 1]) * 256.0 + (double)pv[3 * m];
+                                    const int slice = grp * WPG + w;
+                                    const ImScale sw = sc[slice * 8 + m];
+                                    dots[m] += T * sw.inv;
                                     sxp[m] += sw.sx;
+                                    if (TRK > 1) sxp[m] += sc[(slice + KS) * 8 + m].sx;      // the slice's other warp
                                 }
                             }
                         }
@@ -357,19 +372,24 @@ gemv_imma_kernel(const __grid_constant__ ImBatch batch)
         constexpr int CT = IM_CWARPS * 32;
         constexpr float MAGIC = 12582912.0f;                   // 1.5 * 2^23: float -> int by addition
         constexpr int MAGIC_BITS = 0x4B400000;
-        uint32_t *planes = s_planes + warp * IM_PLANE_WORDS;
+        const int ks = warp % KS, rh = warp / KS;             // K-slice and tile of this warp
+        // MMA row g (and g + 8) carries tile row sg (and sg + 8): neighbouring g differ in bit 2 of the row, so the
+        // eight lanes of a shared-memory phase read distinct swizzled chunks
+        const int sg = ((g & 1) << 2) | (g >> 1);
+        uint32_t *planes = s_planes + ks * (IM_PLANE_WORDS / KS);
         asm volatile("griddepcontrol.wait;" ::: "memory");
         int li = 0, ps = 0, pc = 0;
         bool ok = true;
         for (int pi = 0; pi < batch.count && ok; ++pi) {
             const ImProblem &P = batch.p[pi];
             int glo, ghi;
-            im_group_range(P, batch.cost_total, blockIdx.x, gridDim.x, glo, ghi);
+            im_group_range(P, cost_a0, cost_a1, glo, ghi);
             if (glo >= ghi) continue;
             const int M = P.M, K = P.K, Kb = P.Kb, v = P.v;
             const int cmax = P.ncls - 1;
             const int PBITS = 22 - cmax;                       // |X| <= 2^PBITS
-            const int nwords = 16 * P.ncls;                    // words per digit plane of a warp's slice
+            const int nwords = SLICE * P.ncls;                 // words per digit plane of a slice
+            const int ngroups = SLICE * v / 8;                 // groups of 8 activations in a slice (<= 80)
             bool tab_ready = !tab_smem;
             const uint32_t *tab = tab_smem ? s_tab : P.tab;
 
@@ -377,30 +397,36 @@ gemv_imma_kernel(const __grid_constant__ ImBatch batch)
                 const int c1 = min(c0 + IM_RC, ghi);
                 for (int j = 0; j < P.parts && ok; ++j, ++pc) {
                     const int pw = min(IM_PW, Kb - j * IM_PW);
-                    const int jb0 = j * IM_PW + warp * 16;          // first block of this warp's slice
-                    const bool wvalid = warp * 16 + 4 * t < pw;     // this lane's four blocks exist (pw % 4 == 0)
+                    const int jb0 = j * IM_PW + ks * SLICE;         // first block of this warp's slice
+                    const bool wvalid = ks * SLICE + BPL * t < pw;  // this lane's blocks exist (pw % 8 == 0)
                     const int kend = (j * IM_PW + pw) * v;          // end of the part in x
                     ImScale *scale_out = s_scale + ((size_t)(pc % IM_SLOTS) * IM_CWARPS + warp) * 8;
 
                     // ---- B fragments for this part.  The warp's slice of each row of x (16 blocks) is
                     //      quantised with its own scale: X = rint(x * 2^(PBITS - e)), 2^e > max |x| of the slice.
-                    uint32_t breg[4][NCLS][NM];
+                    uint32_t breg[BPL][NCLS][NM];
 #pragma unroll
-                    for (int e = 0; e < 4; ++e)
+                    for (int e = 0; e < BPL; ++e)
 #pragma unroll
                         for (int c = 0; c < NCLS; ++c)
 #pragma unroll
                             for (int nm = 0; nm < NM; ++nm) breg[e][c][nm] = 0u;
+                    // The TRK warps of a slice share its planes: each quantises every TRK-th group of 8 activations.
+                    constexpr int NU = (SLICE * 20 / 8 + 32 * TRK - 1) / (32 * TRK);   // groups per lane (v <= 20)
+                    auto slice_sync = [&]() {
+                        if (TRK == 1) __syncwarp();
+                        else im_named_bar(1 + ks, TRK * 32);
+                    };
                     for (int m = 0; m < M; ++m) {
                         const uint16_t *xrow = reinterpret_cast<const uint16_t *>(P.x) + (size_t)m * K;
-                        // groups of 8 activations: lane, lane + 32 (the slice has 2 v <= 64 groups)
-                        uint4 q4[2];
+                        uint4 q4[NU];
                         float amax = 0.f;
 #pragma unroll
-                        for (int u = 0; u < 2; ++u) {
-                            const int k0 = jb0 * v + 8 * (lane + 32 * u);
+                        for (int u = 0; u < NU; ++u) {
+                            const int gi = lane + 32 * (rh + TRK * u);
+                            const int k0 = jb0 * v + 8 * gi;
                             q4[u] = make_uint4(0u, 0u, 0u, 0u);
-                            if (lane + 32 * u < 2 * v && k0 < kend) q4[u] = __ldg(reinterpret_cast<const uint4 *>(xrow + k0));
+                            if (gi < ngroups && k0 < kend) q4[u] = __ldg(reinterpret_cast<const uint4 *>(xrow + k0));
                             const uint32_t wds[4] = {q4[u].x, q4[u].y, q4[u].z, q4[u].w};
 #pragma unroll
                             for (int jj = 0; jj < 4; ++jj) {
@@ -411,15 +437,20 @@ gemv_imma_kernel(const __grid_constant__ ImBatch batch)
                         }
 #pragma unroll
                         for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+                        if (TRK > 1) {
+                            if (lane == 0) s_xmax[warp] = amax;
+                            slice_sync();
+                            amax = fmaxf(s_xmax[ks], s_xmax[ks + KS]);
+                        }
                         // amax = f * 2^e with f in [1, 2) (a float from fp16 / bf16 is normal or zero): |x| < 2^(e+1)
                         const int ex = max((int)((__float_as_uint(amax) >> 23) & 0xffu) - 127 + 1, -100);   // (clamped: bf16 can be tinier)
                         const float sc = (amax > 0.f) ? __uint_as_float((uint32_t)(127 + PBITS - ex) << 23) : 1.0f;
                         const double inv = (amax > 0.f) ? __longlong_as_double((long long)(1023 - PBITS + ex) << 52) : 1.0;
                         int xs = 0;
 #pragma unroll
-                        for (int u = 0; u < 2; ++u) {
-                            const int gi = lane + 32 * u;
-                            if (gi < 2 * v) {
+                        for (int u = 0; u < NU; ++u) {
+                            const int gi = lane + 32 * (rh + TRK * u);
+                            if (gi < ngroups) {
                                 const uint32_t wds[4] = {q4[u].x, q4[u].y, q4[u].z, q4[u].w};
                                 int cpos = (8 * gi) % v;                 // position of the group's first activation in its block
 #pragma unroll
@@ -452,23 +483,23 @@ gemv_imma_kernel(const __grid_constant__ ImBatch batch)
                         if (lane == 0) {
                             ImScale o2;
                             o2.inv = inv;
-                            o2.sx = (double)xs * inv;
+                            o2.sx = (double)xs * inv;                    // this warp's share of sum_k x over the slice
                             scale_out[m] = o2;
                         }
-                        __syncwarp();
+                        slice_sync();
 #pragma unroll
                         for (int nm = 0; nm < NM; ++nm) {
                             const int col = g + 8 * nm;
                             const int mc = col / 3, d = col - 3 * mc;
                             if (mc == m && wvalid) {
 #pragma unroll
-                                for (int e = 0; e < 4; ++e)
+                                for (int e = 0; e < BPL; ++e)
 #pragma unroll
                                     for (int c = 0; c < NCLS; ++c)
-                                        if (c <= cmax) breg[e][c][nm] = planes[d * nwords + (4 * t + e) * P.ncls + c];
+                                        if (c <= cmax) breg[e][c][nm] = planes[d * nwords + (BPL * t + e) * P.ncls + c];
                             }
                         }
-                        __syncwarp();
+                        slice_sync();
                     }
                     if (!tab_ready) {
                         if (!im_mbar_wait(bar_tabfull, ps & 1, s_abort)) { ok = false; break; }
@@ -480,35 +511,42 @@ gemv_imma_kernel(const __grid_constant__ ImBatch batch)
                         const int s = li % IM_STAGES;
                         if (!im_mbar_wait(bar_full(s), (li / IM_STAGES) & 1, s_abort)) { ok = false; break; }
                         const unsigned char *stage = s_ring + (size_t)s * IM_STAGE_BYTES;
-                        uint2 ia[TRK], ib[TRK];
+                        // indices of this lane's BPL blocks, tile rows sg and sg + 8 of tile rh (128-byte swizzle:
+                        // 16-byte chunk c of row q sits at chunk c ^ (q & 7))
+                        uint32_t ia[BPL / 2], ib[BPL / 2];
 #pragma unroll
-                        for (int tr = 0; tr < TRK; ++tr) {
-                            ia[tr] = make_uint2(0u, 0u);
-                            ib[tr] = make_uint2(0u, 0u);
-                            if (wvalid) {
-                                const int col = warp * 16 + 4 * t;
-                                ia[tr] = *reinterpret_cast<const uint2 *>(stage + ((size_t)(tr * 16 + g) * pw + col) * 2);
-                                ib[tr] = *reinterpret_cast<const uint2 *>(stage + ((size_t)(tr * 16 + g + 8) * pw + col) * 2);
+                        for (int i = 0; i < BPL / 2; ++i) { ia[i] = 0u; ib[i] = 0u; }
+                        if (wvalid) {
+                            const int boff = (ks * SLICE + BPL * t) * 2;            // byte offset in the part's row
+                            const int row = rh * 16 + sg;
+                            const unsigned char *pa = stage + (size_t)(boff >> 7) * (ROWS * 128) + (size_t)row * 128
+                                                      + ((((boff >> 4) & 7) ^ (row & 7)) << 4) + (boff & 15);
+                            const unsigned char *pb = pa + 8 * 128;                 // row + 8: same row & 7
+                            if (BPL == 8) {
+                                const uint4 qa = *reinterpret_cast<const uint4 *>(pa), qb = *reinterpret_cast<const uint4 *>(pb);
+                                ia[0] = qa.x; ia[1] = qa.y; ia[BPL / 2 - 2] = qa.z; ia[BPL / 2 - 1] = qa.w;
+                                ib[0] = qb.x; ib[1] = qb.y; ib[BPL / 2 - 2] = qb.z; ib[BPL / 2 - 1] = qb.w;
+                            } else {
+                                const uint2 qa = *reinterpret_cast<const uint2 *>(pa), qb = *reinterpret_cast<const uint2 *>(pb);
+                                ia[0] = qa.x; ia[1] = qa.y;
+                                ib[0] = qb.x; ib[1] = qb.y;
                             }
                         }
                         __syncwarp();
                         if (lane == 0) im_mbar_arrive(bar_empty(s));
 
-                        int acc[TRK][NM][4];
+                        int acc[NM][4];
 #pragma unroll
-                        for (int tr = 0; tr < TRK; ++tr)
+                        for (int nm = 0; nm < NM; ++nm)
 #pragma unroll
-                            for (int nm = 0; nm < NM; ++nm)
+                            for (int i = 0; i < 4; ++i) acc[nm][i] = 0;
+                        if (ks * SLICE < pw) {                      // warp-uniform: the slice is not empty
 #pragma unroll
-                                for (int i = 0; i < 4; ++i) acc[tr][nm][i] = 0;
-                        if (warp * 16 < pw) {                       // warp-uniform: the slice is not empty
-#pragma unroll
-                            for (int tr = 0; tr < TRK; ++tr) {
+                            for (int e4 = 0; e4 < BPL; e4 += 4) {
                                 uint32_t w0[4], w1[4];
 #pragma unroll
                                 for (int e = 0; e < 4; ++e) {
-                                    const uint32_t pa = (e < 2) ? ia[tr].x : ia[tr].y;
-                                    const uint32_t pb = (e < 2) ? ib[tr].x : ib[tr].y;
+                                    const uint32_t pa = ia[(e4 + e) >> 1], pb = ib[(e4 + e) >> 1];
                                     const uint32_t i0 = (e & 1) ? (pa >> 16) : (pa & 0xffffu);
                                     const uint32_t i1 = (e & 1) ? (pb >> 16) : (pb & 0xffffu);
                                     w0[e] = tab_smem ? tab[i0] : __ldg(tab + i0);
@@ -521,8 +559,8 @@ gemv_imma_kernel(const __grid_constant__ ImBatch batch)
                                         const uint32_t ma = 0x01010101u << (2 * cp), mb = 0x01010101u << (2 * cp + 1);
 #pragma unroll
                                         for (int nm = 0; nm < NM; ++nm)
-                                            im_mma_u8s8(acc[tr][nm], w0[e] & ma, w1[e] & ma, w0[e] & mb, w1[e] & mb,
-                                                        breg[e][2 * cp][nm], breg[e][2 * cp + 1][nm]);
+                                            im_mma_u8s8(acc[nm], w0[e] & ma, w1[e] & ma, w0[e] & mb, w1[e] & mb,
+                                                        breg[e4 + e][2 * cp][nm], breg[e4 + e][2 * cp + 1][nm]);
                                     }
                                 }
                                 if (NCLS & 1) {
@@ -531,8 +569,8 @@ gemv_imma_kernel(const __grid_constant__ ImBatch batch)
                                     for (int ep = 0; ep < 2; ++ep)
 #pragma unroll
                                         for (int nm = 0; nm < NM; ++nm)
-                                            im_mma_u8s8(acc[tr][nm], w0[2 * ep] & ml, w1[2 * ep] & ml, w0[2 * ep + 1] & ml,
-                                                        w1[2 * ep + 1] & ml, breg[2 * ep][NCLS - 1][nm], breg[2 * ep + 1][NCLS - 1][nm]);
+                                            im_mma_u8s8(acc[nm], w0[2 * ep] & ml, w1[2 * ep] & ml, w0[2 * ep + 1] & ml,
+                                                        w1[2 * ep + 1] & ml, breg[e4 + 2 * ep][NCLS - 1][nm], breg[e4 + 2 * ep + 1][NCLS - 1][nm]);
                                 }
                             }
                         }
@@ -540,12 +578,10 @@ gemv_imma_kernel(const __grid_constant__ ImBatch batch)
                         if (li >= 2 && !im_mbar_wait(bar_pempty(buf), ((li >> 1) & 1) ^ 1, s_abort)) { ok = false; break; }
                         int *mine = s_part + ((size_t)buf * IM_CWARPS + warp) * TILE_INTS;
 #pragma unroll
-                        for (int tr = 0; tr < TRK; ++tr)
-#pragma unroll
-                            for (int nm = 0; nm < NM; ++nm) {
-                                *reinterpret_cast<int2 *>(mine + (tr * 16 + g) * COLS + nm * 8 + 2 * t) = make_int2(acc[tr][nm][0], acc[tr][nm][1]);
-                                *reinterpret_cast<int2 *>(mine + (tr * 16 + g + 8) * COLS + nm * 8 + 2 * t) = make_int2(acc[tr][nm][2], acc[tr][nm][3]);
-                            }
+                        for (int nm = 0; nm < NM; ++nm) {
+                            *reinterpret_cast<int2 *>(mine + sg * COLS + nm * 8 + 2 * t) = make_int2(acc[nm][0], acc[nm][1]);
+                            *reinterpret_cast<int2 *>(mine + (sg + 8) * COLS + nm * 8 + 2 * t) = make_int2(acc[nm][2], acc[nm][3]);
+                        }
                         __syncwarp();
                         if (lane == 0) im_mbar_arrive(bar_pfull(buf));
                     }
@@ -562,6 +598,23 @@ gemv_imma_kernel(const __grid_constant__ ImBatch batch)
 }
 
 // ------------------------------------------------------------------------------------ host side
+typedef CUresult (*im_encode_fn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                 const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                 CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static im_encode_fn im_get_encode()
+{
+    static im_encode_fn fn = nullptr;
+    if (!fn) {
+        void *ptr = nullptr;
+        cudaDriverEntryPointQueryResult qr;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qr) == cudaSuccess &&
+            qr == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<im_encode_fn>(ptr);
+    }
+    return fn;
+}
+
 static int im_sm_count()
 {
     static int n = 0;
@@ -574,16 +627,19 @@ static int im_sm_count()
 }
 
 template <int NCLS, int NM>
-static int im_launch(const ImBatch &b, int groups_total, cudaStream_t s)
+static int im_launch(ImBatch &b, int groups_total, cudaStream_t s)
 {
     constexpr int TRK = (NM == 1) ? 2 : 1;
-    const ImSmem L = im_smem_layout(b.tab_smem_bytes, TRK * 16 * 8 * NM);
+    const ImSmem L = im_smem_layout(b.tab_smem_bytes, 8 * NM, TRK * 16);
     auto kern = gemv_imma_kernel<NCLS, NM>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)L.total);
     if (e != cudaSuccess) return cuda_fail(e);
     cudaLaunchConfig_t cfg = {};
     const int sms = im_sm_count();
-    cfg.gridDim = dim3((unsigned)(groups_total < sms ? groups_total : sms));
+    const int grid = groups_total < sms ? groups_total : sms;
+    b.cost_per = b.cost_total / grid;
+    b.cost_rem = b.cost_total % grid;
+    cfg.gridDim = dim3((unsigned)grid);
     cfg.blockDim = dim3(IM_THREADS);
     cfg.dynamicSmemBytes = L.total;
     cfg.stream = s;
@@ -597,7 +653,7 @@ static int im_launch(const ImBatch &b, int groups_total, cudaStream_t s)
 }
 
 template <int NCLS>
-static int im_launch_nm(const ImBatch &b, int nm, int groups_total, cudaStream_t s)
+static int im_launch_nm(ImBatch &b, int nm, int groups_total, cudaStream_t s)
 {
     if (nm == 1) return im_launch<NCLS, 1>(b, groups_total, s);
     if (nm == 2) return im_launch<NCLS, 2>(b, groups_total, s);
@@ -607,6 +663,8 @@ static int im_launch_nm(const ImBatch &b, int nm, int groups_total, cudaStream_t
 int launch_gemv_imma(const LinearArgs *problems, int count, cudaStream_t s)
 {
     if (count < 1 || count > IM_MAXP) return BTC_ERR_UNSUPPORTED;
+    im_encode_fn enc = im_get_encode();
+    if (!enc) return BTC_ERR_UNSUPPORTED;
     ImBatch b = {};
     b.count = count;
     int ncls_max = 0, m_max = 0, tab_max = 0;
@@ -618,7 +676,7 @@ int launch_gemv_imma(const LinearArgs *problems, int count, cudaStream_t s)
     }
     const int nm = m_max <= 2 ? 1 : (m_max <= 5 ? 2 : 3);
     const int rows = (nm == 1) ? 32 : 16;
-    long long cost = 0;
+    long long cost = 0;                              // must stay below 2^31
     int groups_total = 0;
     for (int i = 0; i < count; ++i) {
         const LinearArgs &a = problems[i];
@@ -631,15 +689,26 @@ int launch_gemv_imma(const LinearArgs *problems, int count, cudaStream_t s)
         p.parts = (a.Kb + IM_PW - 1) / IM_PW;
         p.groups = (a.N + rows - 1) / rows;
         p.ncls = a.v / 4;
-        p.cost_base = cost;
+        {
+            const cuuint64_t dims[2] = {(cuuint64_t)a.Kb, (cuuint64_t)a.N};
+            const cuuint64_t strides[1] = {(cuuint64_t)a.Kb * 2};
+            const cuuint32_t box[2] = {(cuuint32_t)IM_BOX_COLS, (cuuint32_t)rows};
+            const cuuint32_t estr[2] = {1, 1};
+            if (enc(&b.map[i], CU_TENSOR_MAP_DATA_TYPE_UINT16, 2, const_cast<uint16_t *>(a.idx), dims, strides, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+                return BTC_ERR_UNSUPPORTED;                 // shape the tensor map cannot describe: other kernels take it
+        }
+        p.cost_base = (int)cost;
         cost += (long long)p.groups * a.Kb;
         groups_total += p.groups;
         if (p.ncls > ncls_max) ncls_max = p.ncls;
         if (Kc4 * 4 > tab_max) tab_max = Kc4 * 4;
     }
-    b.cost_total = cost;
+    if (cost >= (1ll << 31)) return BTC_ERR_UNSUPPORTED;
+    b.cost_total = (int)cost;
     b.tab_smem_bytes = tab_max;
-    if (im_smem_layout(tab_max, rows * 8 * nm).total > 227u * 1024u) b.tab_smem_bytes = 0;   // gather from global (L1/L2)
+    if (im_smem_layout(tab_max, 8 * nm, rows).total > 227u * 1024u) b.tab_smem_bytes = 0;   // gather from global (L1/L2)
     if (ncls_max <= 4) return im_launch_nm<4>(b, nm, groups_total, s);
     return im_launch_nm<5>(b, nm, groups_total, s);
 }
