@@ -157,7 +157,7 @@ constexpr int IM_NBARS = 2 * IM_STAGES + 6;
 constexpr int IM_SLOTS = 4;                      // scale slots: K-parts whose partial sums may still be in flight
 struct ImScale { double inv; double sx; };       // per (slot, compute warp, row m of x): 1/scale, and sum_k x over the slice
 constexpr int IM_MISC_BYTES = 16 + IM_SLOTS * IM_CWARPS * 8 * (int)sizeof(ImScale) + IM_CWARPS * 4;
-constexpr int IM_PLANE_WORDS = 3 * IM_PW * 5;    // all K-slices together: 3 digits x 256 blocks x (v / 4 <= 5) words
+constexpr int IM_PLANE_WORDS = 3 * (IM_PW + 64) * 5;   // all K-slices: 3 digits x (256 blocks + skew) x (v / 4 <= 5) words
 
 __host__ __device__ inline ImSmem im_smem_layout(int tab_bytes, int cols, int rows)
 {
@@ -376,7 +376,10 @@ gemv_imma_kernel(const __grid_constant__ ImBatch batch)
         // MMA row g (and g + 8) carries tile row sg (and sg + 8): neighbouring g differ in bit 2 of the row, so the
         // eight lanes of a shared-memory phase read distinct swizzled chunks
         const int sg = ((g & 1) << 2) | (g >> 1);
-        uint32_t *planes = s_planes + ks * (IM_PLANE_WORDS / KS);
+        // digit planes of a slice: block b, class c of digit d at word d * PSW + (b + b / BPL) * NCLS + c; the skew
+        // puts the lanes of a fragment read (t: blocks BPL apart, d: planes) on different banks
+        constexpr int PSW = (SLICE + 4) * NCLS;
+        uint32_t *planes = s_planes + ks * (3 * PSW);
         asm volatile("griddepcontrol.wait;" ::: "memory");
         int li = 0, ps = 0, pc = 0;
         bool ok = true;
@@ -388,7 +391,6 @@ gemv_imma_kernel(const __grid_constant__ ImBatch batch)
             const int M = P.M, K = P.K, Kb = P.Kb, v = P.v;
             const int cmax = P.ncls - 1;
             const int PBITS = 22 - cmax;                       // |X| <= 2^PBITS
-            const int nwords = SLICE * P.ncls;                 // words per digit plane of a slice
             const int ngroups = SLICE * v / 8;                 // groups of 8 activations in a slice (<= 80)
             bool tab_ready = !tab_smem;
             const uint32_t *tab = tab_smem ? s_tab : P.tab;
@@ -452,12 +454,14 @@ gemv_imma_kernel(const __grid_constant__ ImBatch batch)
                             const int gi = lane + 32 * (rh + TRK * u);
                             if (gi < ngroups) {
                                 const uint32_t wds[4] = {q4[u].x, q4[u].y, q4[u].z, q4[u].w};
-                                int cpos = (8 * gi) % v;                 // position of the group's first activation in its block
+                                int blk = (8 * gi) / v;                  // block of the group's first activation in the slice
+                                int cpos = 8 * gi - blk * v;             // and its position in that block
 #pragma unroll
                                 for (int h = 0; h < 2; ++h) {
                                     const int c = cpos >> 2;
+                                    const int wi = (blk + blk / BPL) * NCLS + c;
                                     cpos += 4;
-                                    if (cpos >= v) cpos -= v;
+                                    if (cpos >= v) { cpos -= v; ++blk; }
                                     const uint32_t sh = 1u << (cmax - c);
                                     const uint32_t off = 0x8080u - (uint32_t)MAGIC_BITS * sh;    // arithmetic modulo 2^32
                                     float f0, f1, f2, f3;
@@ -468,12 +472,11 @@ gemv_imma_kernel(const __grid_constant__ ImBatch batch)
                                     xs += (int)(b0 + b1 + b2 + b3 - 4u * (uint32_t)MAGIC_BITS);
                                     // Y = X * 2^(cmax - c) + 0x8080: byte d of Y is balanced digit d of X * 2^(cmax-c), + 0x80 for d < 2
                                     const uint32_t y0 = b0 * sh + off, y1 = b1 * sh + off, y2 = b2 * sh + off, y3 = b3 * sh + off;
-                                    const int wi = 2 * gi + h;
 #pragma unroll
                                     for (int d = 0; d < 3; ++d) {
                                         const uint32_t sel = (uint32_t)d | ((uint32_t)(4 + d) << 4);
                                         const uint32_t lo2 = __byte_perm(y0, y1, sel), hi2 = __byte_perm(y2, y3, sel);
-                                        planes[d * nwords + wi] = __byte_perm(lo2, hi2, 0x5410) ^ (d < 2 ? 0x80808080u : 0u);
+                                        planes[d * PSW + wi] = __byte_perm(lo2, hi2, 0x5410) ^ (d < 2 ? 0x80808080u : 0u);
                                     }
                                 }
                             }
@@ -492,11 +495,17 @@ gemv_imma_kernel(const __grid_constant__ ImBatch batch)
                             const int col = g + 8 * nm;
                             const int mc = col / 3, d = col - 3 * mc;
                             if (mc == m && wvalid) {
+                                const uint32_t *src = planes + d * PSW + (BPL * t + t) * NCLS;
 #pragma unroll
-                                for (int e = 0; e < BPL; ++e)
+                                for (int e = 0; e < BPL; ++e) {
+                                    if (NCLS == 4) {
+                                        const uint4 q = *reinterpret_cast<const uint4 *>(src + e * 4);
+                                        breg[e][0][nm] = q.x; breg[e][1][nm] = q.y; breg[e][2][nm] = q.z; breg[e][NCLS - 1][nm] = q.w;
+                                    } else {
 #pragma unroll
-                                    for (int c = 0; c < NCLS; ++c)
-                                        if (c <= cmax) breg[e][c][nm] = planes[d * nwords + (BPL * t + e) * P.ncls + c];
+                                        for (int c = 0; c < NCLS; ++c) breg[e][c][nm] = src[e * NCLS + c];
+                                    }
+                                }
                             }
                         }
                         slice_sync();
