@@ -150,12 +150,13 @@ struct ImSmem {
     uint32_t tab;         // codeword table
     uint32_t ring;        // index stages
     uint32_t part;        // partial sums [2][16 warps][rows][cols]
-    uint32_t acc;         // dot products summed over K-parts, double [IM_RC][rows][cols / 2]
+    uint32_t acc;         // dot products summed over K-parts, float [IM_RC][rows][cols / 2]
     uint32_t total;
 };
 constexpr int IM_NBARS = 2 * IM_STAGES + 6;
 constexpr int IM_SLOTS = 4;                      // scale slots: K-parts whose partial sums may still be in flight
-struct ImScale { double inv; double sx; };       // per (slot, compute warp, row m of x): 1/scale, and sum_k x over the slice
+struct ImScale { float inv; float sx; };         // per (slot, compute warp, row m of x): 1/scale (a power of two), and
+                                                 // the warp's share of sum_k x over the slice
 constexpr int IM_MISC_BYTES = 16 + IM_SLOTS * IM_CWARPS * 8 * (int)sizeof(ImScale) + IM_CWARPS * 4;
 constexpr int IM_PLANE_WORDS = 3 * (IM_PW + 64) * 5;   // all K-slices: 3 digits x (256 blocks + skew) x (v / 4 <= 5) words
 
@@ -173,7 +174,7 @@ __host__ __device__ inline ImSmem im_smem_layout(int tab_bytes, int cols, int ro
     o = (o + 1023u) & ~1023u;                     // swizzled TMA boxes want 1024-byte alignment
     L.ring = o; o += IM_STAGES * IM_STAGE_BYTES;
     L.part = o; o += 2u * IM_CWARPS * 16u * (uint32_t)cols * 4u;           // one 16-row tile per compute warp
-    L.acc = o; o += (uint32_t)IM_RC * (uint32_t)rows * (uint32_t)(cols / 2) * 8u;
+    L.acc = o; o += (uint32_t)IM_RC * (uint32_t)rows * (uint32_t)(cols / 2) * 4u;
     L.total = o;
     return L;
 }
@@ -211,8 +212,8 @@ gemv_imma_kernel(const __grid_constant__ ImBatch batch)
     uint32_t *s_tab = reinterpret_cast<uint32_t *>(smem + L.tab);
     unsigned char *s_ring = smem + L.ring;
     int *s_part = reinterpret_cast<int *>(smem + L.part);
-    double *s_acc = reinterpret_cast<double *>(smem + L.acc);
-    constexpr int ACC_M = COLS / 2;                      // doubles per row of s_acc (>= MAXM)
+    float *s_acc = reinterpret_cast<float *>(smem + L.acc);
+    constexpr int ACC_M = COLS / 2;                      // floats per row of s_acc (>= MAXM)
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     auto bar_full = [&](int s) { return im_smem_u32(bars + s); };
@@ -291,15 +292,18 @@ gemv_imma_kernel(const __grid_constant__ ImBatch batch)
             int glo, ghi;
             im_group_range(P, cost_a0, cost_a1, glo, ghi);
             if (glo >= ghi) continue;
-            const double unshift2 = 2.0 / (double)(1 << (P.ncls - 1));
+            const float unshift2 = 2.0f / (float)(1 << (P.ncls - 1));
             for (int c0 = glo; c0 < ghi && ok; c0 += IM_RC) {
                 const int c1 = min(c0 + IM_RC, ghi);
-                double sxtot[MAXM];                              // sum_k x[m, k] over the parts seen so far
+                float sxtot[MAXM];                               // sum_k x[m, k] over the parts seen so far
 #pragma unroll
-                for (int m = 0; m < MAXM; ++m) sxtot[m] = 0.0;
+                for (int m = 0; m < MAXM; ++m) sxtot[m] = 0.f;
                 for (int j = 0; j < P.parts && ok; ++j, ++pc) {
                     const bool last = (j == P.parts - 1);
                     const ImScale *sc = s_scale + (size_t)(pc % IM_SLOTS) * IM_CWARPS * 8;
+                    float sxp[MAXM];                             // sum_k x[m, k] over this part (fixed order of warps)
+#pragma unroll
+                    for (int m = 0; m < MAXM; ++m) sxp[m] = 0.f;
                     for (int r = c0; r < c1; ++r, ++li) {
                         const int buf = li & 1;
                         const int n = r * ROWS + R;
@@ -310,12 +314,20 @@ gemv_imma_kernel(const __grid_constant__ ImBatch batch)
                             if (P.mu) mu = __half2float(P.mu[n]);
                         }
                         if (!im_mbar_wait(bar_pfull(buf), (li >> 1) & 1, s_abort)) { ok = false; break; }
-                        double *accrow = s_acc + ((size_t)(P.parts > 1 ? (r - c0) : 0) * ROWS + R) * ACC_M;
+                        if (r == c0) {
+#pragma unroll
+                            for (int m = 0; m < MAXM; ++m)
+                                if (m < P.M)
+                                    for (int w = 0; w < IM_CWARPS; ++w) sxp[m] += sc[w * 8 + m].sx;
+#pragma unroll
+                            for (int m = 0; m < MAXM; ++m) sxtot[m] += sxp[m];
+                        }
+                        float *accrow = s_acc + ((size_t)(P.parts > 1 ? (r - c0) : 0) * ROWS + R) * ACC_M;
                         // row R lies in tile R / 16, written by the compute warps (R / 16) * KS + slice
                         const int *base = s_part + ((size_t)buf * IM_CWARPS + (R >> 4) * KS + grp * WPG) * TILE_INTS + (size_t)(R & 15) * COLS;
-                        double dots[MAXM], sxp[MAXM];
+                        float dots[MAXM];
 #pragma unroll
-                        for (int m = 0; m < MAXM; ++m) { dots[m] = 0.0; sxp[m] = 0.0; }
+                        for (int m = 0; m < MAXM; ++m) dots[m] = 0.f;
 #pragma unroll
                         for (int w = 0; w < WPG; ++w) {
                             int pv[COLS];
@@ -331,12 +343,9 @@ gemv_imma_kernel(const __grid_constant__ ImBatch batch)
 #pragma unroll
                             for (int m = 0; m < MAXM; ++m) {
                                 if (m < P.M) {
-                                    const double T = ((double)pv[3 * m + 2] * 256.0 + (double)pv[3 * m + 1]) * 256.0 + (double)pv[3 * m];
-                                    const int slice = grp * WPG + w;
-                                    const ImScale sw = sc[slice * 8 + m];
-                                    dots[m] += T * sw.inv;
-                                    sxp[m] += sw.sx;
-                                    if (TRK > 1) sxp[m] += sc[(slice + KS) * 8 + m].sx;      // the slice's other warp
+                                    // each digit sum is below 2^24 in magnitude, so the conversions are exact
+                                    const float T = ((float)pv[3 * m + 2] * 256.0f + (float)pv[3 * m + 1]) * 256.0f + (float)pv[3 * m];
+                                    dots[m] += T * sc[(grp * WPG + w) * 8 + m].inv;
                                 }
                             }
                         }
@@ -346,18 +355,14 @@ gemv_imma_kernel(const __grid_constant__ ImBatch batch)
                         for (int m = 0; m < MAXM; ++m) {
                             if (m < P.M) {
 #pragma unroll
-                                for (int o = 1; o < SPLIT; o <<= 1) {
-                                    dots[m] += __shfl_xor_sync(0xffffffffu, dots[m], o);
-                                    sxp[m] += __shfl_xor_sync(0xffffffffu, sxp[m], o);
-                                }
-                                if (r == c0) sxtot[m] += sxp[m];
-                                double dot = dots[m] * unshift2 - sxp[m];       // 2 * sum_{bit=1} x - sum x over this part
+                                for (int o = 1; o < SPLIT; o <<= 1) dots[m] += __shfl_xor_sync(0xffffffffu, dots[m], o);
+                                float dot = dots[m] * unshift2 - sxp[m];        // 2 * sum_{bit=1} x - sum x over this part
                                 if (grp == 0) {
                                     if (j > 0) dot += accrow[m];
                                     if (!last) accrow[m] = dot;
                                 }
                                 if (last && live) {
-                                    const float yv = (float)((double)al * dot + (double)mu * sxtot[m]);
+                                    const float yv = al * dot + mu * sxtot[m];
                                     store_from_float(P.y, P.y_dt, (size_t)m * P.N + n, yv);
                                 }
                             }
@@ -447,7 +452,7 @@ gemv_imma_kernel(const __grid_constant__ ImBatch batch)
                         // amax = f * 2^e with f in [1, 2) (a float from fp16 / bf16 is normal or zero): |x| < 2^(e+1)
                         const int ex = max((int)((__float_as_uint(amax) >> 23) & 0xffu) - 127 + 1, -100);   // (clamped: bf16 can be tinier)
                         const float sc = (amax > 0.f) ? __uint_as_float((uint32_t)(127 + PBITS - ex) << 23) : 1.0f;
-                        const double inv = (amax > 0.f) ? __longlong_as_double((long long)(1023 - PBITS + ex) << 52) : 1.0;
+                        const float inv = (amax > 0.f) ? __uint_as_float((uint32_t)(127 - PBITS + ex) << 23) : 1.0f;
                         int xs = 0;
 #pragma unroll
                         for (int u = 0; u < NU; ++u) {
@@ -486,7 +491,7 @@ gemv_imma_kernel(const __grid_constant__ ImBatch batch)
                         if (lane == 0) {
                             ImScale o2;
                             o2.inv = inv;
-                            o2.sx = (double)xs * inv;                    // this warp's share of sum_k x over the slice
+                            o2.sx = (float)xs * inv;                     // this warp's share of sum_k x over the slice
                             scale_out[m] = o2;
                         }
                         slice_sync();
