@@ -39,7 +39,7 @@ namespace btc {
 constexpr int IM_CWARPS = 16;                   // compute warps
 constexpr int IM_EWARPS = 2;                    // epilogue warps
 constexpr int IM_THREADS = (IM_CWARPS + 1 + IM_EWARPS) * 32;
-constexpr int IM_STAGES = 4;
+constexpr int IM_STAGES = 8;                     // most index stages a launch may use (fewer when shared memory is short)
 constexpr int IM_BOX_COLS = 64;                 // blocks per TMA box row: 128 bytes, the swizzle span
 constexpr int IM_STAGE_BYTES = 16 * 1024;       // one iteration's indices: 4 boxes of 32 rows x 128 bytes
 constexpr int IM_PW = 256;                      // blocks per K-part (16 per compute warp)
@@ -70,6 +70,7 @@ struct ImBatch {
     int cost_per, cost_rem;   // the launch's cost line (sum of groups * Kb) cut for the grid: CTA b gets
                               // [per * b + min(b, rem), + per + (b < rem))
     int tab_smem_bytes;       // bytes reserved for the codeword table (0: gather from global memory)
+    int stages;               // index stages in the ring (2 .. IM_STAGES)
 };
 
 // ------------------------------------------------------------------------------------ PTX helpers
@@ -93,12 +94,14 @@ __device__ __forceinline__ bool im_mbar_try(uint32_t bar, uint32_t parity) {
         : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
     return ok != 0;
 }
-// Bounded wait: false (and the CTA-wide abort flag latched) once ~1 s has passed.
+// Bounded wait: false (and the CTA-wide abort flag latched) once ~1 s has passed.  A waiting warp backs off with
+// nanosleep so that it does not take issue slots from the warps it is waiting for.
 __device__ __forceinline__ bool im_mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag) {
     if (im_mbar_try(bar, parity)) return true;
     const long long t0 = clock64();
     int spins = 0;
     while (!im_mbar_try(bar, parity)) {
+        __nanosleep(spins < 4 ? 20 : 100);
         if ((++spins & 255) == 0) {
             if (*abort_flag) return false;
             if (clock64() - t0 > 2000000000LL) {
@@ -160,7 +163,7 @@ struct ImScale { float inv; float sx; };         // per (slot, compute warp, row
 constexpr int IM_MISC_BYTES = 16 + IM_SLOTS * IM_CWARPS * 8 * (int)sizeof(ImScale) + IM_CWARPS * 4;
 constexpr int IM_PLANE_WORDS = 3 * (IM_PW + 64) * 5;   // all K-slices: 3 digits x (256 blocks + skew) x (v / 4 <= 5) words
 
-__host__ __device__ inline ImSmem im_smem_layout(int tab_bytes, int cols, int rows)
+__host__ __device__ inline ImSmem im_smem_layout(int tab_bytes, int cols, int rows, int stages)
 {
     ImSmem L;
     uint32_t o = 0;
@@ -172,7 +175,7 @@ __host__ __device__ inline ImSmem im_smem_layout(int tab_bytes, int cols, int ro
     o = (o + 127u) & ~127u;
     L.tab = o; o += (uint32_t)tab_bytes;
     o = (o + 1023u) & ~1023u;                     // swizzled TMA boxes want 1024-byte alignment
-    L.ring = o; o += IM_STAGES * IM_STAGE_BYTES;
+    L.ring = o; o += (uint32_t)stages * IM_STAGE_BYTES;
     L.part = o; o += 2u * IM_CWARPS * 16u * (uint32_t)cols * 4u;           // one 16-row tile per compute warp
     L.acc = o; o += (uint32_t)IM_RC * (uint32_t)rows * (uint32_t)(cols / 2) * 4u;
     L.total = o;
@@ -203,7 +206,8 @@ gemv_imma_kernel(const __grid_constant__ ImBatch batch)
     constexpr int SLICE = IM_PW / KS;                    // blocks per slice
     constexpr int BPL = SLICE / 4;                       // blocks per lane
     constexpr int MAXM = (NM == 1) ? 2 : (NM == 2 ? 5 : 8);
-    const ImSmem L = im_smem_layout(batch.tab_smem_bytes, COLS, ROWS);
+    const ImSmem L = im_smem_layout(batch.tab_smem_bytes, COLS, ROWS, batch.stages);
+    const int NST = batch.stages;
     uint64_t *bars = reinterpret_cast<uint64_t *>(smem + L.bars);
     volatile int *s_abort = reinterpret_cast<volatile int *>(smem + L.misc);
     ImScale *s_scale = reinterpret_cast<ImScale *>(smem + L.misc + 16);           // [IM_SLOTS][16 warps][8]
@@ -224,7 +228,7 @@ gemv_imma_kernel(const __grid_constant__ ImBatch batch)
     const uint32_t bar_tabfree = im_smem_u32(bars + 2 * IM_STAGES + 5);
 
     if (tid == 0) {
-        for (int s = 0; s < IM_STAGES; ++s) { im_mbar_init(bar_full(s), 1); im_mbar_init(bar_empty(s), IM_CWARPS); }
+        for (int s = 0; s < NST; ++s) { im_mbar_init(bar_full(s), 1); im_mbar_init(bar_empty(s), IM_CWARPS); }
         for (int b = 0; b < 2; ++b) { im_mbar_init(bar_pfull(b), IM_CWARPS); im_mbar_init(bar_pempty(b), IM_EWARPS); }
         im_mbar_init(bar_tabfull, 1);
         im_mbar_init(bar_tabfree, IM_CWARPS);
@@ -263,8 +267,8 @@ gemv_imma_kernel(const __grid_constant__ ImBatch batch)
                 for (int j = 0; j < P.parts && ok; ++j) {
                     const int pw = min(IM_PW, P.Kb - j * IM_PW);          // blocks of this part
                     for (int r = c0; r < c1; ++r, ++li) {
-                        const int s = li % IM_STAGES;
-                        if (li >= IM_STAGES && !im_mbar_wait(bar_empty(s), ((li / IM_STAGES) & 1) ^ 1, s_abort)) { ok = false; break; }
+                        const int s = li % NST;
+                        if (li >= NST && !im_mbar_wait(bar_empty(s), ((li / NST) & 1) ^ 1, s_abort)) { ok = false; break; }
                         // boxes of 64 blocks x ROWS rows; rows past N and blocks past K/v arrive as zeros
                         const int nbox = (pw + IM_BOX_COLS - 1) / IM_BOX_COLS;
                         constexpr uint32_t BOX_BYTES = ROWS * 128;
@@ -522,8 +526,8 @@ gemv_imma_kernel(const __grid_constant__ ImBatch batch)
 
                     // ---- the row groups of the chunk, for this part
                     for (int r = c0; r < c1; ++r, ++li) {
-                        const int s = li % IM_STAGES;
-                        if (!im_mbar_wait(bar_full(s), (li / IM_STAGES) & 1, s_abort)) { ok = false; break; }
+                        const int s = li % NST;
+                        if (!im_mbar_wait(bar_full(s), (li / NST) & 1, s_abort)) { ok = false; break; }
                         const unsigned char *stage = s_ring + (size_t)s * IM_STAGE_BYTES;
                         // indices of this lane's BPL blocks, tile rows sg and sg + 8 of tile rh (128-byte swizzle:
                         // 16-byte chunk c of row q sits at chunk c ^ (q & 7))
@@ -549,11 +553,11 @@ gemv_imma_kernel(const __grid_constant__ ImBatch batch)
                         __syncwarp();
                         if (lane == 0) im_mbar_arrive(bar_empty(s));
 
-                        int acc[NM][4];
+                        int acc[NM][4], acc2[NM][4];                 // two chains: an MMA need not wait for the previous one
 #pragma unroll
                         for (int nm = 0; nm < NM; ++nm)
 #pragma unroll
-                            for (int i = 0; i < 4; ++i) acc[nm][i] = 0;
+                            for (int i = 0; i < 4; ++i) { acc[nm][i] = 0; acc2[nm][i] = 0; }
                         if (ks * SLICE < pw) {                      // warp-uniform: the slice is not empty
 #pragma unroll
                             for (int e4 = 0; e4 < BPL; e4 += 4) {
@@ -573,7 +577,7 @@ gemv_imma_kernel(const __grid_constant__ ImBatch batch)
                                         const uint32_t ma = 0x01010101u << (2 * cp), mb = 0x01010101u << (2 * cp + 1);
 #pragma unroll
                                         for (int nm = 0; nm < NM; ++nm)
-                                            im_mma_u8s8(acc[nm], w0[e] & ma, w1[e] & ma, w0[e] & mb, w1[e] & mb,
+                                            im_mma_u8s8((cp & 1) ? acc2[nm] : acc[nm], w0[e] & ma, w1[e] & ma, w0[e] & mb, w1[e] & mb,
                                                         breg[e4 + e][2 * cp][nm], breg[e4 + e][2 * cp + 1][nm]);
                                     }
                                 }
@@ -588,6 +592,10 @@ gemv_imma_kernel(const __grid_constant__ ImBatch batch)
                                 }
                             }
                         }
+#pragma unroll
+                        for (int nm = 0; nm < NM; ++nm)
+#pragma unroll
+                            for (int i = 0; i < 4; ++i) acc[nm][i] += acc2[nm][i];
                         const int buf = li & 1;
                         if (li >= 2 && !im_mbar_wait(bar_pempty(buf), ((li >> 1) & 1) ^ 1, s_abort)) { ok = false; break; }
                         int *mine = s_part + ((size_t)buf * IM_CWARPS + warp) * TILE_INTS;
@@ -644,7 +652,7 @@ template <int NCLS, int NM>
 static int im_launch(ImBatch &b, int groups_total, cudaStream_t s)
 {
     constexpr int TRK = (NM == 1) ? 2 : 1;
-    const ImSmem L = im_smem_layout(b.tab_smem_bytes, 8 * NM, TRK * 16);
+    const ImSmem L = im_smem_layout(b.tab_smem_bytes, 8 * NM, TRK * 16, b.stages);
     auto kern = gemv_imma_kernel<NCLS, NM>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)L.total);
     if (e != cudaSuccess) return cuda_fail(e);
@@ -722,7 +730,9 @@ int launch_gemv_imma(const LinearArgs *problems, int count, cudaStream_t s)
     if (cost >= (1ll << 31)) return BTC_ERR_UNSUPPORTED;
     b.cost_total = (int)cost;
     b.tab_smem_bytes = tab_max;
-    if (im_smem_layout(tab_max, 8 * nm, rows).total > 227u * 1024u) b.tab_smem_bytes = 0;   // gather from global (L1/L2)
+    if (im_smem_layout(tab_max, 8 * nm, rows, 2).total > 227u * 1024u) b.tab_smem_bytes = 0;   // gather from global (L1/L2)
+    b.stages = IM_STAGES;
+    while (b.stages > 2 && im_smem_layout(b.tab_smem_bytes, 8 * nm, rows, b.stages).total > 227u * 1024u) --b.stages;
     if (ncls_max <= 4) return im_launch_nm<4>(b, nm, groups_total, s);
     return im_launch_nm<5>(b, nm, groups_total, s);
 }
