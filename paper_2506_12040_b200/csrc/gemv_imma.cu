@@ -187,8 +187,10 @@ __host__ __device__ inline ImSmem im_smem_layout(int tab_bytes, int cols, int ro
 // stretch its first point lies in.
 __device__ __forceinline__ void im_group_range(const ImProblem &P, int a0, int a1, int &lo, int &hi)
 {
+    lo = hi = 0;
+    if (a1 <= P.cost_base || a0 >= P.cost_base + P.groups * P.Kb) return;     // (no division for layers of other CTAs)
     const int l = (a0 <= P.cost_base) ? 0 : (a0 - P.cost_base + P.Kb - 1) / P.Kb;
-    const int h = (a1 <= P.cost_base) ? 0 : (a1 - P.cost_base + P.Kb - 1) / P.Kb;
+    const int h = (a1 - P.cost_base + P.Kb - 1) / P.Kb;
     lo = min(l, P.groups);
     hi = min(h, P.groups);
 }
@@ -247,6 +249,8 @@ gemv_imma_kernel(const __grid_constant__ ImBatch batch)
     if (warp == IM_CWARPS) {
         // ============================================================ producer
         int li = 0, ps = 0;
+        int s = 0;                                             // ring stage li % NST; rph = (li / NST) & 1
+        uint32_t rph = 0;
         bool ok = true;
         for (int pi = 0; pi < batch.count && ok; ++pi) {
             const ImProblem &P = batch.p[pi];
@@ -267,8 +271,7 @@ gemv_imma_kernel(const __grid_constant__ ImBatch batch)
                 for (int j = 0; j < P.parts && ok; ++j) {
                     const int pw = min(IM_PW, P.Kb - j * IM_PW);          // blocks of this part
                     for (int r = c0; r < c1; ++r, ++li) {
-                        const int s = li % NST;
-                        if (li >= NST && !im_mbar_wait(bar_empty(s), ((li / NST) & 1) ^ 1, s_abort)) { ok = false; break; }
+                        if (li >= NST && !im_mbar_wait(bar_empty(s), rph ^ 1u, s_abort)) { ok = false; break; }
                         // boxes of 64 blocks x ROWS rows; rows past N and blocks past K/v arrive as zeros
                         const int nbox = (pw + IM_BOX_COLS - 1) / IM_BOX_COLS;
                         constexpr uint32_t BOX_BYTES = ROWS * 128;
@@ -277,6 +280,7 @@ gemv_imma_kernel(const __grid_constant__ ImBatch batch)
                         if (lane < nbox)
                             im_tma_2d(im_smem_u32(s_ring + (size_t)s * IM_STAGE_BYTES + (size_t)lane * BOX_BYTES), &batch.map[pi],
                                       j * IM_PW + lane * IM_BOX_COLS, r * ROWS, bar_full(s));
+                        if (++s == NST) { s = 0; rph ^= 1u; }
                     }
                 }
             }
@@ -391,6 +395,8 @@ gemv_imma_kernel(const __grid_constant__ ImBatch batch)
         uint32_t *planes = s_planes + ks * (3 * PSW);
         asm volatile("griddepcontrol.wait;" ::: "memory");
         int li = 0, ps = 0, pc = 0;
+        int s = 0;                                             // ring stage li % NST; rph = (li / NST) & 1
+        uint32_t rph = 0;
         bool ok = true;
         for (int pi = 0; pi < batch.count && ok; ++pi) {
             const ImProblem &P = batch.p[pi];
@@ -402,7 +408,7 @@ gemv_imma_kernel(const __grid_constant__ ImBatch batch)
             const int PBITS = 22 - cmax;                       // |X| <= 2^PBITS
             const int ngroups = SLICE * v / 8;                 // groups of 8 activations in a slice (<= 80)
             bool tab_ready = !tab_smem;
-            const uint32_t *tab = tab_smem ? s_tab : P.tab;
+            const uint32_t *gtab = P.tab;                      // (s_tab is named directly below so that its loads are shared-memory loads)
 
             for (int c0 = glo; c0 < ghi && ok; c0 += IM_RC) {
                 const int c1 = min(c0 + IM_RC, ghi);
@@ -526,8 +532,7 @@ gemv_imma_kernel(const __grid_constant__ ImBatch batch)
 
                     // ---- the row groups of the chunk, for this part
                     for (int r = c0; r < c1; ++r, ++li) {
-                        const int s = li % NST;
-                        if (!im_mbar_wait(bar_full(s), (li / NST) & 1, s_abort)) { ok = false; break; }
+                        if (!im_mbar_wait(bar_full(s), rph, s_abort)) { ok = false; break; }
                         const unsigned char *stage = s_ring + (size_t)s * IM_STAGE_BYTES;
                         // indices of this lane's BPL blocks, tile rows sg and sg + 8 of tile rh (128-byte swizzle:
                         // 16-byte chunk c of row q sits at chunk c ^ (q & 7))
@@ -552,6 +557,7 @@ gemv_imma_kernel(const __grid_constant__ ImBatch batch)
                         }
                         __syncwarp();
                         if (lane == 0) im_mbar_arrive(bar_empty(s));
+                        if (++s == NST) { s = 0; rph ^= 1u; }
 
                         int acc[NM][4], acc2[NM][4];                 // two chains: an MMA need not wait for the previous one
 #pragma unroll
@@ -567,8 +573,8 @@ gemv_imma_kernel(const __grid_constant__ ImBatch batch)
                                     const uint32_t pa = ia[(e4 + e) >> 1], pb = ib[(e4 + e) >> 1];
                                     const uint32_t i0 = (e & 1) ? (pa >> 16) : (pa & 0xffffu);
                                     const uint32_t i1 = (e & 1) ? (pb >> 16) : (pb & 0xffffu);
-                                    w0[e] = tab_smem ? tab[i0] : __ldg(tab + i0);
-                                    w1[e] = tab_smem ? tab[i1] : __ldg(tab + i1);
+                                    w0[e] = tab_smem ? s_tab[i0] : __ldg(gtab + i0);
+                                    w1[e] = tab_smem ? s_tab[i1] : __ldg(gtab + i1);
                                 }
 #pragma unroll
                                 for (int e = 0; e < 4; ++e) {
