@@ -66,8 +66,15 @@ static int run_linear(Path path, const void *x, int x_dt, const uint16_t *idx, c
 
     rc = BTC_ERR_UNSUPPORTED;
     if (path == PATH_GEMV || M <= 8) {
-        rc = launch_gemv_imma(&a, 1, s);
-        if (rc == BTC_ERR_UNSUPPORTED) rc = launch_gemv_decode(a, s);
+        // M <= 2: the integer-MMA kernel (3 digit columns per row of x fit one MMA); above that the fp16 bit-trick
+        // kernel is the faster one (its cost does not grow with M up to 8)
+        if (M <= 2) {
+            rc = launch_gemv_imma(&a, 1, s);
+            if (rc == BTC_ERR_UNSUPPORTED) rc = launch_gemv_decode(a, s);
+        } else {
+            rc = launch_gemv_decode(a, s);
+            if (rc == BTC_ERR_UNSUPPORTED) rc = launch_gemv_imma(&a, 1, s);
+        }
     }
     else rc = launch_gemm_tcgen05(a, s);
     if (rc == BTC_ERR_UNSUPPORTED) {

@@ -195,7 +195,7 @@ __device__ __forceinline__ void im_group_range(const ImProblem &P, int a0, int a
     hi = min(h, P.groups);
 }
 
-template <int NCLS, int NM>
+template <int NCLS, int NM, bool TAB_SMEM>
 __global__ void __launch_bounds__(IM_THREADS, 1)
 gemv_imma_kernel(const __grid_constant__ ImBatch batch)
 {
@@ -239,7 +239,7 @@ gemv_imma_kernel(const __grid_constant__ ImBatch batch)
     }
     __syncthreads();
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    const bool tab_smem = batch.tab_smem_bytes > 0;
+    constexpr bool tab_smem = TAB_SMEM;                  // codeword table staged in shared memory (else gathered from global)
     const int cost_a0 = batch.cost_per * (int)blockIdx.x + min((int)blockIdx.x, batch.cost_rem);
     const int cost_a1 = cost_a0 + batch.cost_per + ((int)blockIdx.x < batch.cost_rem ? 1 : 0);
 
@@ -417,6 +417,12 @@ gemv_imma_kernel(const __grid_constant__ ImBatch batch)
                     const int jb0 = j * IM_PW + ks * SLICE;         // first block of this warp's slice
                     const bool wvalid = ks * SLICE + BPL * t < pw;  // this lane's blocks exist (pw % 8 == 0)
                     const int kend = (j * IM_PW + pw) * v;          // end of the part in x
+                    // byte offset of this lane's index chunk inside a stage (128-byte swizzle: 16-byte chunk c of row q
+                    // sits at chunk c ^ (q & 7)); rows sg and sg + 8 of tile rh
+                    const int boff = (ks * SLICE + BPL * t) * 2;
+                    const int irow = rh * 16 + sg;
+                    const uint32_t idx_off = (uint32_t)(boff >> 7) * (ROWS * 128) + (uint32_t)irow * 128
+                                             + ((((boff >> 4) & 7) ^ (irow & 7)) << 4) + (boff & 15);
                     ImScale *scale_out = s_scale + ((size_t)(pc % IM_SLOTS) * IM_CWARPS + warp) * 8;
 
                     // ---- B fragments for this part.  The warp's slice of each row of x (16 blocks) is
@@ -540,10 +546,7 @@ gemv_imma_kernel(const __grid_constant__ ImBatch batch)
 #pragma unroll
                         for (int i = 0; i < BPL / 2; ++i) { ia[i] = 0u; ib[i] = 0u; }
                         if (wvalid) {
-                            const int boff = (ks * SLICE + BPL * t) * 2;            // byte offset in the part's row
-                            const int row = rh * 16 + sg;
-                            const unsigned char *pa = stage + (size_t)(boff >> 7) * (ROWS * 128) + (size_t)row * 128
-                                                      + ((((boff >> 4) & 7) ^ (row & 7)) << 4) + (boff & 15);
+                            const unsigned char *pa = stage + idx_off;
                             const unsigned char *pb = pa + 8 * 128;                 // row + 8: same row & 7
                             if (BPL == 8) {
                                 const uint4 qa = *reinterpret_cast<const uint4 *>(pa), qb = *reinterpret_cast<const uint4 *>(pb);
@@ -654,12 +657,12 @@ static int im_sm_count()
     return n;
 }
 
-template <int NCLS, int NM>
+template <int NCLS, int NM, bool TS>
 static int im_launch(ImBatch &b, int groups_total, cudaStream_t s)
 {
     constexpr int TRK = (NM == 1) ? 2 : 1;
     const ImSmem L = im_smem_layout(b.tab_smem_bytes, 8 * NM, TRK * 16, b.stages);
-    auto kern = gemv_imma_kernel<NCLS, NM>;
+    auto kern = gemv_imma_kernel<NCLS, NM, TS>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)L.total);
     if (e != cudaSuccess) return cuda_fail(e);
     cudaLaunchConfig_t cfg = {};
@@ -680,12 +683,12 @@ static int im_launch(ImBatch &b, int groups_total, cudaStream_t s)
     return e == cudaSuccess ? BTC_OK : cuda_fail(e);
 }
 
-template <int NCLS>
+template <int NCLS, bool TS>
 static int im_launch_nm(ImBatch &b, int nm, int groups_total, cudaStream_t s)
 {
-    if (nm == 1) return im_launch<NCLS, 1>(b, groups_total, s);
-    if (nm == 2) return im_launch<NCLS, 2>(b, groups_total, s);
-    return im_launch<NCLS, 3>(b, groups_total, s);
+    if (nm == 1) return im_launch<NCLS, 1, TS>(b, groups_total, s);
+    if (nm == 2) return im_launch<NCLS, 2, TS>(b, groups_total, s);
+    return im_launch<NCLS, 3, TS>(b, groups_total, s);
 }
 
 int launch_gemv_imma(const LinearArgs *problems, int count, cudaStream_t s)
@@ -739,8 +742,9 @@ int launch_gemv_imma(const LinearArgs *problems, int count, cudaStream_t s)
     if (im_smem_layout(tab_max, 8 * nm, rows, 2).total > 227u * 1024u) b.tab_smem_bytes = 0;   // gather from global (L1/L2)
     b.stages = IM_STAGES;
     while (b.stages > 2 && im_smem_layout(b.tab_smem_bytes, 8 * nm, rows, b.stages).total > 227u * 1024u) --b.stages;
-    if (ncls_max <= 4) return im_launch_nm<4>(b, nm, groups_total, s);
-    return im_launch_nm<5>(b, nm, groups_total, s);
+    const bool ts = b.tab_smem_bytes > 0;
+    if (ncls_max <= 4) return ts ? im_launch_nm<4, true>(b, nm, groups_total, s) : im_launch_nm<4, false>(b, nm, groups_total, s);
+    return ts ? im_launch_nm<5, true>(b, nm, groups_total, s) : im_launch_nm<5, false>(b, nm, groups_total, s);
 }
 
 int imma_status_read(int *out)
