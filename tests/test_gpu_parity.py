@@ -181,7 +181,7 @@ def test_gemm_deterministic_and_bounded():
 
 def test_gemv_batch_matches_oracle_and_single_calls():
     """Seven layers of mixed shape (the decode layer set scaled down, ragged N, one with mu, one bf16) in one
-    btc_linear_gemv_batch call: every output against the oracle, and bit-identical to the per-layer call."""
+    btc_linear_gemv_batch call: every output against the oracle, and (for M <= 2, where both run the same kernel) bit-identical to the per-layer call."""
     shapes = [(272, 1024, 16, 4096, False, "f16"), (272, 1024, 16, 4096, True, "f16"), (100, 1024, 16, 8192, False, "f16"),
               (1000, 1024, 16, 8192, False, "bf16"), (688, 2752, 16, 8192, False, "f16"), (37, 320, 20, 65536, False, "f16"),
               (513, 640, 20, 21619, True, "f16"), (64, 96, 12, 777, False, "f16"), (300, 2048, 16, 8192, False, "f16")]
@@ -197,5 +197,9 @@ def test_gemv_batch_matches_oracle_and_single_calls():
             rel, fwd = errors(y, oracle_y(L), L)
             assert rel <= TOL_GEMV and fwd <= TOL_GEMV, (L.spec, M, rel, fwd)
             single = btc.linear_gemv(d["x"], d["idx"], d["Cp"], d["alpha"], L.spec.v, L.spec.Kc, mu=d["mu"])
-            assert torch.equal(single, y), (L.spec, M)
+            if M <= 2:      # same kernel, same arithmetic: identical bits
+                assert torch.equal(single, y), (L.spec, M)
+            else:           # single calls with M > 2 take the fp16 bit-trick kernel
+                rel2, fwd2 = errors(single, oracle_y(L), L)
+                assert rel2 <= TOL_GEMV and fwd2 <= TOL_GEMV, (L.spec, M, rel2, fwd2)
     assert btc.device_status() == 0
