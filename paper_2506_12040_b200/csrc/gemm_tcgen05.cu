@@ -282,6 +282,200 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_x, const GemmParams
     if (warp == 2) tmem_dealloc(tmem_d, BM);
 }
 
+// ------------------------------------------------------------------------------------ v = 16 kernel
+// Same contraction, faster weight supply, for the common v = 16 (a 64-wide k step is four blocks):
+//   warp 0      TMA producer: x tiles, and index tiles (128 rows x 64 blocks = 16 k steps, 128-byte swizzle);
+//               bulk copy of the codeword table into shared memory
+//   warp 1      MMA issuer          warp 2   tensor-memory allocation
+//   warps 4-11  decode: thread (row r, half h) expands blocks 2h, 2h+1 of the k step: two table lookups in shared
+//               memory, and per pair of weights one shift and one LOP3 -- the table keeps the bit of weight t at
+//               (t & 1) * 16 + 4 + (t >> 1), so ((~w << (11 - j)) & 0x80008000) | {1.0, 1.0} is the pair
+//               (2j, 2j+1) as +-1 in bf16 / fp16; then the same warps run the epilogue, two per lane quadrant.
+constexpr int G2_THREADS = 384;
+constexpr int G2_DWARPS = 8;
+constexpr uint32_t G2_IDX_BYTES = 128 * 128;     // one index tile
+
+struct Gemm2Params {
+    LinearArgs a;
+    const float *sumx;
+    const uint32_t *tab;     // fp16-layout codeword words [Kc4]
+    int k_tiles;
+    int tab_bytes;           // > 0: table staged in shared memory
+};
+
+__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+
+template <int BM, int STAGES>
+__global__ void __launch_bounds__(G2_THREADS, 1)
+gemm_v16_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_i, const Gemm2Params p)
+{
+    constexpr uint32_t B_BYTES = BM * G_BK * 2;
+    constexpr uint32_t STAGE_BYTES = G_A_BYTES + B_BYTES;
+    extern __shared__ __align__(1024) unsigned char smem_raw[];
+    const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    unsigned char *smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
+    unsigned char *s_idx = smem_gen + (size_t)STAGES * STAGE_BYTES;                 // 2 index tiles
+    uint32_t *s_tab = reinterpret_cast<uint32_t *>(s_idx + 2 * G2_IDX_BYTES);
+    uint64_t *bars = reinterpret_cast<uint64_t *>(reinterpret_cast<unsigned char *>(s_tab) + ((p.tab_bytes + 15) & ~15));
+    // bars: [0,S) full_x, [S,2S) full_w, [2S,3S) empty, 3S accum, 3S+1.. full_i[2], empty_i[2], tab_full
+    uint32_t *s_tmem = reinterpret_cast<uint32_t *>(bars + 3 * STAGES + 6);
+    volatile int *s_abort = reinterpret_cast<volatile int *>(s_tmem + 1);
+
+    const LinearArgs &a = p.a;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int n0 = blockIdx.x * G_BN, m0 = blockIdx.y * BM;
+    const int KT = p.k_tiles;
+    const bool is_bf16 = (a.x_dt == BTC_BF16);
+    auto bar_full_x = [&](int s) { return smem_u32(bars + s); };
+    auto bar_full_w = [&](int s) { return smem_u32(bars + STAGES + s); };
+    auto bar_empty = [&](int s) { return smem_u32(bars + 2 * STAGES + s); };
+    const uint32_t bar_accum = smem_u32(bars + 3 * STAGES);
+    auto bar_full_i = [&](int b) { return smem_u32(bars + 3 * STAGES + 1 + b); };
+    auto bar_empty_i = [&](int b) { return smem_u32(bars + 3 * STAGES + 3 + b); };
+    const uint32_t bar_tab = smem_u32(bars + 3 * STAGES + 5);
+
+    if (tid == 0) {
+        for (int s = 0; s < STAGES; ++s) {
+            mbar_init(bar_full_x(s), 1);
+            mbar_init(bar_full_w(s), G2_DWARPS);
+            mbar_init(bar_empty(s), 1);
+        }
+        mbar_init(bar_accum, 1);
+        for (int b = 0; b < 2; ++b) { mbar_init(bar_full_i(b), 1); mbar_init(bar_empty_i(b), G2_DWARPS); }
+        mbar_init(bar_tab, 1);
+        *s_abort = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 2) tmem_alloc(smem_u32(s_tmem), BM);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_d = *s_tmem;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            if (p.tab_bytes > 0) {
+                mbar_expect_tx(bar_tab, (uint32_t)p.tab_bytes);
+                bulk_g2s(smem_u32(s_tab), p.tab, (uint32_t)p.tab_bytes, bar_tab);
+            }
+            for (int kt = 0; kt < KT; ++kt) {
+                if ((kt & 15) == 0) {
+                    const int it = kt >> 4, ib = it & 1;
+                    if (it >= 2 && !mbar_wait(bar_empty_i(ib), ((it >> 1) & 1) ^ 1, s_abort)) break;
+                    mbar_expect_tx(bar_full_i(ib), G2_IDX_BYTES);
+                    tma_load_2d(smem_u32(s_idx + (size_t)ib * G2_IDX_BYTES), &tmap_i, it * 64, n0, bar_full_i(ib));
+                }
+                const int s = kt % STAGES;
+                const uint32_t ph = (kt / STAGES) & 1;
+                if (kt >= STAGES && !mbar_wait(bar_empty(s), ph ^ 1, s_abort)) break;
+                mbar_expect_tx(bar_full_x(s), B_BYTES);
+                tma_load_2d(smem_base + s * STAGE_BYTES + G_A_BYTES, &tmap_x, kt * G_BK, m0, bar_full_x(s));
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            uint32_t idesc = (1u << 4) | ((uint32_t)(BM >> 3) << 17) | ((uint32_t)(G_BN >> 4) << 24);
+            if (is_bf16) idesc |= (1u << 7) | (1u << 10);
+            for (int kt = 0; kt < KT; ++kt) {
+                const int s = kt % STAGES;
+                const uint32_t ph = (kt / STAGES) & 1;
+                if (!mbar_wait(bar_full_x(s), ph, s_abort)) break;
+                if (!mbar_wait(bar_full_w(s), ph, s_abort)) break;
+                tc_fence_after();
+                const uint32_t a_addr = smem_base + s * STAGE_BYTES;
+                const uint64_t adesc = make_smem_desc(a_addr);
+                const uint64_t bdesc = make_smem_desc(a_addr + G_A_BYTES);
+#pragma unroll
+                for (int k = 0; k < G_BK / 16; ++k)
+                    umma_f16(tmem_d, adesc + 2 * k, bdesc + 2 * k, idesc, (kt | k) ? 1u : 0u);
+                umma_commit(bar_empty(s));
+            }
+            umma_commit(bar_accum);
+        }
+    } else if (warp >= 4) {
+        const int d = tid - 128;                       // 0 .. 255
+        const int r = d & 127, h = d >> 7;             // weight row of the tile, half of the k step
+        const uint32_t one2 = is_bf16 ? 0x3F803F80u : 0x3C003C00u;
+        const bool tab_smem = p.tab_bytes > 0;
+        if (tab_smem && !mbar_wait(bar_tab, 0, s_abort)) { /* fall through: waits below bail out */ }
+        bool ok = true;
+        for (int kt = 0; kt < KT && ok; ++kt) {
+            const int it = kt >> 4, ib = it & 1;
+            if ((kt & 15) == 0 && !mbar_wait(bar_full_i(ib), (it >> 1) & 1, s_abort)) { ok = false; break; }
+            // index pair of blocks 2h, 2h+1 of this k step: column (kt % 16) * 4 + 2h of the index tile
+            const int boff = (kt & 15) * 8 + 4 * h;
+            const uint32_t pair = *reinterpret_cast<const uint32_t *>(
+                s_idx + (size_t)ib * G2_IDX_BYTES + (size_t)r * 128 + ((((boff >> 4) & 7) ^ (r & 7)) << 4) + (boff & 15));
+            const uint32_t i0 = pair & 0xffffu, i1 = pair >> 16;
+            const uint32_t w0 = ~(tab_smem ? s_tab[i0] : __ldg(p.tab + i0));
+            const uint32_t w1 = ~(tab_smem ? s_tab[i1] : __ldg(p.tab + i1));
+            if ((kt & 15) == 15 || kt == KT - 1) {
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_empty_i(ib));
+            }
+            const int s = kt % STAGES;
+            const uint32_t ph = (kt / STAGES) & 1;
+            if (kt >= STAGES && !mbar_wait(bar_empty(s), ph ^ 1, s_abort)) { ok = false; break; }
+            unsigned char *arow = smem_gen + (size_t)s * STAGE_BYTES + (size_t)r * 128;
+#pragma unroll
+            for (int b = 0; b < 2; ++b) {
+                const uint32_t w = b ? w1 : w0;
+#pragma unroll
+                for (int c = 0; c < 2; ++c) {
+                    uint4 q;
+                    q.x = ((w << (11 - (4 * c + 0))) & 0x80008000u) | one2;
+                    q.y = ((w << (11 - (4 * c + 1))) & 0x80008000u) | one2;
+                    q.z = ((w << (11 - (4 * c + 2))) & 0x80008000u) | one2;
+                    q.w = ((w << (11 - (4 * c + 3))) & 0x80008000u) | one2;
+                    const int chunk = (2 * h + b) * 2 + c;
+                    *reinterpret_cast<uint4 *>(arow + ((chunk ^ (r & 7)) << 4)) = q;
+                }
+            }
+            fence_proxy_async_smem();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_full_w(s));
+        }
+        // ------------------------------------------------------------ epilogue: two warps per lane quadrant
+        if (ok && mbar_wait(bar_accum, 0, s_abort)) {
+            tc_fence_after();
+            const int wl = warp - 4;
+            const int q4 = wl & 3, half = wl >> 2;
+            const int nrow = n0 + q4 * 32 + lane;
+            const int nc = min(nrow, a.N - 1);
+            const float al = __half2float(a.alpha[nc]);
+            const float mu = a.mu ? __half2float(a.mu[nc]) : 0.f;
+            const uint32_t lane_base = (uint32_t)(q4 * 32) << 16;
+#pragma unroll 1
+            for (int c0 = half * (BM / 2); c0 < (half + 1) * (BM / 2); c0 += 32) {
+                uint32_t rr[32];
+                tmem_ld32(tmem_d + lane_base + c0, rr);
+                tmem_ld_wait();
+                if (nrow < a.N) {
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) {
+                        const int m = m0 + c0 + i;
+                        if (m < a.M) {
+                            float y = al * __uint_as_float(rr[i]);
+                            if (a.mu) y += mu * p.sumx[m];
+                            store_from_float(a.y, a.y_dt, (size_t)m * a.N + nrow, y);
+                        }
+                    }
+                }
+            }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (*s_abort) {
+        for (int i = 0; i < 200; ++i) __nanosleep(1000);
+        __syncthreads();
+    }
+    if (warp == 2) tmem_dealloc(tmem_d, BM);
+}
+
 // ------------------------------------------------------------------------------------ host side
 typedef CUresult (*encode_tiled_fn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
                                     const cuuint64_t *, const cuuint32_t *, const cuuint32_t *,
@@ -310,6 +504,19 @@ static int launch_cfg(const CUtensorMap &tm, const GemmParams &p, cudaStream_t s
     if (e != cudaSuccess) return cuda_fail(e);
     dim3 grid((p.a.N + G_BN - 1) / G_BN, (p.a.M + BM - 1) / BM);
     kern<<<grid, G_THREADS, smem, s>>>(tm, p);
+    return cuda_check_launch();
+}
+
+template <int BM, int STAGES>
+static int launch_v16(const CUtensorMap &tm, const CUtensorMap &ti, const Gemm2Params &p, cudaStream_t s)
+{
+    const size_t smem = (size_t)STAGES * (G_A_BYTES + BM * G_BK * 2) + 1024 + 2 * G2_IDX_BYTES + ((p.tab_bytes + 15) & ~15) +
+                        (3 * STAGES + 6) * 8 + 16;
+    auto kern = gemm_v16_kernel<BM, STAGES>;
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return cuda_fail(e);
+    dim3 grid((p.a.N + G_BN - 1) / G_BN, (p.a.M + BM - 1) / BM);
+    kern<<<grid, G2_THREADS, smem, s>>>(tm, ti, p);
     return cuda_check_launch();
 }
 
@@ -347,6 +554,27 @@ int launch_gemm_tcgen05(const LinearArgs &a, cudaStream_t s)
         int rc = cuda_check_launch();
         if (rc != BTC_OK) return rc;
         p.sumx = sx;
+    }
+    if (a.v == 16 && a.Kb % 8 == 0) {
+        // v = 16 kernel: index tiles by TMA, table in shared memory when it fits
+        CUtensorMap ti;
+        const cuuint64_t idims[2] = {(cuuint64_t)a.Kb, (cuuint64_t)a.N};
+        const cuuint64_t istr[1] = {(cuuint64_t)a.Kb * 2};
+        const cuuint32_t ibox[2] = {64, 128};
+        if (enc(&ti, CU_TENSOR_MAP_DATA_TYPE_UINT16, 2, const_cast<uint16_t *>(a.idx), idims, istr, ibox, estr,
+                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS) {
+            Gemm2Params q;
+            q.a = a; q.sumx = p.sumx; q.k_tiles = p.k_tiles;
+            const int Kc4 = (a.Kc + 3) / 4 * 4;
+            q.tab = a.Cp + Kc4;
+            // the table is staged in shared memory when it fits beside the pipeline stages (227 KB per CTA)
+            const size_t fixed = (BM == 256 ? 3 * (G_A_BYTES + 256 * G_BK * 2) : 4 * (G_A_BYTES + 128 * G_BK * 2)) + 1024 +
+                                 2 * G2_IDX_BYTES + 256;
+            q.tab_bytes = (fixed + (size_t)Kc4 * 4 <= 227u * 1024u) ? Kc4 * 4 : 0;
+            if (BM == 256) return launch_v16<256, 3>(tm, ti, q, s);
+            return launch_v16<128, 4>(tm, ti, q, s);
+        }
     }
     if (BM == 256) return launch_cfg<256, 4>(tm, p, s);
     return launch_cfg<128, 6>(tm, p, s);
