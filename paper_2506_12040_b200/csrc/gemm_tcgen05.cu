@@ -287,12 +287,13 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_x, const GemmParams
 //   warp 0      TMA producer: x tiles, and index tiles (128 rows x 64 blocks = 16 k steps, 128-byte swizzle);
 //               bulk copy of the codeword table into shared memory
 //   warp 1      MMA issuer          warp 2   tensor-memory allocation
-//   warps 4-11  decode: thread (row r, half h) expands blocks 2h, 2h+1 of the k step: two table lookups in shared
+//   warps 4-19  decode, in two groups of eight that take the even and the odd k steps (more lookups in flight):
+//               thread (row r, half h) expands blocks 2h, 2h+1 of the k step: two table lookups in shared
 //               memory, and per pair of weights one shift and one LOP3 -- the table keeps the bit of weight t at
 //               (t & 1) * 16 + 4 + (t >> 1), so ((~w << (11 - j)) & 0x80008000) | {1.0, 1.0} is the pair
-//               (2j, 2j+1) as +-1 in bf16 / fp16; then the same warps run the epilogue, two per lane quadrant.
-constexpr int G2_THREADS = 384;
-constexpr int G2_DWARPS = 8;
+//               (2j, 2j+1) as +-1 in bf16 / fp16; then the same warps run the epilogue, four per lane quadrant.
+constexpr int G2_DWARPS = 16;                    // two groups of 8: even and odd k steps
+constexpr int G2_THREADS = 128 + G2_DWARPS * 32;
 constexpr uint32_t G2_IDX_BYTES = 128 * 128;     // one index tile
 
 struct Gemm2Params {
@@ -340,7 +341,7 @@ gemm_v16_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
     if (tid == 0) {
         for (int s = 0; s < STAGES; ++s) {
             mbar_init(bar_full_x(s), 1);
-            mbar_init(bar_full_w(s), G2_DWARPS);
+            mbar_init(bar_full_w(s), G2_DWARPS / 2);
             mbar_init(bar_empty(s), 1);
         }
         mbar_init(bar_accum, 1);
@@ -396,15 +397,20 @@ gemm_v16_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
             umma_commit(bar_accum);
         }
     } else if (warp >= 4) {
-        const int d = tid - 128;                       // 0 .. 255
+        const int d = (tid - 128) & 255;               // position in the group
+        const int grp = (tid - 128) >> 8;              // 0: even k steps, 1: odd k steps
         const int r = d & 127, h = d >> 7;             // weight row of the tile, half of the k step
         const uint32_t one2 = is_bf16 ? 0x3F803F80u : 0x3C003C00u;
         const bool tab_smem = p.tab_bytes > 0;
         if (tab_smem && !mbar_wait(bar_tab, 0, s_abort)) { /* fall through: waits below bail out */ }
         bool ok = true;
-        for (int kt = 0; kt < KT && ok; ++kt) {
+        int cur_it = -1;
+        for (int kt = grp; kt < KT && ok; kt += 2) {
             const int it = kt >> 4, ib = it & 1;
-            if ((kt & 15) == 0 && !mbar_wait(bar_full_i(ib), (it >> 1) & 1, s_abort)) { ok = false; break; }
+            if (it != cur_it) {
+                if (!mbar_wait(bar_full_i(ib), (it >> 1) & 1, s_abort)) { ok = false; break; }
+                cur_it = it;
+            }
             // index pair of blocks 2h, 2h+1 of this k step: column (kt % 16) * 4 + 2h of the index tile
             const int boff = (kt & 15) * 8 + 4 * h;
             const uint32_t pair = *reinterpret_cast<const uint32_t *>(
@@ -412,7 +418,7 @@ gemm_v16_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
             const uint32_t i0 = pair & 0xffffu, i1 = pair >> 16;
             const uint32_t w0 = ~(tab_smem ? s_tab[i0] : __ldg(p.tab + i0));
             const uint32_t w1 = ~(tab_smem ? s_tab[i1] : __ldg(p.tab + i1));
-            if ((kt & 15) == 15 || kt == KT - 1) {
+            if (((kt + 2) >> 4) != it || kt + 2 >= KT) {           // this group's last k step in the index tile
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar_empty_i(ib));
             }
@@ -438,18 +444,18 @@ gemm_v16_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_full_w(s));
         }
-        // ------------------------------------------------------------ epilogue: two warps per lane quadrant
+        // ------------------------------------------------------------ epilogue: four warps per lane quadrant
         if (ok && mbar_wait(bar_accum, 0, s_abort)) {
             tc_fence_after();
             const int wl = warp - 4;
-            const int q4 = wl & 3, half = wl >> 2;
+            const int q4 = wl & 3, quarter = wl >> 2;
             const int nrow = n0 + q4 * 32 + lane;
             const int nc = min(nrow, a.N - 1);
             const float al = __half2float(a.alpha[nc]);
             const float mu = a.mu ? __half2float(a.mu[nc]) : 0.f;
             const uint32_t lane_base = (uint32_t)(q4 * 32) << 16;
 #pragma unroll 1
-            for (int c0 = half * (BM / 2); c0 < (half + 1) * (BM / 2); c0 += 32) {
+            for (int c0 = quarter * (BM / 4); c0 < (quarter + 1) * (BM / 4); c0 += 32) {
                 uint32_t rr[32];
                 tmem_ld32(tmem_d + lane_base + c0, rr);
                 tmem_ld_wait();
