@@ -140,6 +140,21 @@ def run_reference(args):
 
 
 # ----------------------------------------------------------------------------------------------
+def max_over_ranks(seconds: float, dist, device) -> float:
+    """Slowest rank's time (the ranks are independent replicas: no data-path collective, only this reduction)."""
+    if dist is None:
+        return seconds
+    import torch
+    tt = torch.tensor([seconds], device=device, dtype=torch.float64)
+    dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+    return float(tt.item())
+
+
+def whole_job_gbs(world: int, bytes_per_step: int, seconds_all_steps: float, steps: int) -> float:
+    """Aggregate effective GB/s of `world` replicas that each moved bytes_per_step per step."""
+    return world * bytes_per_step / (seconds_all_steps / steps) * 1e-9
+
+
 def run_gpu(args):
     import torch
     import paper_2506_12040_b200 as btc
@@ -228,13 +243,9 @@ def run_gpu(args):
             step1(0)
         torch.cuda.synchronize()
     clocks = clk.summary()
-    t_max = t_total
-    if dist is not None:
-        tt = torch.tensor([t_total], device=dev, dtype=torch.float64)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        t_max = float(tt.item())
+    t_max = max_over_ranks(t_total, dist, dev)
     ms_per_step = t_max / args.steps * 1e3
-    value = world * bytes_step / (t_max / args.steps) * 1e-9
+    value = whole_job_gbs(world, bytes_step, t_max, args.steps)
     launches = args.steps                       # one fused launch per step
     avg_launch_s = t_total / launches
     bytes_per_launch = bytes_step
@@ -355,11 +366,8 @@ def run_gpu(args):
             e1.record(stream)
             stream.synchronize()
         te = e0.elapsed_time(e1) * 1e-3 / n_e2e
-        if dist is not None:
-            tt = torch.tensor([te], device=dev, dtype=torch.float64)
-            dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-            te = float(tt.item())
-        e2e = {"value": world * bytes_step / te * 1e-9, "unit": UNIT,
+        te = max_over_ranks(te, dist, dev)
+        e2e = {"value": whole_job_gbs(world, bytes_step, te, 1), "unit": UNIT,
                "h2d_bytes_per_step": int(sum(x.numel() * 2 for x in xs1)),
                "d2h_bytes_per_step": int(sum(4 * s.N for s in specs)),
                "note": "x from pinned host memory and y back to host every layer; weights resident on the device"}
