@@ -1,7 +1,8 @@
 // Decode path for small M (1..8): streams the index matrices of up to IM_MAXP independent layers
 // once and evaluates every block dot
 //     <x_j, C[idx]> = 2 * sum_{bit=1} x  -  sum x            (identity for +-1 codewords)
-// (block-dot sum of the paper's appendix "Binary codebook LUT-GEMM") with EXACT integer accumulation.
+// (block-dot sum of the paper's appendix "Binary codebook LUT-GEMM") with exact integer accumulation
+// inside every K-slice.
 //
 // Why integers.  One output needs K sign applications.  At the HBM rate an SM receives 180 weights per
 // clock (v = 16), while its plain ALUs issue 64 integer lane-operations per clock and the warp-level
@@ -12,24 +13,27 @@
 //       of byte (t & 3), so `word & (0x01010101 << c)` IS the four bytes {0 or 2^c} of weights
 //       4c .. 4c+3: one LOP3 expands four weights.
 //   B (32 k x 8 cols, s8)  = the activations as three balanced base-256 digits of a block-fixed-point
-//       integer: X = rint(x * 2^s), |X| <= 2^(22 - cmax), with s chosen per row of x from its largest
-//       magnitude, pre-shifted by (cmax - c) so that every product is bit * X * 2^cmax; digit d of
-//       row m sits in column 3 m + d.
-//   D (16 x 8, s32)        = exact partial sums; the digits are recombined once per output.
-// The result is the exact +-1 dot product of the quantised activations; the only roundings are the
-// quantisation of x (2^-20 of the row's largest magnitude for v = 16) and one rounding per output
-// when alpha is applied.
+//       integer: X = rint(x * 2^s), |X| <= 2^(22 - cmax), with s chosen per K-slice (256 or 512
+//       activations of one row of x) from its largest magnitude, pre-shifted by (cmax - c) so that
+//       every product is bit * X * 2^cmax; digit d of row m sits in column 3 m + d.
+//   D (16 x 8, s32)        = exact partial sums.
+// The three digit sums of a (slice, output) are recombined in fp32 (each is below 2^24, so the
+// conversions are exact), scaled by 2^-s and added over the slices; then alpha (and mu) are applied.
+// Roundings: the quantisation of x (2^-20 of the slice's largest magnitude for v = 16) and a handful
+// of fp32 operations per output.
 //
 // Work split: persistent CTAs.  A "row group" is 32 rows (16 when M > 2) of one layer; a CTA owns a
 // contiguous, cost-weighted range of row groups over all layers of the launch.  Layers wider than
 // 256 blocks are cut into K-parts of 256 blocks; a CTA walks up to IM_RC of its row groups part by
 // part, so the activation fragments change only once per part, and the epilogue adds the parts.
-//   warps 0..15  compute: warp w owns blocks 16 w .. 16 w + 15 of the part; lane (g = lane / 4,
-//                t = lane % 4) supplies rows g and g + 8 of each tile and the blocks 16 w + 4 t + e;
-//                its activations stay in registers as MMA B fragments.
-//   warp 16      producer: cp.async.bulk of index tiles into a shared ring, and of the codeword table.
-//   warps 17,18  epilogue: add the 16 partial tiles in a fixed order, add the K-parts, recombine
-//                digits, apply alpha (and mu), store y.
+//   warps 0..15  compute: warp w owns K-slice w % KS of the part and tile w / KS of the row group
+//                (KS = 8 slices of 32 blocks, 2 tiles when M <= 2; 16 slices of 16 blocks, 1 tile
+//                otherwise); lane (g = lane / 4, t = lane % 4) supplies two rows of the tile and
+//                BPL consecutive blocks; its activations stay in registers as MMA B fragments.
+//   warp 16      producer: TMA boxes (64 blocks x rows, 128-byte swizzle) of the index matrix into
+//                a shared ring, bulk copy of the codeword table.
+//   warps 17,18  epilogue: recombine the digits of the K-slices' partial tiles in a fixed order, add
+//                the K-parts, apply alpha (and mu), store y.
 // Every mbarrier wait is bounded; when one runs out the CTA raises a status word and drains.
 #include <cuda.h>
 #include "btc_internal.cuh"
@@ -73,7 +77,6 @@ struct ImBatch {
     int stages;               // index stages in the ring (2 .. IM_STAGES)
 };
 
-// ------------------------------------------------------------------------------------ PTX helpers
 // ------------------------------------------------------------------------------------ PTX helpers
 __device__ __forceinline__ uint32_t im_smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
 __device__ __forceinline__ void im_mbar_init(uint32_t bar, uint32_t count) {
