@@ -319,12 +319,15 @@ gemv_imma_kernel(const __grid_constant__ ImBatch batch)
                         const int buf = li & 1;
                         const int n = r * ROWS + R;
                         const bool live = (n < P.N) && (grp == 0);
-                        float al = 0.f, mu = 0.f;
+                        // alpha / mu of this row: the loads are issued here and first used after the wait below, so their
+                        // latency (a trip to DRAM) hides behind it
+                        unsigned short al_bits = 0, mu_bits = 0;
                         if (last && live) {
-                            al = __half2float(P.alpha[n]);
-                            if (P.mu) mu = __half2float(P.mu[n]);
+                            al_bits = __ldg(reinterpret_cast<const unsigned short *>(P.alpha) + n);
+                            if (P.mu) mu_bits = __ldg(reinterpret_cast<const unsigned short *>(P.mu) + n);
                         }
                         if (!im_mbar_wait(bar_pfull(buf), (li >> 1) & 1, s_abort)) { ok = false; break; }
+                        const float al = __half2float(__ushort_as_half(al_bits)), mu = __half2float(__ushort_as_half(mu_bits));
                         if (r == c0) {
 #pragma unroll
                             for (int m = 0; m < MAXM; ++m)
