@@ -35,6 +35,9 @@ import workloads as wl  # noqa: E402
 METRIC = "effective HBM GB/s at M=1 (us/layer and TFLOP/s at M=2048 in details)"
 UNIT = "GB/s"
 CONFIG_ID = 2
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the fused step kernel, from the ncu capture summarised in
+# profiles/decode_imma_config2_M1_step.md (set to None whenever that kernel changes until it is captured again)
+TRAFFIC_BYTES_PER_LAUNCH = 25721856
 
 
 def measured_peaks():
@@ -401,7 +404,7 @@ def run_gpu(args):
                            "multi_gpu": "replicas only"},
                 "clocks": clocks, "e2e": e2e, "gpu_launches": launches,
                 "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
-                             "frac": achieved / peak, "traffic": None, "peak_source": f"of {peaks['source']}",
+                             "frac": achieved / peak, "traffic": TRAFFIC_BYTES_PER_LAUNCH, "peak_source": f"of {peaks['source']}",
                              "kernel": "gemv_imma_kernel (7 layers per launch)", "bytes_per_launch": bytes_per_launch,
                              "avg_launch_us": avg_launch_s * 1e6},
                 "cpu_baseline": cpu, "details": details}
