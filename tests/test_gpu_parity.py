@@ -203,3 +203,32 @@ def test_gemv_batch_matches_oracle_and_single_calls():
                 rel2, fwd2 = errors(single, oracle_y(L), L)
                 assert rel2 <= TOL_GEMV and fwd2 <= TOL_GEMV, (L.spec, M, rel2, fwd2)
     assert btc.device_status() == 0
+
+
+# ------------------------------------------------------------------ online activation transform
+
+@pytest.mark.parametrize("path,M,k1,k2", [("gemv", 2, 32, 32), ("gemv", 1, 64, 64), ("gemm", 96, 16, 64), ("gemv", 8, 8, 40)])
+def test_online_transform_prologue(path, M, k1, k2):
+    """x' = x * diag(sigma) * (P1 kron P2) before the layer (Section 4.2, applied on the fly): against the oracle's dense
+    K x K Kronecker form in fp64.  The kernel rounds x' to the activation dtype, hence the tensor-core tolerance."""
+    K = k1 * k2
+    v = 16 if K % 16 == 0 else 20
+    L = wl.make_layer(_spec(272, K, v, 4096, x_dtype="f16" if path == "gemv" else "bf16"), M, seed=77 + k1)
+    rng = np.random.default_rng(5 + k1)
+    sigma = rng.choice(np.array([-1, 1], dtype=np.int8), size=K)
+    P1 = np.linalg.qr(rng.standard_normal((k1, k1)))[0].astype(np.float32)
+    P2 = np.linalg.qr(rng.standard_normal((k2, k2)))[0].astype(np.float32)
+    bits = np.zeros((K + 31) // 32, dtype=np.uint32)
+    for i in np.nonzero(sigma < 0)[0]:
+        bits[i >> 5] |= np.uint32(1) << np.uint32(i & 31)
+    d = to_device(L)
+    tr = (torch.from_numpy(bits.view(np.int32)).cuda(), torch.from_numpy(P1).cuda(), torch.from_numpy(P2).cuda())
+    fn = btc.linear_gemv if path == "gemv" else btc.linear_gemm
+    y = fn(d["x"], d["idx"], d["Cp"], d["alpha"], v, 4096, transform=tr)
+    torch.cuda.synchronize()
+    xt = oracle.transform(L.x_f64(), sigma, P1.astype(np.float64), P2.astype(np.float64))
+    ref = oracle.linear(xt, L.idx, L.C_pm1, L.alpha)
+    err = np.abs(y.double().cpu().numpy() - ref)
+    assert err.max() / np.abs(ref).max() <= TOL_GEMM
+    scale = np.outer(np.abs(xt).sum(1), np.abs(L.alpha.astype(np.float64)))
+    assert (err / np.maximum(scale, 1e-300)).max() <= TOL_GEMM
