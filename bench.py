@@ -337,6 +337,92 @@ def run_gpu(args):
                 res["frac_bf16_peak_measured"] = res["btc"]["TFLOPs"] / peaks["bf16_tflops"]
                 gem[f"M{M}_{s.N}x{s.K}"] = res
         details["gemm"] = gem
+
+        # ---- configs 1 and 3: single layers at M = 1 (config 3: v = 20, 65536 centroids gathered from L1/L2, Zipf indices)
+        def time_single(spec, seed, lid, M, copies=24, reps=96):
+            L = wl.make_layer(spec, M, seed, lid)
+            d = dev_layer(L)
+            idxs = [d["idx"]] + [torch.roll(d["idx"], shifts=17 * c + 1, dims=0) for c in range(1, copies)]   # distinct memory
+            x = d["x"][:M].contiguous()
+            outs = [torch.empty((M, spec.N), dtype=torch.float32, device=dev) for _ in range(copies)]
+
+            def one(k):
+                btc.linear_gemv(x, idxs[k % copies], d["Cp"], d["alpha"], spec.v, spec.Kc, out=outs[k % copies])
+            stream = torch.cuda.Stream(device=dev)
+            with torch.cuda.stream(stream):
+                for k in range(4):
+                    one(k)
+                stream.synchronize()
+                g = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(g, stream=stream):
+                    for k in range(reps):
+                        one(k)
+                g.replay()
+                stream.synchronize()
+                e0 = torch.cuda.Event(enable_timing=True)
+                e1 = torch.cuda.Event(enable_timing=True)
+                e0.record(stream)
+                g.replay()
+                e1.record(stream)
+                stream.synchronize()
+            us = e0.elapsed_time(e1) * 1e3 / reps
+            b = algorithmic_bytes(spec, M)
+            return {"us": us, "GBps": b / us * 1e-3, "frac_measured": b / us * 1e-3 / peaks["hbm_gbs"]}
+        c1 = wl.CONFIGS[1]
+        details["config1_M1"] = time_single(c1["layers"][0], c1["seed"], 0, 1, copies=64, reps=128)
+        c3 = wl.CONFIGS[3]
+        details["config3"] = {f"{c3['layers'][li].N}x{c3['layers'][li].K}_M{M}": time_single(c3["layers"][li], c3["seed"], li, M)
+                              for li in (0, 4) for M in c3["M"]}
+
+        # ---- config 5: 32 blocks x 7 projections chained at M = 1 (fp16 activations between layers; q,k,v and gate,up
+        #      are fused launches): 4 launches per block, 128 per token.  Indices of block b are the seeded layer set
+        #      rolled by b rows (distinct memory, same distribution), so every block streams from HBM.
+        def time_chain(Kc, dist_name):
+            cfg5 = wl.config_layers(5, Kc=Kc, idx_dist=dist_name)
+            sp = cfg5["layers"]
+            base5 = [dev_layer(wl.make_layer(s5, 1, cfg5["seed"], i)) for i, s5 in enumerate(sp)]
+            nb = cfg5["n_blocks"]
+            h = [torch.empty((1, 4096), dtype=torch.float16, device=dev) for _ in range(2)]
+            h[0].copy_(base5[0]["x"][:1])
+            qkv = [torch.empty((1, 4096), dtype=torch.float16, device=dev) for _ in range(3)]
+            o_out = torch.empty((1, 4096), dtype=torch.float16, device=dev)
+            gu = [torch.empty((1, 11008), dtype=torch.float16, device=dev) for _ in range(2)]
+            launches = []
+            for b in range(nb):
+                lay = [dict(idx=(base5[i]["idx"] if b == 0 else torch.roll(base5[i]["idx"], shifts=b, dims=0)), C_packed=base5[i]["Cp"],
+                            alpha=base5[i]["alpha"], v=sp[i].v, Kc=sp[i].Kc) for i in range(7)]
+                xin, xout = h[b & 1], h[(b + 1) & 1]
+                launches.append(btc.GemvBatch([dict(x=xin, out=qkv[i], **lay[i]) for i in range(3)]))
+                launches.append(btc.GemvBatch([dict(x=qkv[0], out=o_out, **lay[3])]))
+                launches.append(btc.GemvBatch([dict(x=o_out, out=gu[i - 4], **lay[i]) for i in (4, 5)]))
+                launches.append(btc.GemvBatch([dict(x=gu[0], out=xout, **lay[6])]))
+            stream = torch.cuda.Stream(device=dev)
+            with torch.cuda.stream(stream):
+                for L5 in launches:
+                    L5.run()
+                stream.synchronize()
+                g = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(g, stream=stream):
+                    for L5 in launches:
+                        L5.run()
+                g.replay()
+                stream.synchronize()
+                ts = []
+                for _ in range(5):
+                    e0 = torch.cuda.Event(enable_timing=True)
+                    e1 = torch.cuda.Event(enable_timing=True)
+                    e0.record(stream)
+                    g.replay()
+                    e1.record(stream)
+                    stream.synchronize()
+                    ts.append(e0.elapsed_time(e1) * 1e-3)
+            t = float(np.median(ts))
+            finite = bool(torch.isfinite(h[nb & 1].float()).all())
+            nbytes = nb * sum(algorithmic_bytes(s5, 1) for s5 in sp)
+            return {"tokens_per_s": 1.0 / t, "us_per_token": t * 1e6, "GBps": nbytes / t * 1e-9,
+                    "frac_measured": nbytes / t * 1e-9 / peaks["hbm_gbs"], "launches": len(launches), "finite": finite}
+        details["config5_chain"] = {f"Kc{Kc}_{dn}": time_chain(Kc, dn)
+                                    for (Kc, dn) in ((4096, "uniform"), (256, "uniform"), (65536, "uniform"), (4096, "zipf"))}
         details["device_status"] = btc.device_status()
 
     # ---- end to end: host buffers in, host buffers out, through the same calls
