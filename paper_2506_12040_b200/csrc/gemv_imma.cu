@@ -41,7 +41,7 @@
 namespace btc {
 
 constexpr int IM_CWARPS = 16;                   // compute warps
-constexpr int IM_EWARPS = 2;                    // epilogue warps
+constexpr int IM_EWARPS = 2;                    // epilogue warps (four would cap the kernel at 80 registers: spills)
 constexpr int IM_THREADS = (IM_CWARPS + 1 + IM_EWARPS) * 32;
 constexpr int IM_STAGES = 8;                     // most index stages a launch may use (fewer when shared memory is short)
 constexpr int IM_BOX_COLS = 64;                 // blocks per TMA box row: 128 bytes, the swizzle span
@@ -63,7 +63,8 @@ struct ImProblem {
     int parts;                // ceil(Kb / IM_PW)
     int groups;               // row groups: ceil(N / (16 * TRK))
     int ncls;                 // v / 4
-    int cost_base;            // sum over earlier layers of groups * Kb
+    int cost;                 // cost of one row group (blocks, plus the per-part fragment rebuild; see launch_gemv_imma)
+    int cost_base;            // sum over earlier layers of groups * cost
 };
 
 struct ImBatch {
@@ -191,9 +192,9 @@ __host__ __device__ inline ImSmem im_smem_layout(int tab_bytes, int cols, int ro
 __device__ __forceinline__ void im_group_range(const ImProblem &P, int a0, int a1, int &lo, int &hi)
 {
     lo = hi = 0;
-    if (a1 <= P.cost_base || a0 >= P.cost_base + P.groups * P.Kb) return;     // (no division for layers of other CTAs)
-    const int l = (a0 <= P.cost_base) ? 0 : (a0 - P.cost_base + P.Kb - 1) / P.Kb;
-    const int h = (a1 - P.cost_base + P.Kb - 1) / P.Kb;
+    if (a1 <= P.cost_base || a0 >= P.cost_base + P.groups * P.cost) return;     // (no division for layers of other CTAs)
+    const int l = (a0 <= P.cost_base) ? 0 : (a0 - P.cost_base + P.cost - 1) / P.cost;
+    const int h = (a1 - P.cost_base + P.cost - 1) / P.cost;
     lo = min(l, P.groups);
     hi = min(h, P.groups);
 }
@@ -737,7 +738,11 @@ int launch_gemv_imma(const LinearArgs *problems, int count, cudaStream_t s)
                 return BTC_ERR_UNSUPPORTED;                 // shape the tensor map cannot describe: other kernels take it
         }
         p.cost_base = (int)cost;
-        cost += (long long)p.groups * a.Kb;
+        // measured: an iteration (one row group x one part of up to 256 blocks) costs about the same whatever the
+        // part's width, and rebuilding the activation fragments for a part costs ~1.5 iterations, shared by the
+        // (few) row groups a CTA walks with it; a single-part layer rebuilds only once per CTA
+        p.cost = p.parts > 1 ? p.parts * (IM_PW + 110) : a.Kb + 40;
+        cost += (long long)p.groups * p.cost;
         groups_total += p.groups;
         if (p.ncls > ncls_max) ncls_max = p.ncls;
         if (Kc4 * 4 > tab_max) tab_max = Kc4 * 4;
