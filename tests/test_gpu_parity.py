@@ -232,3 +232,47 @@ def test_online_transform_prologue(path, M, k1, k2):
     assert err.max() / np.abs(ref).max() <= TOL_GEMM
     scale = np.outer(np.abs(xt).sum(1), np.abs(L.alpha.astype(np.float64)))
     assert (err / np.maximum(scale, 1e-300)).max() <= TOL_GEMM
+
+
+# ------------------------------------------------------------------ invariants through the production kernels
+
+@pytest.mark.parametrize("path,M", [("gemv", 1), ("gemv", 6), ("gemm", 72)])
+def test_codebook_permutation_and_negation_invariance(path, M):
+    """Relabelling the centroids (codebook rows permuted, indices remapped) must not change y at all, and negating
+    every centroid together with every alpha must give the same y: both hold bit for bit, because each kernel sees the
+    same weights in the same order."""
+    N, K, v, Kc = 304, 1024, 16, 4096
+    L = wl.make_layer(_spec(N, K, v, Kc, x_dtype="f16" if path == "gemv" else "bf16"), M, seed=31)
+    y0, _ = run_layer(L, path)
+    rng = np.random.default_rng(3)
+    perm = rng.permutation(Kc)                       # new position of old centroid k is inv[k]
+    inv = np.empty(Kc, dtype=np.int64)
+    inv[perm] = np.arange(Kc)
+    L1 = wl.LayerData(L.spec, M, L.C_pm1[perm].copy(), inv[L.idx].astype(np.uint16), L.alpha, L.x_bits, L.mu)
+    y1, _ = run_layer(L1, path)
+    assert torch.equal(y0, y1)
+    L2 = wl.LayerData(L.spec, M, (-L.C_pm1).astype(np.int8), L.idx, (-L.alpha).astype(np.float16), L.x_bits, L.mu)
+    y2, _ = run_layer(L2, path)
+    rel, fwd = errors(y2, oracle_y(L), L)
+    tol = TOL_GEMV if path == "gemv" else TOL_GEMM
+    assert rel <= tol and fwd <= tol
+    if path == "gemm":                               # exact +-1 products, same accumulation order
+        assert torch.equal(y0, y2)
+
+
+def test_gemv_is_linear_in_x_for_powers_of_two():
+    """Scaling x by a power of two scales y by the same factor exactly (the per-slice block-fixed-point scale follows)."""
+    L = wl.make_layer(_spec(272, 2048, 16, 8192), 2, seed=8)
+    y0, _ = run_layer(L, "gemv")
+    L4 = wl.LayerData(L.spec, 2, L.C_pm1, L.idx, L.alpha, (L.x_bits.view(np.float16) * np.float16(4.0)).view(np.uint16), L.mu)
+    y4, _ = run_layer(L4, "gemv")
+    assert torch.equal(y4, 4.0 * y0)
+
+
+def test_rows_of_x_are_independent():
+    """Row m of y depends on row m of x only: running rows one at a time gives the same numbers as running them together."""
+    L = wl.make_layer(_spec(272, 1024, 16, 4096), 2, seed=21)
+    y, d = run_layer(L, "gemv")
+    for m in range(2):
+        ym = btc.linear_gemv(d["x"][m:m + 1].contiguous(), d["idx"], d["Cp"], d["alpha"], 16, 4096)
+        assert torch.equal(ym[0], y[m])
