@@ -276,3 +276,16 @@ def test_rows_of_x_are_independent():
     for m in range(2):
         ym = btc.linear_gemv(d["x"][m:m + 1].contiguous(), d["idx"], d["Cp"], d["alpha"], 16, 4096)
         assert torch.equal(ym[0], y[m])
+
+
+def test_gemm_many_tiles_ragged_shapes():
+    """More tiles than SMs, ragged N and M, and a K that ends inside an index tile (17 k steps); 30 sampled rows of y
+    (all columns) against the oracle, with mu."""
+    N, K, M = 2100, 1088, 2300
+    L = wl.make_layer(_spec(N, K, 16, 7132, x_dtype="bf16", with_mu=True), M, seed=123)
+    y, _ = run_layer(L, "gemm")
+    rows = np.unique(np.concatenate([[0, 127, 128, 255, 256, M - 1], (np.arange(24) * 97 + 13) % M]))
+    sub = wl.LayerData(L.spec, len(rows), L.C_pm1, L.idx, L.alpha, L.x_bits[rows].copy(), L.mu)
+    rel, fwd = errors(y[torch.from_numpy(rows).cuda()], oracle_y(sub), sub)
+    assert rel <= TOL_GEMM and fwd <= TOL_GEMM, (rel, fwd)
+    assert bool(torch.isfinite(y).all()) and btc.device_status() == 0
