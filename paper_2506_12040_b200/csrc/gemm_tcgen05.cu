@@ -287,12 +287,13 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_x, const GemmParams
 //   warp 0      TMA producer: x tiles, and index tiles (128 rows x 64 blocks = 16 k steps, 128-byte swizzle);
 //               bulk copy of the codeword table into shared memory
 //   warp 1      MMA issuer          warp 2   tensor-memory allocation
-//   warps 4-19  decode, in two groups of eight that take the even and the odd k steps (more lookups in flight):
-//               thread (row r, half h) expands blocks 2h, 2h+1 of the k step: two table lookups in shared
+//   warps 4-19  decode, in GROUPS groups (2 of eight warps with 256-row x tiles, 4 of four warps with 128-row ones)
+//               that take the k steps g, g + GROUPS, ...: a group has GROUPS MMA k steps of time for its lookups,
+//               stores and proxy fence.  A thread expands 2 or 4 blocks of its weight row: table lookups in shared
 //               memory, and per pair of weights one shift and one LOP3 -- the table keeps the bit of weight t at
 //               (t & 1) * 16 + 4 + (t >> 1), so ((~w << (11 - j)) & 0x80008000) | {1.0, 1.0} is the pair
 //               (2j, 2j+1) as +-1 in bf16 / fp16; then the same warps run the epilogue, four per lane quadrant.
-constexpr int G2_DWARPS = 16;                    // two groups of 8: even and odd k steps
+constexpr int G2_DWARPS = 16;                    // decode warps, in GROUPS groups that take the k steps g, g + GROUPS, ...
 constexpr int G2_THREADS = 128 + G2_DWARPS * 32;
 constexpr uint32_t G2_IDX_BYTES = 128 * 128;     // one index tile
 
@@ -309,7 +310,7 @@ __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void *src, uint32_t
                  ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
 }
 
-template <int BM, int STAGES>
+template <int BM, int STAGES, int GROUPS>
 __global__ void __launch_bounds__(G2_THREADS, 1)
 gemm_v16_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_i, const Gemm2Params p)
 {
@@ -341,7 +342,7 @@ gemm_v16_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
     if (tid == 0) {
         for (int s = 0; s < STAGES; ++s) {
             mbar_init(bar_full_x(s), 1);
-            mbar_init(bar_full_w(s), G2_DWARPS / 2);
+            mbar_init(bar_full_w(s), G2_DWARPS / GROUPS);
             mbar_init(bar_empty(s), 1);
         }
         mbar_init(bar_accum, 1);
@@ -397,28 +398,39 @@ gemm_v16_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
             umma_commit(bar_accum);
         }
     } else if (warp >= 4) {
-        const int d = (tid - 128) & 255;               // position in the group
-        const int grp = (tid - 128) >> 8;              // 0: even k steps, 1: odd k steps
-        const int r = d & 127, h = d >> 7;             // weight row of the tile, half of the k step
+        // A stage's barrier phases are waited on by parity, which is only meaningful for the phase right after the
+        // last one a thread has seen.  With GROUPS == STAGES a group always meets the same stage, phase after phase;
+        // with 2 groups and 3 stages a group meets a stage every other phase, one k step of its own in between.
+        static_assert(GROUPS == 2 || GROUPS == STAGES, "a group must see every phase of the stages it writes, or every other");
+        constexpr int GT = G2_DWARPS * 32 / GROUPS;    // threads of a group: 256 or 128
+        constexpr int BPT = 4 * 128 / GT;              // blocks of the k step per thread: 2 or 4
+        const int d = (tid - 128) % GT;                // position in the group
+        const int grp = (tid - 128) / GT;
+        const int r = d & 127, h = d >> 7;             // weight row of the tile, part of the k step
         const uint32_t one2 = is_bf16 ? 0x3F803F80u : 0x3C003C00u;
         const bool tab_smem = p.tab_bytes > 0;
         if (tab_smem && !mbar_wait(bar_tab, 0, s_abort)) { /* fall through: waits below bail out */ }
         bool ok = true;
         int cur_it = -1;
-        for (int kt = grp; kt < KT && ok; kt += 2) {
+        for (int kt = grp; kt < KT && ok; kt += GROUPS) {
             const int it = kt >> 4, ib = it & 1;
             if (it != cur_it) {
                 if (!mbar_wait(bar_full_i(ib), (it >> 1) & 1, s_abort)) { ok = false; break; }
                 cur_it = it;
             }
-            // index pair of blocks 2h, 2h+1 of this k step: column (kt % 16) * 4 + 2h of the index tile
-            const int boff = (kt & 15) * 8 + 4 * h;
-            const uint32_t pair = *reinterpret_cast<const uint32_t *>(
-                s_idx + (size_t)ib * G2_IDX_BYTES + (size_t)r * 128 + ((((boff >> 4) & 7) ^ (r & 7)) << 4) + (boff & 15));
-            const uint32_t i0 = pair & 0xffffu, i1 = pair >> 16;
-            const uint32_t w0 = ~(tab_smem ? s_tab[i0] : __ldg(p.tab + i0));
-            const uint32_t w1 = ~(tab_smem ? s_tab[i1] : __ldg(p.tab + i1));
-            if (((kt + 2) >> 4) != it || kt + 2 >= KT) {           // this group's last k step in the index tile
+            // indices of blocks h * BPT .. of this k step: columns (kt % 16) * 4 + h * BPT .. of the index tile
+            const int boff = (kt & 15) * 8 + 2 * BPT * h;
+            const unsigned char *ip = s_idx + (size_t)ib * G2_IDX_BYTES + (size_t)r * 128 + ((((boff >> 4) & 7) ^ (r & 7)) << 4) + (boff & 15);
+            uint32_t pairs[BPT / 2];
+            pairs[0] = *reinterpret_cast<const uint32_t *>(ip);
+            if (BPT == 4) pairs[BPT / 2 - 1] = *reinterpret_cast<const uint32_t *>(ip + 4);
+            uint32_t w[BPT];
+#pragma unroll
+            for (int b = 0; b < BPT; ++b) {
+                const uint32_t i = (b & 1) ? (pairs[b >> 1] >> 16) : (pairs[b >> 1] & 0xffffu);
+                w[b] = ~(tab_smem ? s_tab[i] : __ldg(p.tab + i));
+            }
+            if (((kt + GROUPS) >> 4) != it || kt + GROUPS >= KT) {   // this group's last k step in the index tile
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar_empty_i(ib));
             }
@@ -427,16 +439,15 @@ gemm_v16_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
             if (kt >= STAGES && !mbar_wait(bar_empty(s), ph ^ 1, s_abort)) { ok = false; break; }
             unsigned char *arow = smem_gen + (size_t)s * STAGE_BYTES + (size_t)r * 128;
 #pragma unroll
-            for (int b = 0; b < 2; ++b) {
-                const uint32_t w = b ? w1 : w0;
+            for (int b = 0; b < BPT; ++b) {
 #pragma unroll
                 for (int c = 0; c < 2; ++c) {
                     uint4 q;
-                    q.x = ((w << (11 - (4 * c + 0))) & 0x80008000u) | one2;
-                    q.y = ((w << (11 - (4 * c + 1))) & 0x80008000u) | one2;
-                    q.z = ((w << (11 - (4 * c + 2))) & 0x80008000u) | one2;
-                    q.w = ((w << (11 - (4 * c + 3))) & 0x80008000u) | one2;
-                    const int chunk = (2 * h + b) * 2 + c;
+                    q.x = ((w[b] << (11 - (4 * c + 0))) & 0x80008000u) | one2;
+                    q.y = ((w[b] << (11 - (4 * c + 1))) & 0x80008000u) | one2;
+                    q.z = ((w[b] << (11 - (4 * c + 2))) & 0x80008000u) | one2;
+                    q.w = ((w[b] << (11 - (4 * c + 3))) & 0x80008000u) | one2;
+                    const int chunk = (BPT * h + b) * 2 + c;
                     *reinterpret_cast<uint4 *>(arow + ((chunk ^ (r & 7)) << 4)) = q;
                 }
             }
@@ -513,12 +524,12 @@ static int launch_cfg(const CUtensorMap &tm, const GemmParams &p, cudaStream_t s
     return cuda_check_launch();
 }
 
-template <int BM, int STAGES>
+template <int BM, int STAGES, int GROUPS>
 static int launch_v16(const CUtensorMap &tm, const CUtensorMap &ti, const Gemm2Params &p, cudaStream_t s)
 {
     const size_t smem = (size_t)STAGES * (G_A_BYTES + BM * G_BK * 2) + 1024 + 2 * G2_IDX_BYTES + ((p.tab_bytes + 15) & ~15) +
                         (3 * STAGES + 6) * 8 + 16;
-    auto kern = gemm_v16_kernel<BM, STAGES>;
+    auto kern = gemm_v16_kernel<BM, STAGES, GROUPS>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return cuda_fail(e);
     dim3 grid((p.a.N + G_BN - 1) / G_BN, (p.a.M + BM - 1) / BM);
@@ -578,8 +589,8 @@ int launch_gemm_tcgen05(const LinearArgs &a, cudaStream_t s)
             const size_t fixed = (BM == 256 ? 3 * (G_A_BYTES + 256 * G_BK * 2) : 4 * (G_A_BYTES + 128 * G_BK * 2)) + 1024 +
                                  2 * G2_IDX_BYTES + 256;
             q.tab_bytes = (fixed + (size_t)Kc4 * 4 <= 227u * 1024u) ? Kc4 * 4 : 0;
-            if (BM == 256) return launch_v16<256, 3>(tm, ti, q, s);
-            return launch_v16<128, 4>(tm, ti, q, s);
+            if (BM == 256) return launch_v16<256, 3, 2>(tm, ti, q, s);
+            return launch_v16<128, 4, 4>(tm, ti, q, s);
         }
     }
     if (BM == 256) return launch_cfg<256, 4>(tm, p, s);
