@@ -49,13 +49,17 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
         : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
     return ok != 0;
 }
-// Bounded wait.  Returns false (and latches *abort_flag) when the deadline passes.
+// Bounded wait.  Returns false (and latches *abort_flag) when the deadline passes.  BACKOFF: sleep between polls;
+// every role but the MMA issuer uses it, because a warp that spins takes issue slots from the one thread whose
+// instruction stream paces the tensor core.
+template <bool BACKOFF = true>
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag) {
-    if (*abort_flag) return false;
     if (mbar_try_wait(bar, parity)) return true;
+    if (*abort_flag) return false;
     const long long t0 = clock64();
     int spins = 0;
     while (!mbar_try_wait(bar, parity)) {
+        if (BACKOFF) __nanosleep(spins < 8 ? 32 : 128);
         if ((++spins & 63) == 0) {
             if (*abort_flag) return false;
             if (clock64() - t0 > 4000000000LL) {   // ~2 s at 2 GHz
@@ -198,8 +202,8 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_x, const GemmParams
             for (int kt = 0; kt < KT; ++kt) {
                 const int s = kt % STAGES;
                 const uint32_t ph = (kt / STAGES) & 1;
-                mbar_wait(bar_full_x(s), ph, s_abort);
-                mbar_wait(bar_full_w(s), ph, s_abort);
+                mbar_wait<false>(bar_full_x(s), ph, s_abort);
+                mbar_wait<false>(bar_full_w(s), ph, s_abort);
                 tc_fence_after();
                 const uint32_t a_addr = smem_base + s * STAGE_BYTES;
                 const uint64_t adesc = make_smem_desc(a_addr);
@@ -384,8 +388,8 @@ gemm_v16_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
             for (int kt = 0; kt < KT; ++kt) {
                 const int s = kt % STAGES;
                 const uint32_t ph = (kt / STAGES) & 1;
-                if (!mbar_wait(bar_full_x(s), ph, s_abort)) break;
-                if (!mbar_wait(bar_full_w(s), ph, s_abort)) break;
+                if (!mbar_wait<false>(bar_full_x(s), ph, s_abort)) break;
+                if (!mbar_wait<false>(bar_full_w(s), ph, s_abort)) break;
                 tc_fence_after();
                 const uint32_t a_addr = smem_base + s * STAGE_BYTES;
                 const uint64_t adesc = make_smem_desc(a_addr);
@@ -493,6 +497,205 @@ gemm_v16_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
     if (warp == 2) tmem_dealloc(tmem_d, BM);
 }
 
+// ------------------------------------------------------------------------------------ v = 16, weights in tensor memory
+// With both operands in shared memory the kernel above is bound by shared-memory bandwidth: per 64-wide k step the
+// tensor core reads the A and B tiles while the decode warps write 16 KB of A and TMA writes the x tile, more than
+// the 128 bytes per clock an SM's shared memory delivers (66 % of the MMA rate at best with 256-row x tiles, 50 % with
+// 128-row ones).  Here the decoded +-1 tile never touches shared memory: each decode thread owns one weight row =
+// one tensor-memory lane, expands the row's 64 weights of a k step into 32 registers and stores them with
+// tcgen05.st into a ring of A tiles in tensor memory (32 columns per k step); the MMAs take A from tensor memory and
+// only the x tile from shared memory.
+//   warp 0 TMA producer (x tiles, index tiles, table) | warp 1 MMA issuer | warp 2 tensor-memory allocation
+//   warps 4-19: four groups of four warps; group g expands the k steps g, g + 4, ...; then all 16 run the epilogue.
+// Tensor memory (512 columns): accumulator in columns [0, BM), A ring of G4_ASTAGES x 32 columns from column 256.
+constexpr int G4_ASTAGES = 8;
+constexpr int G4_A_COL0 = 256;
+
+__device__ __forceinline__ void umma_f16_ts(uint32_t tmem_d, uint32_t tmem_a, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+        ::"r"(tmem_d), "r"(tmem_a), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32]) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+        "{%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,"
+        "%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32};"
+        :: "r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
+           "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]),
+           "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]),
+           "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
+        : "memory");
+}
+__device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+template <int BM, int STAGES>
+__global__ void __launch_bounds__(G2_THREADS, 1)
+gemm_v16t_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_i, const Gemm2Params p)
+{
+    constexpr uint32_t B_BYTES = BM * G_BK * 2;                    // a stage is one x tile
+    static_assert(BM <= G4_A_COL0, "accumulator and A ring must not overlap");
+    extern __shared__ __align__(1024) unsigned char smem_raw[];
+    const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    unsigned char *smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
+    unsigned char *s_idx = smem_gen + (size_t)STAGES * B_BYTES;                     // 2 index tiles
+    uint32_t *s_tab = reinterpret_cast<uint32_t *>(s_idx + 2 * G2_IDX_BYTES);
+    uint64_t *bars = reinterpret_cast<uint64_t *>(reinterpret_cast<unsigned char *>(s_tab) + ((p.tab_bytes + 15) & ~15));
+    // bars: [0,S) full_x, [S,2S) empty_x, then full_a[AS], empty_a[AS], accum, full_i[2], empty_i[2], tab_full
+    constexpr int NB = 2 * STAGES + 2 * G4_ASTAGES + 6;
+    uint32_t *s_tmem = reinterpret_cast<uint32_t *>(bars + NB);
+    volatile int *s_abort = reinterpret_cast<volatile int *>(s_tmem + 1);
+
+    const LinearArgs &a = p.a;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int n0 = blockIdx.x * G_BN, m0 = blockIdx.y * BM;
+    const int KT = p.k_tiles;
+    const bool is_bf16 = (a.x_dt == BTC_BF16);
+    auto bar_full_x = [&](int s) { return smem_u32(bars + s); };
+    auto bar_empty_x = [&](int s) { return smem_u32(bars + STAGES + s); };
+    auto bar_full_a = [&](int s) { return smem_u32(bars + 2 * STAGES + s); };
+    auto bar_empty_a = [&](int s) { return smem_u32(bars + 2 * STAGES + G4_ASTAGES + s); };
+    const uint32_t bar_accum = smem_u32(bars + 2 * STAGES + 2 * G4_ASTAGES);
+    auto bar_full_i = [&](int b) { return smem_u32(bars + 2 * STAGES + 2 * G4_ASTAGES + 1 + b); };
+    auto bar_empty_i = [&](int b) { return smem_u32(bars + 2 * STAGES + 2 * G4_ASTAGES + 3 + b); };
+    const uint32_t bar_tab = smem_u32(bars + 2 * STAGES + 2 * G4_ASTAGES + 5);
+
+    if (tid == 0) {
+        for (int s = 0; s < STAGES; ++s) { mbar_init(bar_full_x(s), 1); mbar_init(bar_empty_x(s), 1); }
+        for (int s = 0; s < G4_ASTAGES; ++s) { mbar_init(bar_full_a(s), 4); mbar_init(bar_empty_a(s), 1); }
+        mbar_init(bar_accum, 1);
+        for (int b = 0; b < 2; ++b) { mbar_init(bar_full_i(b), 1); mbar_init(bar_empty_i(b), G2_DWARPS); }
+        mbar_init(bar_tab, 1);
+        *s_abort = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 2) tmem_alloc(smem_u32(s_tmem), 512);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_d = *s_tmem;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            if (p.tab_bytes > 0) {
+                mbar_expect_tx(bar_tab, (uint32_t)p.tab_bytes);
+                bulk_g2s(smem_u32(s_tab), p.tab, (uint32_t)p.tab_bytes, bar_tab);
+            }
+            for (int kt = 0; kt < KT; ++kt) {
+                if ((kt & 15) == 0) {
+                    const int it = kt >> 4, ib = it & 1;
+                    if (it >= 2 && !mbar_wait(bar_empty_i(ib), ((it >> 1) & 1) ^ 1, s_abort)) break;
+                    mbar_expect_tx(bar_full_i(ib), G2_IDX_BYTES);
+                    tma_load_2d(smem_u32(s_idx + (size_t)ib * G2_IDX_BYTES), &tmap_i, it * 64, n0, bar_full_i(ib));
+                }
+                const int s = kt % STAGES;
+                if (kt >= STAGES && !mbar_wait(bar_empty_x(s), ((kt / STAGES) & 1) ^ 1, s_abort)) break;
+                mbar_expect_tx(bar_full_x(s), B_BYTES);
+                tma_load_2d(smem_base + s * B_BYTES, &tmap_x, kt * G_BK, m0, bar_full_x(s));
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            uint32_t idesc = (1u << 4) | ((uint32_t)(BM >> 3) << 17) | ((uint32_t)(G_BN >> 4) << 24);
+            if (is_bf16) idesc |= (1u << 7) | (1u << 10);
+            for (int kt = 0; kt < KT; ++kt) {
+                const int s = kt % STAGES, sa = kt % G4_ASTAGES;
+                if (!mbar_wait<false>(bar_full_x(s), (kt / STAGES) & 1, s_abort)) break;
+                if (!mbar_wait<false>(bar_full_a(sa), (kt / G4_ASTAGES) & 1, s_abort)) break;
+                tc_fence_after();
+                const uint64_t bdesc = make_smem_desc(smem_base + s * B_BYTES);
+                const uint32_t a_tm = tmem_d + G4_A_COL0 + sa * 32;
+#pragma unroll
+                for (int k = 0; k < G_BK / 16; ++k)
+                    umma_f16_ts(tmem_d, a_tm + 8 * k, bdesc + 2 * k, idesc, (kt | k) ? 1u : 0u);
+                umma_commit(bar_empty_x(s));
+                umma_commit(bar_empty_a(sa));
+            }
+            umma_commit(bar_accum);
+        }
+    } else if (warp >= 4) {
+        const int r = (tid - 128) & 127;               // weight row of the tile = tensor-memory lane
+        const int grp = (tid - 128) >> 7;              // k steps grp, grp + 4, ...: an A stage (kt % 8) is always met by the same
+                                                       // group, phase after phase, so its parity waits are unambiguous
+        const uint32_t one2 = is_bf16 ? 0x3F803F80u : 0x3C003C00u;
+        const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
+        const bool tab_smem = p.tab_bytes > 0;
+        if (tab_smem && !mbar_wait(bar_tab, 0, s_abort)) { /* fall through: waits below bail out */ }
+        bool ok = true;
+        int cur_it = -1;
+        for (int kt = grp; kt < KT && ok; kt += 4) {
+            const int it = kt >> 4, ib = it & 1;
+            if (it != cur_it) {
+                if (!mbar_wait(bar_full_i(ib), (it >> 1) & 1, s_abort)) { ok = false; break; }
+                cur_it = it;
+            }
+            // the four indices of this row's k step: columns (kt % 16) * 4 .. + 3 of the index tile (8 bytes)
+            const int boff = (kt & 15) * 8;
+            const uint2 quad = *reinterpret_cast<const uint2 *>(
+                s_idx + (size_t)ib * G2_IDX_BYTES + (size_t)r * 128 + ((((boff >> 4) & 7) ^ (r & 7)) << 4) + (boff & 15));
+            uint32_t w[4];
+            w[0] = ~(tab_smem ? s_tab[quad.x & 0xffffu] : __ldg(p.tab + (quad.x & 0xffffu)));
+            w[1] = ~(tab_smem ? s_tab[quad.x >> 16] : __ldg(p.tab + (quad.x >> 16)));
+            w[2] = ~(tab_smem ? s_tab[quad.y & 0xffffu] : __ldg(p.tab + (quad.y & 0xffffu)));
+            w[3] = ~(tab_smem ? s_tab[quad.y >> 16] : __ldg(p.tab + (quad.y >> 16)));
+            if (((kt + 4) >> 4) != it || kt + 4 >= KT) {           // this group's last k step in the index tile
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_empty_i(ib));
+            }
+            // register j holds the weights 2j, 2j+1 of the k step (K elements 2j, 2j+1 of this row of A)
+            uint32_t regs[32];
+#pragma unroll
+            for (int b = 0; b < 4; ++b)
+#pragma unroll
+                for (int j = 0; j < 8; ++j) regs[8 * b + j] = ((w[b] << (11 - j)) & 0x80008000u) | one2;
+            const int sa = kt % G4_ASTAGES;
+            if (kt >= G4_ASTAGES && !mbar_wait(bar_empty_a(sa), ((kt / G4_ASTAGES) & 1) ^ 1, s_abort)) { ok = false; break; }
+            tc_fence_after();
+            tmem_st32(tmem_d + lane_base + G4_A_COL0 + sa * 32, regs);
+            tmem_st_wait();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_full_a(sa));
+        }
+        // ------------------------------------------------------------ epilogue: four warps per lane quadrant
+        if (ok && mbar_wait(bar_accum, 0, s_abort)) {
+            tc_fence_after();
+            const int wl = warp - 4;
+            const int q4 = wl & 3, quarter = wl >> 2;
+            const int nrow = n0 + q4 * 32 + lane;
+            const int nc = min(nrow, a.N - 1);
+            const float al = __half2float(a.alpha[nc]);
+            const float mu = a.mu ? __half2float(a.mu[nc]) : 0.f;
+#pragma unroll 1
+            for (int c0 = quarter * (BM / 4); c0 < (quarter + 1) * (BM / 4); c0 += 32) {
+                uint32_t rr[32];
+                tmem_ld32(tmem_d + lane_base + c0, rr);
+                tmem_ld_wait();
+                if (nrow < a.N) {
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) {
+                        const int m = m0 + c0 + i;
+                        if (m < a.M) {
+                            float y = al * __uint_as_float(rr[i]);
+                            if (a.mu) y += mu * p.sumx[m];
+                            store_from_float(a.y, a.y_dt, (size_t)m * a.N + nrow, y);
+                        }
+                    }
+                }
+            }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (*s_abort) {
+        for (int i = 0; i < 200; ++i) __nanosleep(1000);
+        __syncthreads();
+    }
+    if (warp == 2) tmem_dealloc(tmem_d, 512);
+}
+
 // ------------------------------------------------------------------------------------ host side
 typedef CUresult (*encode_tiled_fn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
                                     const cuuint64_t *, const cuuint32_t *, const cuuint32_t *,
@@ -530,6 +733,19 @@ static int launch_v16(const CUtensorMap &tm, const CUtensorMap &ti, const Gemm2P
     const size_t smem = (size_t)STAGES * (G_A_BYTES + BM * G_BK * 2) + 1024 + 2 * G2_IDX_BYTES + ((p.tab_bytes + 15) & ~15) +
                         (3 * STAGES + 6) * 8 + 16;
     auto kern = gemm_v16_kernel<BM, STAGES, GROUPS>;
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return cuda_fail(e);
+    dim3 grid((p.a.N + G_BN - 1) / G_BN, (p.a.M + BM - 1) / BM);
+    kern<<<grid, G2_THREADS, smem, s>>>(tm, ti, p);
+    return cuda_check_launch();
+}
+
+template <int BM, int STAGES>
+static int launch_v16t(const CUtensorMap &tm, const CUtensorMap &ti, const Gemm2Params &p, cudaStream_t s)
+{
+    const size_t smem = (size_t)STAGES * (BM * G_BK * 2) + 1024 + 2 * G2_IDX_BYTES + ((p.tab_bytes + 15) & ~15) +
+                        (2 * STAGES + 2 * G4_ASTAGES + 6) * 8 + 16;
+    auto kern = gemm_v16t_kernel<BM, STAGES>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return cuda_fail(e);
     dim3 grid((p.a.N + G_BN - 1) / G_BN, (p.a.M + BM - 1) / BM);
@@ -589,8 +805,12 @@ int launch_gemm_tcgen05(const LinearArgs &a, cudaStream_t s)
             const size_t fixed = (BM == 256 ? 3 * (G_A_BYTES + 256 * G_BK * 2) : 4 * (G_A_BYTES + 128 * G_BK * 2)) + 1024 +
                                  2 * G2_IDX_BYTES + 256;
             q.tab_bytes = (fixed + (size_t)Kc4 * 4 <= 227u * 1024u) ? Kc4 * 4 : 0;
-            if (BM == 256) return launch_v16<256, 3, 2>(tm, ti, q, s);
-            return launch_v16<128, 4, 4>(tm, ti, q, s);
+            {   // weights through tensor memory: shared memory holds only x tiles, index tiles and the table
+                const size_t fixed_t = (size_t)(BM == 256 ? 5 : 9) * (BM * G_BK * 2) + 1024 + 2 * G2_IDX_BYTES + 512;
+                q.tab_bytes = (fixed_t + (size_t)Kc4 * 4 <= 227u * 1024u) ? Kc4 * 4 : 0;
+                if (BM == 256) return launch_v16t<256, 5>(tm, ti, q, s);
+                return launch_v16t<128, 9>(tm, ti, q, s);
+            }
         }
     }
     if (BM == 256) return launch_cfg<256, 4>(tm, p, s);
