@@ -507,8 +507,7 @@ gemm_v16_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
 // only the x tile from shared memory.
 //   warp 0 TMA producer (x tiles, index tiles, table) | warp 1 MMA issuer | warp 2 tensor-memory allocation
 //   warps 4-19: four groups of four warps; group g expands the k steps g, g + 4, ...; then all 16 run the epilogue.
-// Tensor memory (512 columns): accumulator in columns [0, BM), A ring of G4_ASTAGES x 32 columns from column 256.
-constexpr int G4_ASTAGES = 8;
+// Tensor memory (512 columns): accumulator in columns [0, BM), A ring of STAGES x 32 columns from column 256.
 constexpr int G4_A_COL0 = 256;
 
 __device__ __forceinline__ void umma_f16_ts(uint32_t tmem_d, uint32_t tmem_a, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
@@ -543,8 +542,11 @@ gemm_v16t_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
     unsigned char *s_idx = smem_gen + (size_t)STAGES * B_BYTES;                     // 2 index tiles
     uint32_t *s_tab = reinterpret_cast<uint32_t *>(s_idx + 2 * G2_IDX_BYTES);
     uint64_t *bars = reinterpret_cast<uint64_t *>(reinterpret_cast<unsigned char *>(s_tab) + ((p.tab_bytes + 15) & ~15));
-    // bars: [0,S) full_x, [S,2S) empty_x, then full_a[AS], empty_a[AS], accum, full_i[2], empty_i[2], tab_full
-    constexpr int NB = 2 * STAGES + 2 * G4_ASTAGES + 6;
+    // One ring of STAGES stages holds both operands of a k step: the x tile in shared memory and the A tile in tensor
+    // memory.  full[s]: the TMA arrival (with its bytes) plus the four decode warps; empty[s]: the MMAs' commit.
+    // bars: [0,S) full, [S,2S) empty, accum, full_i[2], empty_i[2], tab_full
+    static_assert(STAGES % 4 == 0 && STAGES * 32 <= 512 - G4_A_COL0, "a decode group must meet a stage in consecutive phases");
+    constexpr int NB = 2 * STAGES + 6;
     uint32_t *s_tmem = reinterpret_cast<uint32_t *>(bars + NB);
     volatile int *s_abort = reinterpret_cast<volatile int *>(s_tmem + 1);
 
@@ -553,18 +555,15 @@ gemm_v16t_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
     const int n0 = blockIdx.x * G_BN, m0 = blockIdx.y * BM;
     const int KT = p.k_tiles;
     const bool is_bf16 = (a.x_dt == BTC_BF16);
-    auto bar_full_x = [&](int s) { return smem_u32(bars + s); };
-    auto bar_empty_x = [&](int s) { return smem_u32(bars + STAGES + s); };
-    auto bar_full_a = [&](int s) { return smem_u32(bars + 2 * STAGES + s); };
-    auto bar_empty_a = [&](int s) { return smem_u32(bars + 2 * STAGES + G4_ASTAGES + s); };
-    const uint32_t bar_accum = smem_u32(bars + 2 * STAGES + 2 * G4_ASTAGES);
-    auto bar_full_i = [&](int b) { return smem_u32(bars + 2 * STAGES + 2 * G4_ASTAGES + 1 + b); };
-    auto bar_empty_i = [&](int b) { return smem_u32(bars + 2 * STAGES + 2 * G4_ASTAGES + 3 + b); };
-    const uint32_t bar_tab = smem_u32(bars + 2 * STAGES + 2 * G4_ASTAGES + 5);
+    auto bar_full = [&](int s) { return smem_u32(bars + s); };
+    auto bar_empty = [&](int s) { return smem_u32(bars + STAGES + s); };
+    const uint32_t bar_accum = smem_u32(bars + 2 * STAGES);
+    auto bar_full_i = [&](int b) { return smem_u32(bars + 2 * STAGES + 1 + b); };
+    auto bar_empty_i = [&](int b) { return smem_u32(bars + 2 * STAGES + 3 + b); };
+    const uint32_t bar_tab = smem_u32(bars + 2 * STAGES + 5);
 
     if (tid == 0) {
-        for (int s = 0; s < STAGES; ++s) { mbar_init(bar_full_x(s), 1); mbar_init(bar_empty_x(s), 1); }
-        for (int s = 0; s < G4_ASTAGES; ++s) { mbar_init(bar_full_a(s), 4); mbar_init(bar_empty_a(s), 1); }
+        for (int s = 0; s < STAGES; ++s) { mbar_init(bar_full(s), 1 + 4); mbar_init(bar_empty(s), 1); }
         mbar_init(bar_accum, 1);
         for (int b = 0; b < 2; ++b) { mbar_init(bar_full_i(b), 1); mbar_init(bar_empty_i(b), G2_DWARPS); }
         mbar_init(bar_tab, 1);
@@ -591,9 +590,9 @@ gemm_v16t_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                     tma_load_2d(smem_u32(s_idx + (size_t)ib * G2_IDX_BYTES), &tmap_i, it * 64, n0, bar_full_i(ib));
                 }
                 const int s = kt % STAGES;
-                if (kt >= STAGES && !mbar_wait(bar_empty_x(s), ((kt / STAGES) & 1) ^ 1, s_abort)) break;
-                mbar_expect_tx(bar_full_x(s), B_BYTES);
-                tma_load_2d(smem_base + s * B_BYTES, &tmap_x, kt * G_BK, m0, bar_full_x(s));
+                if (kt >= STAGES && !mbar_wait(bar_empty(s), ((kt / STAGES) & 1) ^ 1, s_abort)) break;
+                mbar_expect_tx(bar_full(s), B_BYTES);
+                tma_load_2d(smem_base + s * B_BYTES, &tmap_x, kt * G_BK, m0, bar_full(s));
             }
         }
     } else if (warp == 1) {
@@ -601,24 +600,22 @@ gemm_v16t_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
             uint32_t idesc = (1u << 4) | ((uint32_t)(BM >> 3) << 17) | ((uint32_t)(G_BN >> 4) << 24);
             if (is_bf16) idesc |= (1u << 7) | (1u << 10);
             for (int kt = 0; kt < KT; ++kt) {
-                const int s = kt % STAGES, sa = kt % G4_ASTAGES;
-                if (!mbar_wait<false>(bar_full_x(s), (kt / STAGES) & 1, s_abort)) break;
-                if (!mbar_wait<false>(bar_full_a(sa), (kt / G4_ASTAGES) & 1, s_abort)) break;
+                const int s = kt % STAGES;
+                if (!mbar_wait<false>(bar_full(s), (kt / STAGES) & 1, s_abort)) break;
                 tc_fence_after();
                 const uint64_t bdesc = make_smem_desc(smem_base + s * B_BYTES);
-                const uint32_t a_tm = tmem_d + G4_A_COL0 + sa * 32;
+                const uint32_t a_tm = tmem_d + G4_A_COL0 + s * 32;
 #pragma unroll
                 for (int k = 0; k < G_BK / 16; ++k)
                     umma_f16_ts(tmem_d, a_tm + 8 * k, bdesc + 2 * k, idesc, (kt | k) ? 1u : 0u);
-                umma_commit(bar_empty_x(s));
-                umma_commit(bar_empty_a(sa));
+                umma_commit(bar_empty(s));
             }
             umma_commit(bar_accum);
         }
     } else if (warp >= 4) {
         const int r = (tid - 128) & 127;               // weight row of the tile = tensor-memory lane
-        const int grp = (tid - 128) >> 7;              // k steps grp, grp + 4, ...: an A stage (kt % 8) is always met by the same
-                                                       // group, phase after phase, so its parity waits are unambiguous
+        const int grp = (tid - 128) >> 7;              // k steps grp, grp + 4, ...: STAGES is a multiple of 4, so a stage is always
+                                                       // met by the same group, phase after phase: its parity waits are unambiguous
         const uint32_t one2 = is_bf16 ? 0x3F803F80u : 0x3C003C00u;
         const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
         const bool tab_smem = p.tab_bytes > 0;
@@ -650,14 +647,14 @@ gemm_v16t_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
             for (int b = 0; b < 4; ++b)
 #pragma unroll
                 for (int j = 0; j < 8; ++j) regs[8 * b + j] = ((w[b] << (11 - j)) & 0x80008000u) | one2;
-            const int sa = kt % G4_ASTAGES;
-            if (kt >= G4_ASTAGES && !mbar_wait(bar_empty_a(sa), ((kt / G4_ASTAGES) & 1) ^ 1, s_abort)) { ok = false; break; }
+            const int sa = kt % STAGES;
+            if (kt >= STAGES && !mbar_wait(bar_empty(sa), ((kt / STAGES) & 1) ^ 1, s_abort)) { ok = false; break; }
             tc_fence_after();
             tmem_st32(tmem_d + lane_base + G4_A_COL0 + sa * 32, regs);
             tmem_st_wait();
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(bar_full_a(sa));
+            if (lane == 0) mbar_arrive(bar_full(sa));
         }
         // ------------------------------------------------------------ epilogue: four warps per lane quadrant
         if (ok && mbar_wait(bar_accum, 0, s_abort)) {
@@ -744,7 +741,7 @@ template <int BM, int STAGES>
 static int launch_v16t(const CUtensorMap &tm, const CUtensorMap &ti, const Gemm2Params &p, cudaStream_t s)
 {
     const size_t smem = (size_t)STAGES * (BM * G_BK * 2) + 1024 + 2 * G2_IDX_BYTES + ((p.tab_bytes + 15) & ~15) +
-                        (2 * STAGES + 2 * G4_ASTAGES + 6) * 8 + 16;
+                        (2 * STAGES + 6) * 8 + 16;
     auto kern = gemm_v16t_kernel<BM, STAGES>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return cuda_fail(e);
@@ -806,10 +803,10 @@ int launch_gemm_tcgen05(const LinearArgs &a, cudaStream_t s)
                                  2 * G2_IDX_BYTES + 256;
             q.tab_bytes = (fixed + (size_t)Kc4 * 4 <= 227u * 1024u) ? Kc4 * 4 : 0;
             {   // weights through tensor memory: shared memory holds only x tiles, index tiles and the table
-                const size_t fixed_t = (size_t)(BM == 256 ? 5 : 9) * (BM * G_BK * 2) + 1024 + 2 * G2_IDX_BYTES + 512;
+                const size_t fixed_t = (size_t)(BM == 256 ? 4 : 8) * (BM * G_BK * 2) + 1024 + 2 * G2_IDX_BYTES + 512;
                 q.tab_bytes = (fixed_t + (size_t)Kc4 * 4 <= 227u * 1024u) ? Kc4 * 4 : 0;
-                if (BM == 256) return launch_v16t<256, 5>(tm, ti, q, s);
-                return launch_v16t<128, 9>(tm, ti, q, s);
+                if (BM == 256) return launch_v16t<256, 4>(tm, ti, q, s);
+                return launch_v16t<128, 8>(tm, ti, q, s);
             }
         }
     }
