@@ -530,22 +530,24 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32
 }
 __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
-template <int BM, int STAGES>
+template <int BM, int STAGES, int KS>
 __global__ void __launch_bounds__(G2_THREADS, 1)
 gemm_v16t_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_i, const Gemm2Params p)
 {
-    constexpr uint32_t B_BYTES = BM * G_BK * 2;                    // a stage is one x tile
+    constexpr uint32_t B_BYTES = BM * G_BK * 2;                    // one x tile (64 k); a stage holds KS of them
+    constexpr uint32_t STAGE_BYTES = KS * B_BYTES;
+    constexpr int ACOLS = 32 * KS;                                 // tensor-memory columns of a stage's A tile
     static_assert(BM <= G4_A_COL0, "accumulator and A ring must not overlap");
     extern __shared__ __align__(1024) unsigned char smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     unsigned char *smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
-    unsigned char *s_idx = smem_gen + (size_t)STAGES * B_BYTES;                     // 2 index tiles
+    unsigned char *s_idx = smem_gen + (size_t)STAGES * STAGE_BYTES;                 // 2 index tiles
     uint32_t *s_tab = reinterpret_cast<uint32_t *>(s_idx + 2 * G2_IDX_BYTES);
     uint64_t *bars = reinterpret_cast<uint64_t *>(reinterpret_cast<unsigned char *>(s_tab) + ((p.tab_bytes + 15) & ~15));
     // One ring of STAGES stages holds both operands of a k step: the x tile in shared memory and the A tile in tensor
     // memory.  full[s]: the TMA arrival (with its bytes) plus the four decode warps; empty[s]: the MMAs' commit.
     // bars: [0,S) full, [S,2S) empty, accum, full_i[2], empty_i[2], tab_full
-    static_assert(STAGES % 4 == 0 && STAGES * 32 <= 512 - G4_A_COL0, "a decode group must meet a stage in consecutive phases");
+    static_assert(STAGES % 4 == 0 && STAGES * ACOLS <= 512 - G4_A_COL0 && 16 % KS == 0, "a decode group must meet a stage in consecutive phases");
     constexpr int NB = 2 * STAGES + 6;
     uint32_t *s_tmem = reinterpret_cast<uint32_t *>(bars + NB);
     volatile int *s_abort = reinterpret_cast<volatile int *>(s_tmem + 1);
@@ -554,6 +556,7 @@ gemm_v16t_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int n0 = blockIdx.x * G_BN, m0 = blockIdx.y * BM;
     const int KT = p.k_tiles;
+    const int NS = (KT + KS - 1) / KS;                              // stages' worth of k steps
     const bool is_bf16 = (a.x_dt == BTC_BF16);
     auto bar_full = [&](int s) { return smem_u32(bars + s); };
     auto bar_empty = [&](int s) { return smem_u32(bars + STAGES + s); };
@@ -582,32 +585,38 @@ gemm_v16t_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                 mbar_expect_tx(bar_tab, (uint32_t)p.tab_bytes);
                 bulk_g2s(smem_u32(s_tab), p.tab, (uint32_t)p.tab_bytes, bar_tab);
             }
-            for (int kt = 0; kt < KT; ++kt) {
-                if ((kt & 15) == 0) {
-                    const int it = kt >> 4, ib = it & 1;
+            for (int ks = 0; ks < NS; ++ks) {
+                const int kt0 = ks * KS;
+                if ((kt0 & 15) == 0) {
+                    const int it = kt0 >> 4, ib = it & 1;
                     if (it >= 2 && !mbar_wait(bar_empty_i(ib), ((it >> 1) & 1) ^ 1, s_abort)) break;
                     mbar_expect_tx(bar_full_i(ib), G2_IDX_BYTES);
                     tma_load_2d(smem_u32(s_idx + (size_t)ib * G2_IDX_BYTES), &tmap_i, it * 64, n0, bar_full_i(ib));
                 }
-                const int s = kt % STAGES;
-                if (kt >= STAGES && !mbar_wait(bar_empty(s), ((kt / STAGES) & 1) ^ 1, s_abort)) break;
-                mbar_expect_tx(bar_full(s), B_BYTES);
-                tma_load_2d(smem_base + s * B_BYTES, &tmap_x, kt * G_BK, m0, bar_full(s));
+                const int s = ks % STAGES;
+                if (ks >= STAGES && !mbar_wait(bar_empty(s), ((ks / STAGES) & 1) ^ 1, s_abort)) break;
+                mbar_expect_tx(bar_full(s), STAGE_BYTES);
+#pragma unroll
+                for (int j = 0; j < KS; ++j)             // (a box past K arrives as zeros)
+                    tma_load_2d(smem_base + s * STAGE_BYTES + j * B_BYTES, &tmap_x, (kt0 + j) * G_BK, m0, bar_full(s));
             }
         }
     } else if (warp == 1) {
         if (lane == 0) {
             uint32_t idesc = (1u << 4) | ((uint32_t)(BM >> 3) << 17) | ((uint32_t)(G_BN >> 4) << 24);
             if (is_bf16) idesc |= (1u << 7) | (1u << 10);
-            for (int kt = 0; kt < KT; ++kt) {
-                const int s = kt % STAGES;
-                if (!mbar_wait<false>(bar_full(s), (kt / STAGES) & 1, s_abort)) break;
+            for (int ks = 0; ks < NS; ++ks) {
+                const int s = ks % STAGES;
+                if (!mbar_wait<false>(bar_full(s), (ks / STAGES) & 1, s_abort)) break;
                 tc_fence_after();
-                const uint64_t bdesc = make_smem_desc(smem_base + s * B_BYTES);
-                const uint32_t a_tm = tmem_d + G4_A_COL0 + s * 32;
+                const uint32_t a_tm = tmem_d + G4_A_COL0 + s * ACOLS;
 #pragma unroll
-                for (int k = 0; k < G_BK / 16; ++k)
-                    umma_f16_ts(tmem_d, a_tm + 8 * k, bdesc + 2 * k, idesc, (kt | k) ? 1u : 0u);
+                for (int j = 0; j < KS; ++j) {
+                    const uint64_t bdesc = make_smem_desc(smem_base + s * STAGE_BYTES + j * B_BYTES);
+#pragma unroll
+                    for (int k = 0; k < G_BK / 16; ++k)
+                        umma_f16_ts(tmem_d, a_tm + 32 * j + 8 * k, bdesc + 2 * k, idesc, (ks | j | k) ? 1u : 0u);
+                }
                 umma_commit(bar_empty(s));
             }
             umma_commit(bar_accum);
@@ -622,35 +631,42 @@ gemm_v16t_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
         if (tab_smem && !mbar_wait(bar_tab, 0, s_abort)) { /* fall through: waits below bail out */ }
         bool ok = true;
         int cur_it = -1;
-        for (int kt = grp; kt < KT && ok; kt += 4) {
-            const int it = kt >> 4, ib = it & 1;
+        for (int ks = grp; ks < NS && ok; ks += 4) {
+            const int kt0 = ks * KS;
+            const int it = kt0 >> 4, ib = it & 1;
             if (it != cur_it) {
                 if (!mbar_wait(bar_full_i(ib), (it >> 1) & 1, s_abort)) { ok = false; break; }
                 cur_it = it;
             }
-            // the four indices of this row's k step: columns (kt % 16) * 4 .. + 3 of the index tile (8 bytes)
-            const int boff = (kt & 15) * 8;
-            const uint2 quad = *reinterpret_cast<const uint2 *>(
-                s_idx + (size_t)ib * G2_IDX_BYTES + (size_t)r * 128 + ((((boff >> 4) & 7) ^ (r & 7)) << 4) + (boff & 15));
-            uint32_t w[4];
-            w[0] = ~(tab_smem ? s_tab[quad.x & 0xffffu] : __ldg(p.tab + (quad.x & 0xffffu)));
-            w[1] = ~(tab_smem ? s_tab[quad.x >> 16] : __ldg(p.tab + (quad.x >> 16)));
-            w[2] = ~(tab_smem ? s_tab[quad.y & 0xffffu] : __ldg(p.tab + (quad.y & 0xffffu)));
-            w[3] = ~(tab_smem ? s_tab[quad.y >> 16] : __ldg(p.tab + (quad.y >> 16)));
-            if (((kt + 4) >> 4) != it || kt + 4 >= KT) {           // this group's last k step in the index tile
+            // the four indices per k step of this row: columns (kt % 16) * 4 .. + 3 of the index tile (8 bytes each)
+            uint32_t w[KS][4];
+#pragma unroll
+            for (int j = 0; j < KS; ++j) {
+                const int boff = ((kt0 + j) & 15) * 8;
+                const uint2 quad = *reinterpret_cast<const uint2 *>(
+                    s_idx + (size_t)ib * G2_IDX_BYTES + (size_t)r * 128 + ((((boff >> 4) & 7) ^ (r & 7)) << 4) + (boff & 15));
+                w[j][0] = ~(tab_smem ? s_tab[quad.x & 0xffffu] : __ldg(p.tab + (quad.x & 0xffffu)));
+                w[j][1] = ~(tab_smem ? s_tab[quad.x >> 16] : __ldg(p.tab + (quad.x >> 16)));
+                w[j][2] = ~(tab_smem ? s_tab[quad.y & 0xffffu] : __ldg(p.tab + (quad.y & 0xffffu)));
+                w[j][3] = ~(tab_smem ? s_tab[quad.y >> 16] : __ldg(p.tab + (quad.y >> 16)));
+            }
+            if ((((ks + 4) * KS) >> 4) != it || ks + 4 >= NS) {     // this group's last stage in the index tile
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar_empty_i(ib));
             }
-            // register j holds the weights 2j, 2j+1 of the k step (K elements 2j, 2j+1 of this row of A)
-            uint32_t regs[32];
-#pragma unroll
-            for (int b = 0; b < 4; ++b)
-#pragma unroll
-                for (int j = 0; j < 8; ++j) regs[8 * b + j] = ((w[b] << (11 - j)) & 0x80008000u) | one2;
-            const int sa = kt % STAGES;
-            if (kt >= STAGES && !mbar_wait(bar_empty(sa), ((kt / STAGES) & 1) ^ 1, s_abort)) { ok = false; break; }
+            const int sa = ks % STAGES;
+            if (ks >= STAGES && !mbar_wait(bar_empty(sa), ((ks / STAGES) & 1) ^ 1, s_abort)) { ok = false; break; }
             tc_fence_after();
-            tmem_st32(tmem_d + lane_base + G4_A_COL0 + sa * 32, regs);
+#pragma unroll
+            for (int j = 0; j < KS; ++j) {
+                // register i holds the weights 2i, 2i+1 of the k step (K elements 2i, 2i+1 of this row of A)
+                uint32_t regs[32];
+#pragma unroll
+                for (int b = 0; b < 4; ++b)
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) regs[8 * b + i] = ((w[j][b] << (11 - i)) & 0x80008000u) | one2;
+                tmem_st32(tmem_d + lane_base + G4_A_COL0 + sa * ACOLS + 32 * j, regs);
+            }
             tmem_st_wait();
             tc_fence_before();
             __syncwarp();
@@ -737,12 +753,12 @@ static int launch_v16(const CUtensorMap &tm, const CUtensorMap &ti, const Gemm2P
     return cuda_check_launch();
 }
 
-template <int BM, int STAGES>
+template <int BM, int STAGES, int KS>
 static int launch_v16t(const CUtensorMap &tm, const CUtensorMap &ti, const Gemm2Params &p, cudaStream_t s)
 {
-    const size_t smem = (size_t)STAGES * (BM * G_BK * 2) + 1024 + 2 * G2_IDX_BYTES + ((p.tab_bytes + 15) & ~15) +
+    const size_t smem = (size_t)STAGES * KS * (BM * G_BK * 2) + 1024 + 2 * G2_IDX_BYTES + ((p.tab_bytes + 15) & ~15) +
                         (2 * STAGES + 6) * 8 + 16;
-    auto kern = gemm_v16t_kernel<BM, STAGES>;
+    auto kern = gemm_v16t_kernel<BM, STAGES, KS>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return cuda_fail(e);
     dim3 grid((p.a.N + G_BN - 1) / G_BN, (p.a.M + BM - 1) / BM);
@@ -805,8 +821,8 @@ int launch_gemm_tcgen05(const LinearArgs &a, cudaStream_t s)
             {   // weights through tensor memory: shared memory holds only x tiles, index tiles and the table
                 const size_t fixed_t = (size_t)(BM == 256 ? 4 : 8) * (BM * G_BK * 2) + 1024 + 2 * G2_IDX_BYTES + 512;
                 q.tab_bytes = (fixed_t + (size_t)Kc4 * 4 <= 227u * 1024u) ? Kc4 * 4 : 0;
-                if (BM == 256) return launch_v16t<256, 4>(tm, ti, q, s);
-                return launch_v16t<128, 8>(tm, ti, q, s);
+                if (BM == 256) return launch_v16t<256, 4, 1>(tm, ti, q, s);
+                return launch_v16t<128, 4, 2>(tm, ti, q, s);
             }
         }
     }
