@@ -75,6 +75,9 @@ struct ImBatch {
     int cost_per, cost_rem;   // the launch's cost line (sum of groups * Kb) cut for the grid: CTA b gets
                               // [per * b + min(b, rem), + per + (b < rem))
     int tab_smem_bytes;       // bytes reserved for the codeword table (0: gather from global memory)
+    int tab_head;             // entries of every table that are staged there; the rest is gathered from global memory
+                              // (L1/L2): a table of 65536 codewords does not fit, and with frequency-ordered codebooks
+                              // the head serves most lookups
     int stages;               // index stages in the ring (2 .. IM_STAGES)
 };
 
@@ -199,7 +202,9 @@ __device__ __forceinline__ void im_group_range(const ImProblem &P, int a0, int a
     hi = min(h, P.groups);
 }
 
-template <int NCLS, int NM, bool TAB_SMEM>
+// TAB_MODE 0: tables gathered from global memory; 1: whole tables in shared memory; 2: the first tab_head entries in
+// shared memory, the rest from global memory.
+template <int NCLS, int NM, int TAB_MODE>
 __global__ void __launch_bounds__(IM_THREADS, 1)
 gemv_imma_kernel(const __grid_constant__ ImBatch batch)
 {
@@ -243,7 +248,8 @@ gemv_imma_kernel(const __grid_constant__ ImBatch batch)
     }
     __syncthreads();
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    constexpr bool tab_smem = TAB_SMEM;                  // codeword table staged in shared memory (else gathered from global)
+    constexpr bool tab_smem = TAB_MODE != 0;             // (part of) the codeword table is staged in shared memory
+    const uint32_t tab_head = (uint32_t)batch.tab_head;
     const int cost_a0 = batch.cost_per * (int)blockIdx.x + min((int)blockIdx.x, batch.cost_rem);
     const int cost_a1 = cost_a0 + batch.cost_per + ((int)blockIdx.x < batch.cost_rem ? 1 : 0);
 
@@ -264,7 +270,7 @@ gemv_imma_kernel(const __grid_constant__ ImBatch batch)
             if (tab_smem) {
                 if (ps > 0 && !im_mbar_wait(bar_tabfree, (ps - 1) & 1, s_abort)) break;
                 if (lane == 0) {
-                    const uint32_t bytes = (uint32_t)((P.Kc + 3) / 4 * 16);
+                    const uint32_t bytes = (uint32_t)(min((P.Kc + 3) / 4 * 4, batch.tab_head) * 4);
                     im_mbar_expect_tx(bar_tabfull, bytes);
                     im_bulk_g2s(im_smem_u32(s_tab), P.tab, bytes, bar_tabfull);
                 }
@@ -583,8 +589,12 @@ gemv_imma_kernel(const __grid_constant__ ImBatch batch)
                                     const uint32_t pa = ia[(e4 + e) >> 1], pb = ib[(e4 + e) >> 1];
                                     const uint32_t i0 = (e & 1) ? (pa >> 16) : (pa & 0xffffu);
                                     const uint32_t i1 = (e & 1) ? (pb >> 16) : (pb & 0xffffu);
-                                    w0[e] = tab_smem ? s_tab[i0] : __ldg(gtab + i0);
-                                    w1[e] = tab_smem ? s_tab[i1] : __ldg(gtab + i1);
+                                    if (TAB_MODE == 1) { w0[e] = s_tab[i0]; w1[e] = s_tab[i1]; }
+                                    else if (TAB_MODE == 0) { w0[e] = __ldg(gtab + i0); w1[e] = __ldg(gtab + i1); }
+                                    else {
+                                        w0[e] = i0 < tab_head ? s_tab[i0] : __ldg(gtab + i0);
+                                        w1[e] = i1 < tab_head ? s_tab[i1] : __ldg(gtab + i1);
+                                    }
                                 }
 #pragma unroll
                                 for (int e = 0; e < 4; ++e) {
@@ -664,7 +674,7 @@ static int im_sm_count()
     return n;
 }
 
-template <int NCLS, int NM, bool TS>
+template <int NCLS, int NM, int TS>
 static int im_launch(ImBatch &b, int groups_total, cudaStream_t s)
 {
     constexpr int TRK = (NM == 1) ? 2 : 1;
@@ -690,7 +700,7 @@ static int im_launch(ImBatch &b, int groups_total, cudaStream_t s)
     return e == cudaSuccess ? BTC_OK : cuda_fail(e);
 }
 
-template <int NCLS, bool TS>
+template <int NCLS, int TS>
 static int im_launch_nm(ImBatch &b, int nm, int groups_total, cudaStream_t s)
 {
     if (nm == 1) return im_launch<NCLS, 1, TS>(b, groups_total, s);
@@ -749,13 +759,28 @@ int launch_gemv_imma(const LinearArgs *problems, int count, cudaStream_t s)
     }
     if (cost >= (1ll << 31)) return BTC_ERR_UNSUPPORTED;
     b.cost_total = (int)cost;
+    // the whole table in shared memory when it fits beside at least four index stages; else as much of its head as fits
+    int mode = 1;
     b.tab_smem_bytes = tab_max;
-    if (im_smem_layout(tab_max, 8 * nm, rows, 2).total > 227u * 1024u) b.tab_smem_bytes = 0;   // gather from global (L1/L2)
+    b.tab_head = tab_max / 4;
+    if (im_smem_layout(tab_max, 8 * nm, rows, 4).total > 227u * 1024u) {
+        mode = 2;
+        int head_bytes = tab_max;
+        while (head_bytes > 0 && im_smem_layout(head_bytes, 8 * nm, rows, 4).total > 227u * 1024u) head_bytes -= 4096;
+        if (head_bytes <= 0) { mode = 0; head_bytes = 0; }
+        b.tab_smem_bytes = head_bytes;
+        b.tab_head = head_bytes / 4;
+    }
     b.stages = IM_STAGES;
     while (b.stages > 2 && im_smem_layout(b.tab_smem_bytes, 8 * nm, rows, b.stages).total > 227u * 1024u) --b.stages;
-    const bool ts = b.tab_smem_bytes > 0;
-    if (ncls_max <= 4) return ts ? im_launch_nm<4, true>(b, nm, groups_total, s) : im_launch_nm<4, false>(b, nm, groups_total, s);
-    return ts ? im_launch_nm<5, true>(b, nm, groups_total, s) : im_launch_nm<5, false>(b, nm, groups_total, s);
+    if (ncls_max <= 4) {
+        if (mode == 1) return im_launch_nm<4, 1>(b, nm, groups_total, s);
+        if (mode == 2) return im_launch_nm<4, 2>(b, nm, groups_total, s);
+        return im_launch_nm<4, 0>(b, nm, groups_total, s);
+    }
+    if (mode == 1) return im_launch_nm<5, 1>(b, nm, groups_total, s);
+    if (mode == 2) return im_launch_nm<5, 2>(b, nm, groups_total, s);
+    return im_launch_nm<5, 0>(b, nm, groups_total, s);
 }
 
 int imma_status_read(int *out)
