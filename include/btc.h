@@ -102,12 +102,14 @@ BTC_API int btc_codebook_pack_host(const int8_t *C_pm1_host, int Kc, int v, uint
  *            256-byte aligned; may be NULL when that function returns 0.  Contents are
  *            undefined afterwards; concurrent calls need distinct workspaces.
  *
- * btc_linear_gemv: the memory-bound decode path, 1 <= M <= 8, fp32 accumulation of the
- *   identity <x, c> = 2 * sum_{bit=1} x - sum x  (or its signed-sum equivalent).
- * btc_linear_gemm: any M >= 1, built for M >= 128: index tiles are decoded to +-1 bf16 tiles in
- *   shared memory and multiplied on the tcgen05 tensor cores with fp32 accumulation in
- *   tensor memory; alpha (and mu) are applied in fp32 in the epilogue.  fp16 x is accepted and
- *   multiplied as fp16.
+ * btc_linear_gemv: the decode path, 1 <= M <= 8, built on the identity <x, c> = 2 * sum_{bit=1} x - sum x.
+ *   M <= 2: x is quantised per K-slice to a block-fixed-point integer (2^-20 of the slice's largest magnitude
+ *   for v = 16), the sums over set bits are exact integer sums on the warp-level int8 MMA, recombined and added
+ *   over the slices in fp32.  M = 3..8: masked codeword bits act as fp16 numbers on the warp-level fp16 MMA with
+ *   fp32 accumulation.  Both stay well inside a relative error of 2e-3 against the exact product.
+ * btc_linear_gemm: any M >= 1, built for M >= 128: index tiles are decoded to +-1 bf16 (fp16 for fp16 x) tiles
+ *   and multiplied on the tcgen05 tensor cores with fp32 accumulation in tensor memory; alpha (and mu) are
+ *   applied in fp32 in the epilogue.  M <= 8 is forwarded to the decode path.
  * Errors: NULL / SHAPE / ALIGN / UNSUPPORTED / WORKSPACE as above; BTC_ERR_CUDA if a launch
  * fails.  Both are asynchronous: a device-side failure shows up at the caller's next sync.
  */

@@ -1,21 +1,22 @@
 // Tensor-core path: y[M,N] = x[M,K] * W^[N,K]^T with W^ = alpha * C[idx] (+ mu), for large M.
 //
-// The contraction runs on the 5th-generation tensor cores (tcgen05.mma, kind::f16, fp32 accumulators
-// in tensor memory).  Roles inside one CTA (one 128 x BM output tile, BM in {128, 256}):
-//   warp 0     TMA producer: x tiles [BM rows x 64 k] -> shared memory (128-byte swizzle)
+// The contraction runs on the 5th-generation tensor cores (tcgen05.mma, kind::f16, fp32 accumulators in tensor
+// memory).  The weight tile is the A operand (128 rows = UMMA M), x is the B operand (BM rows = UMMA N, loaded by TMA
+// with the 128-byte swizzle), so the accumulator holds y^T: tensor-memory lane = output feature n, column = activation
+// row m, and a warp stores 32 consecutive n for one m (coalesced).  The decoded tile is pure +-1 and the row scale is
+// applied in the fp32 epilogue, which is exact for a row-wise alpha.
+//
+// Two kernels: gemm_v16t_kernel (v = 16; decoded weights go straight into tensor memory, see its header) and
+// gemm_tcgen05_kernel (any v; one thread per weight row writes the +-1 tile into shared memory):
+//   warp 0     TMA producer: x tiles [BM rows x 64 k] -> shared memory
 //   warp 1     MMA issuer: one elected thread issues tcgen05.mma for every 64-wide k step
 //   warp 2     allocates / frees tensor memory
-//   warps 4-7  decode producers: thread r expands the indices of weight row n0+r for the current
-//              64-wide k step into +-1 bf16 (or fp16) in the same swizzled K-major layout the MMA
-//              reads (A operand); afterwards the same warps run the epilogue: tcgen05.ld, scale by
-//              alpha_n in fp32 (+ mu_n * sum_k x[m,k]), store y.
-// The weight tile is the A operand (128 rows = UMMA M), x is the B operand (BM rows = UMMA N), so the
-// accumulator holds y^T: tensor-memory lane = output feature n, column = activation row m, and a warp
-// stores 32 consecutive n for one m (coalesced).  Keeping the decoded tile pure +-1 and applying the
-// row scale in the fp32 epilogue is exact for a row-wise alpha.
+//   warps 4-7  decode producers: thread r expands the indices of weight row n0+r for the current 64-wide k step into
+//              +-1 bf16 (or fp16) in the swizzled K-major layout the MMA reads; afterwards the same warps run the
+//              epilogue: tcgen05.ld, scale by alpha_n in fp32 (+ mu_n * sum_k x[m,k]), store y.
 //
-// Every mbarrier wait is bounded: after ~2 s of polling the CTA raises a status word, stops waiting
-// and runs to completion (the output is then undefined and btc_device_status reports the timeout).
+// Every mbarrier wait is bounded: after ~2 s of polling the CTA raises a status word, stops waiting and runs to
+// completion (the output is then undefined and btc_device_status reports the timeout).
 #include <cuda.h>
 #include "btc_internal.cuh"
 
@@ -286,18 +287,12 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_x, const GemmParams
     if (warp == 2) tmem_dealloc(tmem_d, BM);
 }
 
-// ------------------------------------------------------------------------------------ v = 16 kernel
-// Same contraction, faster weight supply, for the common v = 16 (a 64-wide k step is four blocks):
-//   warp 0      TMA producer: x tiles, and index tiles (128 rows x 64 blocks = 16 k steps, 128-byte swizzle);
-//               bulk copy of the codeword table into shared memory
-//   warp 1      MMA issuer          warp 2   tensor-memory allocation
-//   warps 4-19  decode, in GROUPS groups (2 of eight warps with 256-row x tiles, 4 of four warps with 128-row ones)
-//               that take the k steps g, g + GROUPS, ...: a group has GROUPS MMA k steps of time for its lookups,
-//               stores and proxy fence.  A thread expands 2 or 4 blocks of its weight row: table lookups in shared
-//               memory, and per pair of weights one shift and one LOP3 -- the table keeps the bit of weight t at
-//               (t & 1) * 16 + 4 + (t >> 1), so ((~w << (11 - j)) & 0x80008000) | {1.0, 1.0} is the pair
-//               (2j, 2j+1) as +-1 in bf16 / fp16; then the same warps run the epilogue, four per lane quadrant.
-constexpr int G2_DWARPS = 16;                    // decode warps, in GROUPS groups that take the k steps g, g + GROUPS, ...
+// ------------------------------------------------------------------------------------ v = 16: shared declarations
+// For v = 16 a 64-wide k step is four blocks.  The codeword table of the "fp16 layout" keeps the bit of weight t at
+// (t & 1) * 16 + 4 + (t >> 1), so ((~w << (11 - j)) & 0x80008000) | {1.0, 1.0} is the pair of weights (2j, 2j+1) as +-1
+// in bf16 / fp16: one shift and one LOP3 per pair.  Index tiles (128 rows x 64 blocks = 16 k steps, 128-byte swizzle)
+// arrive by TMA; the table is bulk-copied into shared memory when it fits.
+constexpr int G2_DWARPS = 16;                    // decode warps (four groups of four)
 constexpr int G2_THREADS = 128 + G2_DWARPS * 32;
 constexpr uint32_t G2_IDX_BYTES = 128 * 128;     // one index tile
 
@@ -312,189 +307,6 @@ struct Gemm2Params {
 __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar) {
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                  ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
-}
-
-template <int BM, int STAGES, int GROUPS>
-__global__ void __launch_bounds__(G2_THREADS, 1)
-gemm_v16_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_i, const Gemm2Params p)
-{
-    constexpr uint32_t B_BYTES = BM * G_BK * 2;
-    constexpr uint32_t STAGE_BYTES = G_A_BYTES + B_BYTES;
-    extern __shared__ __align__(1024) unsigned char smem_raw[];
-    const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-    unsigned char *smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
-    unsigned char *s_idx = smem_gen + (size_t)STAGES * STAGE_BYTES;                 // 2 index tiles
-    uint32_t *s_tab = reinterpret_cast<uint32_t *>(s_idx + 2 * G2_IDX_BYTES);
-    uint64_t *bars = reinterpret_cast<uint64_t *>(reinterpret_cast<unsigned char *>(s_tab) + ((p.tab_bytes + 15) & ~15));
-    // bars: [0,S) full_x, [S,2S) full_w, [2S,3S) empty, 3S accum, 3S+1.. full_i[2], empty_i[2], tab_full
-    uint32_t *s_tmem = reinterpret_cast<uint32_t *>(bars + 3 * STAGES + 6);
-    volatile int *s_abort = reinterpret_cast<volatile int *>(s_tmem + 1);
-
-    const LinearArgs &a = p.a;
-    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int n0 = blockIdx.x * G_BN, m0 = blockIdx.y * BM;
-    const int KT = p.k_tiles;
-    const bool is_bf16 = (a.x_dt == BTC_BF16);
-    auto bar_full_x = [&](int s) { return smem_u32(bars + s); };
-    auto bar_full_w = [&](int s) { return smem_u32(bars + STAGES + s); };
-    auto bar_empty = [&](int s) { return smem_u32(bars + 2 * STAGES + s); };
-    const uint32_t bar_accum = smem_u32(bars + 3 * STAGES);
-    auto bar_full_i = [&](int b) { return smem_u32(bars + 3 * STAGES + 1 + b); };
-    auto bar_empty_i = [&](int b) { return smem_u32(bars + 3 * STAGES + 3 + b); };
-    const uint32_t bar_tab = smem_u32(bars + 3 * STAGES + 5);
-
-    if (tid == 0) {
-        for (int s = 0; s < STAGES; ++s) {
-            mbar_init(bar_full_x(s), 1);
-            mbar_init(bar_full_w(s), G2_DWARPS / GROUPS);
-            mbar_init(bar_empty(s), 1);
-        }
-        mbar_init(bar_accum, 1);
-        for (int b = 0; b < 2; ++b) { mbar_init(bar_full_i(b), 1); mbar_init(bar_empty_i(b), G2_DWARPS); }
-        mbar_init(bar_tab, 1);
-        *s_abort = 0;
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    }
-    if (warp == 2) tmem_alloc(smem_u32(s_tmem), BM);
-    tc_fence_before();
-    __syncthreads();
-    tc_fence_after();
-    const uint32_t tmem_d = *s_tmem;
-
-    if (warp == 0) {
-        if (lane == 0) {
-            if (p.tab_bytes > 0) {
-                mbar_expect_tx(bar_tab, (uint32_t)p.tab_bytes);
-                bulk_g2s(smem_u32(s_tab), p.tab, (uint32_t)p.tab_bytes, bar_tab);
-            }
-            for (int kt = 0; kt < KT; ++kt) {
-                if ((kt & 15) == 0) {
-                    const int it = kt >> 4, ib = it & 1;
-                    if (it >= 2 && !mbar_wait(bar_empty_i(ib), ((it >> 1) & 1) ^ 1, s_abort)) break;
-                    mbar_expect_tx(bar_full_i(ib), G2_IDX_BYTES);
-                    tma_load_2d(smem_u32(s_idx + (size_t)ib * G2_IDX_BYTES), &tmap_i, it * 64, n0, bar_full_i(ib));
-                }
-                const int s = kt % STAGES;
-                const uint32_t ph = (kt / STAGES) & 1;
-                if (kt >= STAGES && !mbar_wait(bar_empty(s), ph ^ 1, s_abort)) break;
-                mbar_expect_tx(bar_full_x(s), B_BYTES);
-                tma_load_2d(smem_base + s * STAGE_BYTES + G_A_BYTES, &tmap_x, kt * G_BK, m0, bar_full_x(s));
-            }
-        }
-    } else if (warp == 1) {
-        if (lane == 0) {
-            uint32_t idesc = (1u << 4) | ((uint32_t)(BM >> 3) << 17) | ((uint32_t)(G_BN >> 4) << 24);
-            if (is_bf16) idesc |= (1u << 7) | (1u << 10);
-            for (int kt = 0; kt < KT; ++kt) {
-                const int s = kt % STAGES;
-                const uint32_t ph = (kt / STAGES) & 1;
-                if (!mbar_wait<false>(bar_full_x(s), ph, s_abort)) break;
-                if (!mbar_wait<false>(bar_full_w(s), ph, s_abort)) break;
-                tc_fence_after();
-                const uint32_t a_addr = smem_base + s * STAGE_BYTES;
-                const uint64_t adesc = make_smem_desc(a_addr);
-                const uint64_t bdesc = make_smem_desc(a_addr + G_A_BYTES);
-#pragma unroll
-                for (int k = 0; k < G_BK / 16; ++k)
-                    umma_f16(tmem_d, adesc + 2 * k, bdesc + 2 * k, idesc, (kt | k) ? 1u : 0u);
-                umma_commit(bar_empty(s));
-            }
-            umma_commit(bar_accum);
-        }
-    } else if (warp >= 4) {
-        // A stage's barrier phases are waited on by parity, which is only meaningful for the phase right after the
-        // last one a thread has seen.  With GROUPS == STAGES a group always meets the same stage, phase after phase;
-        // with 2 groups and 3 stages a group meets a stage every other phase, one k step of its own in between.
-        static_assert(GROUPS == 2 || GROUPS == STAGES, "a group must see every phase of the stages it writes, or every other");
-        constexpr int GT = G2_DWARPS * 32 / GROUPS;    // threads of a group: 256 or 128
-        constexpr int BPT = 4 * 128 / GT;              // blocks of the k step per thread: 2 or 4
-        const int d = (tid - 128) % GT;                // position in the group
-        const int grp = (tid - 128) / GT;
-        const int r = d & 127, h = d >> 7;             // weight row of the tile, part of the k step
-        const uint32_t one2 = is_bf16 ? 0x3F803F80u : 0x3C003C00u;
-        const bool tab_smem = p.tab_bytes > 0;
-        if (tab_smem && !mbar_wait(bar_tab, 0, s_abort)) { /* fall through: waits below bail out */ }
-        bool ok = true;
-        int cur_it = -1;
-        for (int kt = grp; kt < KT && ok; kt += GROUPS) {
-            const int it = kt >> 4, ib = it & 1;
-            if (it != cur_it) {
-                if (!mbar_wait(bar_full_i(ib), (it >> 1) & 1, s_abort)) { ok = false; break; }
-                cur_it = it;
-            }
-            // indices of blocks h * BPT .. of this k step: columns (kt % 16) * 4 + h * BPT .. of the index tile
-            const int boff = (kt & 15) * 8 + 2 * BPT * h;
-            const unsigned char *ip = s_idx + (size_t)ib * G2_IDX_BYTES + (size_t)r * 128 + ((((boff >> 4) & 7) ^ (r & 7)) << 4) + (boff & 15);
-            uint32_t pairs[BPT / 2];
-            pairs[0] = *reinterpret_cast<const uint32_t *>(ip);
-            if (BPT == 4) pairs[BPT / 2 - 1] = *reinterpret_cast<const uint32_t *>(ip + 4);
-            uint32_t w[BPT];
-#pragma unroll
-            for (int b = 0; b < BPT; ++b) {
-                const uint32_t i = (b & 1) ? (pairs[b >> 1] >> 16) : (pairs[b >> 1] & 0xffffu);
-                w[b] = ~(tab_smem ? s_tab[i] : __ldg(p.tab + i));
-            }
-            if (((kt + GROUPS) >> 4) != it || kt + GROUPS >= KT) {   // this group's last k step in the index tile
-                __syncwarp();
-                if (lane == 0) mbar_arrive(bar_empty_i(ib));
-            }
-            const int s = kt % STAGES;
-            const uint32_t ph = (kt / STAGES) & 1;
-            if (kt >= STAGES && !mbar_wait(bar_empty(s), ph ^ 1, s_abort)) { ok = false; break; }
-            unsigned char *arow = smem_gen + (size_t)s * STAGE_BYTES + (size_t)r * 128;
-#pragma unroll
-            for (int b = 0; b < BPT; ++b) {
-#pragma unroll
-                for (int c = 0; c < 2; ++c) {
-                    uint4 q;
-                    q.x = ((w[b] << (11 - (4 * c + 0))) & 0x80008000u) | one2;
-                    q.y = ((w[b] << (11 - (4 * c + 1))) & 0x80008000u) | one2;
-                    q.z = ((w[b] << (11 - (4 * c + 2))) & 0x80008000u) | one2;
-                    q.w = ((w[b] << (11 - (4 * c + 3))) & 0x80008000u) | one2;
-                    const int chunk = (BPT * h + b) * 2 + c;
-                    *reinterpret_cast<uint4 *>(arow + ((chunk ^ (r & 7)) << 4)) = q;
-                }
-            }
-            fence_proxy_async_smem();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(bar_full_w(s));
-        }
-        // ------------------------------------------------------------ epilogue: four warps per lane quadrant
-        if (ok && mbar_wait(bar_accum, 0, s_abort)) {
-            tc_fence_after();
-            const int wl = warp - 4;
-            const int q4 = wl & 3, quarter = wl >> 2;
-            const int nrow = n0 + q4 * 32 + lane;
-            const int nc = min(nrow, a.N - 1);
-            const float al = __half2float(a.alpha[nc]);
-            const float mu = a.mu ? __half2float(a.mu[nc]) : 0.f;
-            const uint32_t lane_base = (uint32_t)(q4 * 32) << 16;
-#pragma unroll 1
-            for (int c0 = quarter * (BM / 4); c0 < (quarter + 1) * (BM / 4); c0 += 32) {
-                uint32_t rr[32];
-                tmem_ld32(tmem_d + lane_base + c0, rr);
-                tmem_ld_wait();
-                if (nrow < a.N) {
-#pragma unroll
-                    for (int i = 0; i < 32; ++i) {
-                        const int m = m0 + c0 + i;
-                        if (m < a.M) {
-                            float y = al * __uint_as_float(rr[i]);
-                            if (a.mu) y += mu * p.sumx[m];
-                            store_from_float(a.y, a.y_dt, (size_t)m * a.N + nrow, y);
-                        }
-                    }
-                }
-            }
-        }
-    }
-    tc_fence_before();
-    __syncthreads();
-    if (*s_abort) {
-        for (int i = 0; i < 200; ++i) __nanosleep(1000);
-        __syncthreads();
-    }
-    if (warp == 2) tmem_dealloc(tmem_d, BM);
 }
 
 // ------------------------------------------------------------------------------------ v = 16, weights in tensor memory
@@ -740,19 +552,6 @@ static int launch_cfg(const CUtensorMap &tm, const GemmParams &p, cudaStream_t s
     return cuda_check_launch();
 }
 
-template <int BM, int STAGES, int GROUPS>
-static int launch_v16(const CUtensorMap &tm, const CUtensorMap &ti, const Gemm2Params &p, cudaStream_t s)
-{
-    const size_t smem = (size_t)STAGES * (G_A_BYTES + BM * G_BK * 2) + 1024 + 2 * G2_IDX_BYTES + ((p.tab_bytes + 15) & ~15) +
-                        (3 * STAGES + 6) * 8 + 16;
-    auto kern = gemm_v16_kernel<BM, STAGES, GROUPS>;
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return cuda_fail(e);
-    dim3 grid((p.a.N + G_BN - 1) / G_BN, (p.a.M + BM - 1) / BM);
-    kern<<<grid, G2_THREADS, smem, s>>>(tm, ti, p);
-    return cuda_check_launch();
-}
-
 template <int BM, int STAGES, int KS>
 static int launch_v16t(const CUtensorMap &tm, const CUtensorMap &ti, const Gemm2Params &p, cudaStream_t s)
 {
@@ -802,7 +601,7 @@ int launch_gemm_tcgen05(const LinearArgs &a, cudaStream_t s)
         p.sumx = sx;
     }
     if (a.v == 16 && a.Kb % 8 == 0) {
-        // v = 16 kernel: index tiles by TMA, table in shared memory when it fits
+        // v = 16: index tiles by TMA, table in shared memory when it fits, weights through tensor memory
         CUtensorMap ti;
         const cuuint64_t idims[2] = {(cuuint64_t)a.Kb, (cuuint64_t)a.N};
         const cuuint64_t istr[1] = {(cuuint64_t)a.Kb * 2};
@@ -814,16 +613,11 @@ int launch_gemm_tcgen05(const LinearArgs &a, cudaStream_t s)
             q.a = a; q.sumx = p.sumx; q.k_tiles = p.k_tiles;
             const int Kc4 = (a.Kc + 3) / 4 * 4;
             q.tab = a.Cp + Kc4;
-            // the table is staged in shared memory when it fits beside the pipeline stages (227 KB per CTA)
-            const size_t fixed = (BM == 256 ? 3 * (G_A_BYTES + 256 * G_BK * 2) : 4 * (G_A_BYTES + 128 * G_BK * 2)) + 1024 +
-                                 2 * G2_IDX_BYTES + 256;
-            q.tab_bytes = (fixed + (size_t)Kc4 * 4 <= 227u * 1024u) ? Kc4 * 4 : 0;
-            {   // weights through tensor memory: shared memory holds only x tiles, index tiles and the table
-                const size_t fixed_t = (size_t)(BM == 256 ? 4 : 8) * (BM * G_BK * 2) + 1024 + 2 * G2_IDX_BYTES + 512;
-                q.tab_bytes = (fixed_t + (size_t)Kc4 * 4 <= 227u * 1024u) ? Kc4 * 4 : 0;
-                if (BM == 256) return launch_v16t<256, 4, 1>(tm, ti, q, s);
-                return launch_v16t<128, 4, 2>(tm, ti, q, s);
-            }
+            // shared memory holds only x tiles (4 stages of 32 KB either way), index tiles and the table
+            const size_t fixed_t = (size_t)4 * (256 * G_BK * 2) + 1024 + 2 * G2_IDX_BYTES + 512;
+            q.tab_bytes = (fixed_t + (size_t)Kc4 * 4 <= 227u * 1024u) ? Kc4 * 4 : 0;
+            if (BM == 256) return launch_v16t<256, 4, 1>(tm, ti, q, s);
+            return launch_v16t<128, 4, 2>(tm, ti, q, s);
         }
     }
     if (BM == 256) return launch_cfg<256, 4>(tm, p, s);
