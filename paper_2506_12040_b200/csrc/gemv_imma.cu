@@ -663,6 +663,34 @@ static im_encode_fn im_get_encode()
     return fn;
 }
 
+// Tensor map of an index matrix {K/v, N} (16-bit words), box {64, rows}, 128-byte swizzle.  Encoding goes through the
+// driver and costs about a microsecond; a decode step re-uses the same matrices call after call, so the last few
+// maps are kept per host thread, keyed by everything the encoding depends on.
+static bool im_tensor_map(im_encode_fn enc, const uint16_t *idx, int Kb, int N, int rows, CUtensorMap *out)
+{
+    struct Entry { const uint16_t *idx; int Kb, N, rows; CUtensorMap map; };
+    constexpr int SLOTS = 64;
+    thread_local Entry cache[SLOTS];
+    thread_local int used = 0, next = 0;
+    for (int i = 0; i < used; ++i)
+        if (cache[i].idx == idx && cache[i].Kb == Kb && cache[i].N == N && cache[i].rows == rows) { *out = cache[i].map; return true; }
+    const cuuint64_t dims[2] = {(cuuint64_t)Kb, (cuuint64_t)N};
+    const cuuint64_t strides[1] = {(cuuint64_t)Kb * 2};
+    const cuuint32_t box[2] = {(cuuint32_t)IM_BOX_COLS, (cuuint32_t)rows};
+    const cuuint32_t estr[2] = {1, 1};
+    CUtensorMap m;
+    if (enc(&m, CU_TENSOR_MAP_DATA_TYPE_UINT16, 2, const_cast<uint16_t *>(idx), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+        return false;
+    Entry &e = cache[next];
+    e.idx = idx; e.Kb = Kb; e.N = N; e.rows = rows; e.map = m;
+    next = (next + 1) % SLOTS;
+    if (used < SLOTS) ++used;
+    *out = m;
+    return true;
+}
+
 static int im_sm_count()
 {
     static int n = 0;
@@ -737,16 +765,8 @@ int launch_gemv_imma(const LinearArgs *problems, int count, cudaStream_t s)
         p.parts = (a.Kb + IM_PW - 1) / IM_PW;
         p.groups = (a.N + rows - 1) / rows;
         p.ncls = a.v / 4;
-        {
-            const cuuint64_t dims[2] = {(cuuint64_t)a.Kb, (cuuint64_t)a.N};
-            const cuuint64_t strides[1] = {(cuuint64_t)a.Kb * 2};
-            const cuuint32_t box[2] = {(cuuint32_t)IM_BOX_COLS, (cuuint32_t)rows};
-            const cuuint32_t estr[2] = {1, 1};
-            if (enc(&b.map[i], CU_TENSOR_MAP_DATA_TYPE_UINT16, 2, const_cast<uint16_t *>(a.idx), dims, strides, box, estr,
-                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
-                return BTC_ERR_UNSUPPORTED;                 // shape the tensor map cannot describe: other kernels take it
-        }
+        if (!im_tensor_map(enc, a.idx, a.Kb, a.N, rows, &b.map[i]))
+            return BTC_ERR_UNSUPPORTED;                     // shape the tensor map cannot describe: other kernels take it
         p.cost_base = (int)cost;
         // measured: an iteration (one row group x one part of up to 256 blocks) costs about the same whatever the
         // part's width, and rebuilding the activation fragments for a part costs ~1.5 iterations, shared by the
