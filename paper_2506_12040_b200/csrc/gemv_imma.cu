@@ -64,16 +64,14 @@ struct ImProblem {
     int groups;               // row groups: ceil(N / (16 * TRK))
     int ncls;                 // v / 4
     int cost;                 // cost of one row group (blocks, plus the per-part fragment rebuild; see launch_gemv_imma)
-    int cost_base;            // sum over earlier layers of groups * cost
+    int cta_begin, cta_count; // the CTAs that work on this layer (no CTA works on two layers: each switch would cost a
+                              // table load and a fragment rebuild, and the slowest CTA sets the launch's time)
 };
 
 struct ImBatch {
     CUtensorMap map[IM_MAXP]; // idx of each layer as a 2-D tensor {K/v, N} of 16-bit words, box {64, rows}, 128-byte swizzle
     ImProblem p[IM_MAXP];
     int count;
-    int cost_total;           // sum over layers of groups * Kb (host bookkeeping)
-    int cost_per, cost_rem;   // the launch's cost line (sum of groups * Kb) cut for the grid: CTA b gets
-                              // [per * b + min(b, rem), + per + (b < rem))
     int tab_smem_bytes;       // bytes reserved for the codeword table (0: gather from global memory)
     int tab_head;             // entries of every table that are staged there; the rest is gathered from global memory
                               // (L1/L2): a table of 65536 codewords does not fit, and with frequency-ordered codebooks
@@ -189,17 +187,14 @@ __host__ __device__ inline ImSmem im_smem_layout(int tab_bytes, int cols, int ro
     return L;
 }
 
-// Row groups [lo, hi) of layer P that fall to this CTA: the launch's work is laid on a line (a row
-// group of a layer costs its Kb), cut into one stretch [a0, a1) per CTA; a row group belongs to the
-// stretch its first point lies in.
-__device__ __forceinline__ void im_group_range(const ImProblem &P, int a0, int a1, int &lo, int &hi)
+// Row groups [lo, hi) of layer P that fall to CTA b: the layer's cta_count CTAs split its row groups evenly.
+__device__ __forceinline__ void im_group_range(const ImProblem &P, int b, int &lo, int &hi)
 {
     lo = hi = 0;
-    if (a1 <= P.cost_base || a0 >= P.cost_base + P.groups * P.cost) return;     // (no division for layers of other CTAs)
-    const int l = (a0 <= P.cost_base) ? 0 : (a0 - P.cost_base + P.cost - 1) / P.cost;
-    const int h = (a1 - P.cost_base + P.cost - 1) / P.cost;
-    lo = min(l, P.groups);
-    hi = min(h, P.groups);
+    const int r = b - P.cta_begin;
+    if (r < 0 || r >= P.cta_count) return;
+    lo = (int)((long long)P.groups * r / P.cta_count);
+    hi = (int)((long long)P.groups * (r + 1) / P.cta_count);
 }
 
 // TAB_MODE 0: tables gathered from global memory; 1: whole tables in shared memory; 2: the first tab_head entries in
@@ -250,8 +245,6 @@ gemv_imma_kernel(const __grid_constant__ ImBatch batch)
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     constexpr bool tab_smem = TAB_MODE != 0;             // (part of) the codeword table is staged in shared memory
     const uint32_t tab_head = (uint32_t)batch.tab_head;
-    const int cost_a0 = batch.cost_per * (int)blockIdx.x + min((int)blockIdx.x, batch.cost_rem);
-    const int cost_a1 = cost_a0 + batch.cost_per + ((int)blockIdx.x < batch.cost_rem ? 1 : 0);
 
     // All three roles walk the same sequence: layers pi (those with row groups for this CTA, counted
     // by ps), chunks [c0, c1) of at most IM_RC row groups, K-parts j (counted by pc), row groups r; li
@@ -265,7 +258,7 @@ gemv_imma_kernel(const __grid_constant__ ImBatch batch)
         for (int pi = 0; pi < batch.count && ok; ++pi) {
             const ImProblem &P = batch.p[pi];
             int glo, ghi;
-            im_group_range(P, cost_a0, cost_a1, glo, ghi);
+            im_group_range(P, (int)blockIdx.x, glo, ghi);
             if (glo >= ghi) continue;
             if (tab_smem) {
                 if (ps > 0 && !im_mbar_wait(bar_tabfree, (ps - 1) & 1, s_abort)) break;
@@ -308,7 +301,7 @@ gemv_imma_kernel(const __grid_constant__ ImBatch batch)
         for (int pi = 0; pi < batch.count && ok; ++pi) {
             const ImProblem &P = batch.p[pi];
             int glo, ghi;
-            im_group_range(P, cost_a0, cost_a1, glo, ghi);
+            im_group_range(P, (int)blockIdx.x, glo, ghi);
             if (glo >= ghi) continue;
             const float unshift2 = 2.0f / (float)(1 << (P.ncls - 1));
             for (int c0 = glo; c0 < ghi && ok; c0 += IM_RC) {
@@ -414,7 +407,7 @@ gemv_imma_kernel(const __grid_constant__ ImBatch batch)
         for (int pi = 0; pi < batch.count && ok; ++pi) {
             const ImProblem &P = batch.p[pi];
             int glo, ghi;
-            im_group_range(P, cost_a0, cost_a1, glo, ghi);
+            im_group_range(P, (int)blockIdx.x, glo, ghi);
             if (glo >= ghi) continue;
             const int M = P.M, K = P.K, Kb = P.Kb, v = P.v;
             const int cmax = P.ncls - 1;
@@ -702,6 +695,40 @@ static int im_sm_count()
     return n;
 }
 
+// Gives every layer a whole number of CTAs in proportion to its work (row groups x cost per row group), at least one
+// and at most one per row group, and returns the grid size.
+static int im_assign_ctas(ImBatch &b, int budget)
+{
+    double work[IM_MAXP], total = 0.0;
+    for (int i = 0; i < b.count; ++i) { work[i] = (double)b.p[i].groups * b.p[i].cost; total += work[i]; }
+    int sum = 0;
+    for (int i = 0; i < b.count; ++i) {
+        int c = (int)(budget * work[i] / total);
+        c = c < 1 ? 1 : (c > b.p[i].groups ? b.p[i].groups : c);
+        b.p[i].cta_count = c;
+        sum += c;
+    }
+    while (sum < budget) {                          // spare CTAs go where the load per CTA is highest
+        int best = -1;
+        for (int i = 0; i < b.count; ++i)
+            if (b.p[i].cta_count < b.p[i].groups &&
+                (best < 0 || work[i] / b.p[i].cta_count > work[best] / b.p[best].cta_count)) best = i;
+        if (best < 0) break;
+        ++b.p[best].cta_count; ++sum;
+    }
+    while (sum > budget) {                          // (only when the floor of one CTA per layer overshoots)
+        int best = -1;
+        for (int i = 0; i < b.count; ++i)
+            if (b.p[i].cta_count > 1 &&
+                (best < 0 || work[i] / (b.p[i].cta_count - 1) < work[best] / (b.p[best].cta_count - 1))) best = i;
+        if (best < 0) break;
+        --b.p[best].cta_count; --sum;
+    }
+    int begin = 0;
+    for (int i = 0; i < b.count; ++i) { b.p[i].cta_begin = begin; begin += b.p[i].cta_count; }
+    return begin;
+}
+
 template <int NCLS, int NM, int TS>
 static int im_launch(ImBatch &b, int groups_total, cudaStream_t s)
 {
@@ -712,9 +739,7 @@ static int im_launch(ImBatch &b, int groups_total, cudaStream_t s)
     if (e != cudaSuccess) return cuda_fail(e);
     cudaLaunchConfig_t cfg = {};
     const int sms = im_sm_count();
-    const int grid = groups_total < sms ? groups_total : sms;
-    b.cost_per = b.cost_total / grid;
-    b.cost_rem = b.cost_total % grid;
+    const int grid = im_assign_ctas(b, groups_total < sms ? groups_total : sms);
     cfg.gridDim = dim3((unsigned)grid);
     cfg.blockDim = dim3(IM_THREADS);
     cfg.dynamicSmemBytes = L.total;
@@ -752,7 +777,6 @@ int launch_gemv_imma(const LinearArgs *problems, int count, cudaStream_t s)
     }
     const int nm = m_max <= 2 ? 1 : (m_max <= 5 ? 2 : 3);
     const int rows = (nm == 1) ? 32 : 16;
-    long long cost = 0;                              // must stay below 2^31
     int groups_total = 0;
     for (int i = 0; i < count; ++i) {
         const LinearArgs &a = problems[i];
@@ -767,18 +791,14 @@ int launch_gemv_imma(const LinearArgs *problems, int count, cudaStream_t s)
         p.ncls = a.v / 4;
         if (!im_tensor_map(enc, a.idx, a.Kb, a.N, rows, &b.map[i]))
             return BTC_ERR_UNSUPPORTED;                     // shape the tensor map cannot describe: other kernels take it
-        p.cost_base = (int)cost;
         // measured: an iteration (one row group x one part of up to 256 blocks) costs about the same whatever the
         // part's width, and rebuilding the activation fragments for a part costs ~1.5 iterations, shared by the
         // (few) row groups a CTA walks with it; a single-part layer rebuilds only once per CTA
         p.cost = p.parts > 1 ? p.parts * (IM_PW + 110) : a.Kb + 40;
-        cost += (long long)p.groups * p.cost;
         groups_total += p.groups;
         if (p.ncls > ncls_max) ncls_max = p.ncls;
         if (Kc4 * 4 > tab_max) tab_max = Kc4 * 4;
     }
-    if (cost >= (1ll << 31)) return BTC_ERR_UNSUPPORTED;
-    b.cost_total = (int)cost;
     // the whole table in shared memory when it fits beside at least four index stages; else as much of its head as fits
     int mode = 1;
     b.tab_smem_bytes = tab_max;
