@@ -695,37 +695,36 @@ static int im_sm_count()
     return n;
 }
 
-// Gives every layer a whole number of CTAs in proportion to its work (row groups x cost per row group), at least one
-// and at most one per row group, and returns the grid size.
+// Gives every layer a whole number of CTAs so that the largest load of any CTA -- ceil(groups / CTAs) row groups times
+// the layer's cost per row group; row groups are not divisible -- is as small as the budget allows, and returns the
+// grid size.  Smallest feasible load by bisection; a load T needs ceil(groups / floor(T / cost)) CTAs of a layer.
 static int im_assign_ctas(ImBatch &b, int budget)
 {
-    double work[IM_MAXP], total = 0.0;
-    for (int i = 0; i < b.count; ++i) { work[i] = (double)b.p[i].groups * b.p[i].cost; total += work[i]; }
-    int sum = 0;
+    auto ctas_needed = [&](long long T) {
+        long long sum = 0;
+        for (int i = 0; i < b.count; ++i) {
+            const long long per = T / b.p[i].cost;                    // row groups one CTA may take
+            if (per < 1) return (long long)1 << 40;
+            sum += (b.p[i].groups + per - 1) / per;
+        }
+        return sum;
+    };
+    long long lo = 1, hi = 0;
     for (int i = 0; i < b.count; ++i) {
-        int c = (int)(budget * work[i] / total);
-        c = c < 1 ? 1 : (c > b.p[i].groups ? b.p[i].groups : c);
-        b.p[i].cta_count = c;
-        sum += c;
+        const long long all = (long long)b.p[i].groups * b.p[i].cost;
+        if (all > hi) hi = all;                                       // one CTA per layer always fits (budget >= count)
     }
-    while (sum < budget) {                          // spare CTAs go where the load per CTA is highest
-        int best = -1;
-        for (int i = 0; i < b.count; ++i)
-            if (b.p[i].cta_count < b.p[i].groups &&
-                (best < 0 || work[i] / b.p[i].cta_count > work[best] / b.p[best].cta_count)) best = i;
-        if (best < 0) break;
-        ++b.p[best].cta_count; ++sum;
-    }
-    while (sum > budget) {                          // (only when the floor of one CTA per layer overshoots)
-        int best = -1;
-        for (int i = 0; i < b.count; ++i)
-            if (b.p[i].cta_count > 1 &&
-                (best < 0 || work[i] / (b.p[i].cta_count - 1) < work[best] / (b.p[best].cta_count - 1))) best = i;
-        if (best < 0) break;
-        --b.p[best].cta_count; --sum;
+    while (lo < hi) {
+        const long long mid = (lo + hi) / 2;
+        if (ctas_needed(mid) <= budget) hi = mid; else lo = mid + 1;
     }
     int begin = 0;
-    for (int i = 0; i < b.count; ++i) { b.p[i].cta_begin = begin; begin += b.p[i].cta_count; }
+    for (int i = 0; i < b.count; ++i) {
+        const long long per = lo / b.p[i].cost;
+        b.p[i].cta_count = (int)((b.p[i].groups + per - 1) / per);
+        b.p[i].cta_begin = begin;
+        begin += b.p[i].cta_count;
+    }
     return begin;
 }
 
