@@ -543,12 +543,12 @@ gemv_imma_kernel(const __grid_constant__ ImBatch batch)
                     }
 
                     // ---- the row groups of the chunk, for this part
-                    for (int r = c0; r < c1; ++r, ++li) {
-                        if (!im_mbar_wait(bar_full(s), rph, s_abort)) { ok = false; break; }
+                    // Loads this lane's indices of the next row group from the ring (tile rows sg and sg + 8 of tile rh;
+                    // 128-byte swizzle: 16-byte chunk c of row q sits at chunk c ^ (q & 7)) and frees the stage.
+                    uint32_t ia[BPL / 2], ib[BPL / 2];
+                    auto load_indices = [&]() -> bool {
+                        if (!im_mbar_wait(bar_full(s), rph, s_abort)) return false;
                         const unsigned char *stage = s_ring + (size_t)s * IM_STAGE_BYTES;
-                        // indices of this lane's BPL blocks, tile rows sg and sg + 8 of tile rh (128-byte swizzle:
-                        // 16-byte chunk c of row q sits at chunk c ^ (q & 7))
-                        uint32_t ia[BPL / 2], ib[BPL / 2];
 #pragma unroll
                         for (int i = 0; i < BPL / 2; ++i) { ia[i] = 0u; ib[i] = 0u; }
                         if (wvalid) {
@@ -567,7 +567,10 @@ gemv_imma_kernel(const __grid_constant__ ImBatch batch)
                         __syncwarp();
                         if (lane == 0) im_mbar_arrive(bar_empty(s));
                         if (++s == NST) { s = 0; rph ^= 1u; }
-
+                        return true;
+                    };
+                    if (!load_indices()) { ok = false; break; }
+                    for (int r = c0; r < c1; ++r, ++li) {
                         int acc[NM][4], acc2[NM][4];                 // two chains: an MMA need not wait for the previous one
 #pragma unroll
                         for (int nm = 0; nm < NM; ++nm)
@@ -611,6 +614,9 @@ gemv_imma_kernel(const __grid_constant__ ImBatch batch)
                                 }
                             }
                         }
+                        // the next row group's indices are fetched while this one's MMAs drain (their codewords are in
+                        // registers by now), so the barrier round trip is off the critical path
+                        if (r + 1 < c1 && !load_indices()) { ok = false; break; }
 #pragma unroll
                         for (int nm = 0; nm < NM; ++nm)
 #pragma unroll
