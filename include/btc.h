@@ -196,6 +196,13 @@ BTC_API int btc_validate_indices(const uint16_t *idx, size_t count, int Kc, int 
  * BTC_ERR_TIMEOUT if a bounded wait inside a tensor-core kernel ran out since the library was
  * loaded (the output of that launch is undefined).  This helper SYNCHRONISES the device. */
 BTC_API int btc_device_status(int *status_host);
+/* Clears the status word (SYNCHRONISES the device).  Host bookkeeping, no counterpart in the paper. */
+BTC_API int btc_device_status_reset(void);
+/* Failure-detection self-test (no counterpart in the paper): launches one warp that waits, with a limit of about a
+ * millisecond, on a barrier nothing will ever arrive on.  The wait must give up, raise the status word
+ * (btc_device_status then reports BTC_ERR_TIMEOUT) and let the kernel return, leaving the context usable: the same
+ * path every bounded wait of the linear kernels takes when its partner is lost.  Asynchronous like the other calls. */
+BTC_API int btc_selftest_bounded_wait(void *stream);
 
 /* Bits per weight.  mode 0: log2(Kc)/v; 1: ceil(log2 Kc)/v (the paper's accounting, Section 4.3);
  * 2: 16/v (uint16 containers as stored here).  Adds scale_bits_per_row/K, and v*Kc/(N*K) for the

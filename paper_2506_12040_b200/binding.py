@@ -20,7 +20,7 @@ _DT = {torch.float16: BTC_F16, torch.bfloat16: BTC_BF16, torch.float32: BTC_F32}
 EXPORTS = (
     "btc_version", "btc_status_string", "btc_last_cuda_error", "btc_codebook_packed_bytes",
     "btc_codebook_pack", "btc_codebook_pack_host", "btc_linear_workspace_bytes", "btc_linear_gemv",
-    "btc_linear_gemm", "btc_linear_gemv_batch", "btc_linear_gemm_static_scratch", "btc_decode_pm1", "btc_validate_indices", "btc_bits_per_weight", "btc_device_status",
+    "btc_linear_gemm", "btc_linear_gemv_batch", "btc_linear_gemm_static_scratch", "btc_decode_pm1", "btc_validate_indices", "btc_bits_per_weight", "btc_device_status", "btc_device_status_reset", "btc_selftest_bounded_wait",
 )
 
 
@@ -71,6 +71,7 @@ def _load() -> ctypes.CDLL:
     L.btc_decode_pm1.argtypes = [vp, vp, ci, ci, ci, ci, vp, vp]
     L.btc_validate_indices.argtypes = [vp, sz, ci, vp, vp]
     L.btc_device_status.argtypes = [ctypes.POINTER(ctypes.c_int)]
+    L.btc_selftest_bounded_wait.argtypes = [vp]
     L.btc_bits_per_weight.restype = ctypes.c_double
     L.btc_bits_per_weight.argtypes = [ci] * 7
     return L
@@ -289,6 +290,19 @@ def device_status() -> int:
     if st:
         raise BtcError(st, "btc_device_status")
     return int(out.value)
+
+
+def device_status_reset() -> None:
+    st = lib.btc_device_status_reset()
+    if st:
+        raise BtcError(st, "btc_device_status_reset")
+
+
+def selftest_bounded_wait() -> None:
+    """Launches the bounded-wait self-test on the current stream (see btc_selftest_bounded_wait)."""
+    st = lib.btc_selftest_bounded_wait(_stream())
+    if st:
+        raise BtcError(st, "btc_selftest_bounded_wait")
 
 
 def bits_per_weight(N, K, v, Kc, scale_bits_per_row=0, mode="container", with_codebook=False) -> float:

@@ -45,6 +45,8 @@ size_t gemm_tcgen05_workspace_bytes(int M, int N, int K, int v, int Kc);
 constexpr int IM_MAXP = 8;
 int launch_gemv_imma(const LinearArgs *problems, int count, cudaStream_t s);
 int imma_status_read(int *out);
+int imma_status_reset();
+int imma_selftest_wait(cudaStream_t s);
 
 // transform.cu: x' = x * D * (P1 (x) P2) into xt (same dtype/shape as x).
 int launch_transform(const void *x, int x_dt, const btc_transform &T, void *xt, int M, int K,

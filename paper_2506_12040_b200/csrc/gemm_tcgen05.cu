@@ -626,6 +626,19 @@ int launch_gemm_tcgen05(const LinearArgs &a, cudaStream_t s)
 
 }  // namespace btc
 
+extern "C" BTC_API int btc_device_status_reset(void)
+{
+    const int zero = 0;
+    cudaError_t e = cudaMemcpyToSymbol(btc::g_gemm_status, &zero, sizeof(int));
+    if (e != cudaSuccess) return btc::cuda_fail(e);
+    return btc::imma_status_reset();
+}
+
+extern "C" BTC_API int btc_selftest_bounded_wait(void *stream)
+{
+    return btc::imma_selftest_wait((cudaStream_t)stream);
+}
+
 extern "C" BTC_API int btc_device_status(int *status_host)
 {
     if (!status_host) return BTC_ERR_NULL;

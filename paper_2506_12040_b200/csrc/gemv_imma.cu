@@ -101,7 +101,8 @@ __device__ __forceinline__ bool im_mbar_try(uint32_t bar, uint32_t parity) {
 }
 // Bounded wait: false (and the CTA-wide abort flag latched) once ~1 s has passed.  A waiting warp backs off with
 // nanosleep so that it does not take issue slots from the warps it is waiting for.
-__device__ __forceinline__ bool im_mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag) {
+__device__ __forceinline__ bool im_mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag,
+                                             long long limit_clk = 2000000000LL) {
     if (im_mbar_try(bar, parity)) return true;
     const long long t0 = clock64();
     int spins = 0;
@@ -109,7 +110,7 @@ __device__ __forceinline__ bool im_mbar_wait(uint32_t bar, uint32_t parity, vola
         __nanosleep(spins < 4 ? 20 : 100);
         if ((++spins & 255) == 0) {
             if (*abort_flag) return false;
-            if (clock64() - t0 > 2000000000LL) {
+            if (clock64() - t0 > limit_clk) {
                 *abort_flag = 1;
                 atomicExch(&g_imma_status, (int)BTC_ERR_TIMEOUT);
                 return false;
@@ -826,6 +827,34 @@ int launch_gemv_imma(const LinearArgs *problems, int count, cudaStream_t s)
     if (mode == 1) return im_launch_nm<5, 1>(b, nm, groups_total, s);
     if (mode == 2) return im_launch_nm<5, 2>(b, nm, groups_total, s);
     return im_launch_nm<5, 0>(b, nm, groups_total, s);
+}
+
+// Self-test of the bounded wait: one warp waits (with a ~1 ms limit) on a barrier that nothing ever arrives on, which
+// must raise the status word and return -- the same code path a lost producer or consumer would take in the kernels.
+__global__ void im_selftest_wait_kernel()
+{
+    __shared__ uint64_t bar;
+    __shared__ int abort_flag;
+    if (threadIdx.x == 0) {
+        im_mbar_init(im_smem_u32(&bar), 1);
+        abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    (void)im_mbar_wait(im_smem_u32(&bar), 0, &abort_flag, 2000000LL);
+}
+
+int imma_selftest_wait(cudaStream_t s)
+{
+    im_selftest_wait_kernel<<<1, 32, 0, s>>>();
+    return cuda_check_launch();
+}
+
+int imma_status_reset()
+{
+    const int zero = 0;
+    cudaError_t e = cudaMemcpyToSymbol(g_imma_status, &zero, sizeof(int));
+    return e == cudaSuccess ? BTC_OK : cuda_fail(e);
 }
 
 int imma_status_read(int *out)

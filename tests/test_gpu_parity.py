@@ -289,3 +289,20 @@ def test_gemm_many_tiles_ragged_shapes():
     rel, fwd = errors(y[torch.from_numpy(rows).cuda()], oracle_y(sub), sub)
     assert rel <= TOL_GEMM and fwd <= TOL_GEMM, (rel, fwd)
     assert bool(torch.isfinite(y).all()) and btc.device_status() == 0
+
+
+# ------------------------------------------------------------------ failure detection without a GPU fault
+
+def test_bounded_wait_gives_up_and_context_stays_usable():
+    """A wait whose partner never arrives must run out (about a millisecond here), raise the status word and return;
+    afterwards the status can be cleared and the kernels still work."""
+    assert btc.device_status() == 0
+    btc.selftest_bounded_wait()
+    torch.cuda.synchronize()
+    assert btc.device_status() == 7          # BTC_ERR_TIMEOUT
+    btc.device_status_reset()
+    assert btc.device_status() == 0
+    L = wl.make_layer(_spec(272, 1024, 16, 4096), 1, seed=2)
+    y, _ = run_layer(L, "gemv")
+    rel, fwd = errors(y, oracle_y(L), L)
+    assert rel <= TOL_GEMV and fwd <= TOL_GEMV and btc.device_status() == 0
