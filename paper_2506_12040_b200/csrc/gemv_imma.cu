@@ -627,8 +627,10 @@ gemv_imma_kernel(const __grid_constant__ ImBatch batch)
                         int *mine = s_part + ((size_t)buf * IM_CWARPS + warp) * TILE_INTS;
 #pragma unroll
                         for (int nm = 0; nm < NM; ++nm) {
-                            *reinterpret_cast<int2 *>(mine + sg * COLS + nm * 8 + 2 * t) = make_int2(acc[nm][0], acc[nm][1]);
-                            *reinterpret_cast<int2 *>(mine + (sg + 8) * COLS + nm * 8 + 2 * t) = make_int2(acc[nm][2], acc[nm][3]);
+                            if (nm * 8 + 2 * t < 3 * M) {               // columns 3 m + d, m < M: the others are never read
+                                *reinterpret_cast<int2 *>(mine + sg * COLS + nm * 8 + 2 * t) = make_int2(acc[nm][0], acc[nm][1]);
+                                *reinterpret_cast<int2 *>(mine + (sg + 8) * COLS + nm * 8 + 2 * t) = make_int2(acc[nm][2], acc[nm][3]);
+                            }
                         }
                         __syncwarp();
                         if (lane == 0) im_mbar_arrive(bar_pfull(buf));
