@@ -727,13 +727,23 @@ static int im_assign_ctas(ImBatch &b, int budget)
         const long long mid = (lo + hi) / 2;
         if (ctas_needed(mid) <= budget) hi = mid; else lo = mid + 1;
     }
-    int begin = 0;
+    int sum = 0;
     for (int i = 0; i < b.count; ++i) {
         const long long per = lo / b.p[i].cost;
         b.p[i].cta_count = (int)((b.p[i].groups + per - 1) / per);
-        b.p[i].cta_begin = begin;
-        begin += b.p[i].cta_count;
+        sum += b.p[i].cta_count;
     }
+    while (sum < budget) {                          // spare CTAs: more SMs streaming, where the average load is highest
+        int best = -1;
+        for (int i = 0; i < b.count; ++i)
+            if (b.p[i].cta_count < b.p[i].groups &&
+                (best < 0 || (double)b.p[i].groups * b.p[i].cost / b.p[i].cta_count >
+                                 (double)b.p[best].groups * b.p[best].cost / b.p[best].cta_count)) best = i;
+        if (best < 0) break;
+        ++b.p[best].cta_count; ++sum;
+    }
+    int begin = 0;
+    for (int i = 0; i < b.count; ++i) { b.p[i].cta_begin = begin; begin += b.p[i].cta_count; }
     return begin;
 }
 
