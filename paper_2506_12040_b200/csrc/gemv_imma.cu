@@ -389,7 +389,6 @@ gemv_imma_kernel(const __grid_constant__ ImBatch batch)
     } else {
         // ============================================================ compute warps
         const int g = lane >> 2, t = lane & 3;
-        constexpr int CT = IM_CWARPS * 32;
         constexpr float MAGIC = 12582912.0f;                   // 1.5 * 2^23: float -> int by addition
         constexpr int MAGIC_BITS = 0x4B400000;
         const int ks = warp % KS, rh = warp / KS;             // K-slice and tile of this warp
