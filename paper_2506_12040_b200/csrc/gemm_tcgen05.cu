@@ -349,7 +349,11 @@ gemm_v16t_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
     constexpr uint32_t B_BYTES = BM * G_BK * 2;                    // one x tile (64 k); a stage holds KS of them
     constexpr uint32_t STAGE_BYTES = KS * B_BYTES;
     constexpr int ACOLS = 32 * KS;                                 // tensor-memory columns of a stage's A tile
-    static_assert(BM <= G4_A_COL0, "accumulator and A ring must not overlap");
+    // With 128-row x tiles an MMA runs for 64 clk, less than it takes one thread to issue it next to sixteen busy decode
+    // warps; then two threads issue (warp 1: even stages into accumulator 0; warp 3: odd stages into accumulator 1 in
+    // columns [128, 256)) and the epilogue adds the two accumulators.
+    constexpr int NACC = (BM == 128) ? 2 : 1;
+    static_assert(BM * ((BM == 128) ? 2 : 1) <= G4_A_COL0, "accumulators and A ring must not overlap");
     extern __shared__ __align__(1024) unsigned char smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     unsigned char *smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
@@ -379,7 +383,7 @@ gemm_v16t_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
 
     if (tid == 0) {
         for (int s = 0; s < STAGES; ++s) { mbar_init(bar_full(s), 1 + 4); mbar_init(bar_empty(s), 1); }
-        mbar_init(bar_accum, 1);
+        mbar_init(bar_accum, NACC);
         for (int b = 0; b < 2; ++b) { mbar_init(bar_full_i(b), 1); mbar_init(bar_empty_i(b), G2_DWARPS); }
         mbar_init(bar_tab, 1);
         *s_abort = 0;
@@ -413,11 +417,13 @@ gemm_v16t_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                     tma_load_2d(smem_base + s * STAGE_BYTES + j * B_BYTES, &tmap_x, (kt0 + j) * G_BK, m0, bar_full(s));
             }
         }
-    } else if (warp == 1) {
+    } else if (warp == 1 || (NACC == 2 && warp == 3)) {
         if (lane == 0) {
+            const int me = (warp == 1) ? 0 : 1;                    // which accumulator / which stages
             uint32_t idesc = (1u << 4) | ((uint32_t)(BM >> 3) << 17) | ((uint32_t)(G_BN >> 4) << 24);
             if (is_bf16) idesc |= (1u << 7) | (1u << 10);
-            for (int ks = 0; ks < NS; ++ks) {
+            const uint32_t d_tm = tmem_d + me * BM;
+            for (int ks = me; ks < NS; ks += NACC) {
                 const int s = ks % STAGES;
                 if (!mbar_wait<false>(bar_full(s), (ks / STAGES) & 1, s_abort)) break;
                 tc_fence_after();
@@ -427,7 +433,7 @@ gemm_v16t_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                     const uint64_t bdesc = make_smem_desc(smem_base + s * STAGE_BYTES + j * B_BYTES);
 #pragma unroll
                     for (int k = 0; k < G_BK / 16; ++k)
-                        umma_f16_ts(tmem_d, a_tm + 32 * j + 8 * k, bdesc + 2 * k, idesc, (ks | j | k) ? 1u : 0u);
+                        umma_f16_ts(d_tm, a_tm + 32 * j + 8 * k, bdesc + 2 * k, idesc, (ks >= NACC || j || k) ? 1u : 0u);
                 }
                 umma_commit(bar_empty(s));
             }
@@ -498,6 +504,13 @@ gemm_v16t_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                 uint32_t rr[32];
                 tmem_ld32(tmem_d + lane_base + c0, rr);
                 tmem_ld_wait();
+                if (NACC == 2 && NS > 1) {                         // (with a single stage accumulator 1 was never written)
+                    uint32_t r2[32];
+                    tmem_ld32(tmem_d + lane_base + BM + c0, r2);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) rr[i] = __float_as_uint(__uint_as_float(rr[i]) + __uint_as_float(r2[i]));
+                }
                 if (nrow < a.N) {
 #pragma unroll
                     for (int i = 0; i < 32; ++i) {
