@@ -32,8 +32,10 @@
 //                BPL consecutive blocks; its activations stay in registers as MMA B fragments.
 //   warp 16      producer: TMA boxes (64 blocks x rows, 128-byte swizzle) of the index matrix into
 //                a shared ring, bulk copy of the codeword table.
-//   warps 17,18  epilogue: recombine the digits of the K-slices' partial tiles in a fixed order, add
-//                the K-parts, apply alpha (and mu), store y.
+//   warps 17,18  epilogue: add the K-slices' partial results in a fixed order (with M <= 2 they arrive as
+//                integer digit sums and are recombined here; with more rows of x each compute warp
+//                recombines its own), add the K-parts, apply alpha (and mu, both staged in shared
+//                memory once per chunk of row groups), store y.
 // Every mbarrier wait is bounded; when one runs out the CTA raises a status word and drains.
 #include <cuda.h>
 #include "btc_internal.cuh"
@@ -64,6 +66,7 @@ struct ImProblem {
     int groups;               // row groups: ceil(N / (16 * TRK))
     int ncls;                 // v / 4
     int cost;                 // cost of one row group (blocks, plus the per-part fragment rebuild; see launch_gemv_imma)
+    int per, rem;             // groups / cta_count and groups % cta_count
     int cta_begin, cta_count; // the CTAs that work on this layer (no CTA works on two layers: each switch would cost a
                               // table load and a fragment rebuild, and the slowest CTA sets the launch's time)
 };
@@ -155,10 +158,12 @@ __device__ __forceinline__ void im_unpack2(uint32_t w, int dt, float &lo, float 
 struct ImSmem {
     uint32_t bars;        // mbarriers: full[S], empty[S], part_full[2], part_empty[2], tab_full, tab_free
     uint32_t misc;        // abort flag, per-part scale slots
+    uint32_t rowsc;       // alpha and mu of the rows of the current chunk, float [2][IM_RC * 32]
     uint32_t planes;      // per compute warp: digit planes of its K-slice of one row of x
     uint32_t tab;         // codeword table
     uint32_t ring;        // index stages
-    uint32_t part;        // partial sums [2][16 warps][rows][cols]
+    uint32_t part;        // partial sums, two buffers: digit sums int [16 warps][16 rows][8 cols] (M <= 2), else partial dot
+                          // products float [tile][16 rows][m][K-slice]
     uint32_t acc;         // dot products summed over K-parts, float [IM_RC][rows][cols / 2]
     uint32_t total;
 };
@@ -177,25 +182,28 @@ __host__ __device__ inline ImSmem im_smem_layout(int tab_bytes, int cols, int ro
     o = (o + 15u) & ~15u;
     L.misc = o; o += IM_MISC_BYTES;
     o = (o + 15u) & ~15u;
+    L.rowsc = o; o += 2u * IM_RC * 32u * 4u;
     L.planes = o; o += IM_PLANE_WORDS * 4;
     o = (o + 127u) & ~127u;
     L.tab = o; o += (uint32_t)tab_bytes;
     o = (o + 1023u) & ~1023u;                     // swizzled TMA boxes want 1024-byte alignment
     L.ring = o; o += (uint32_t)stages * IM_STAGE_BYTES;
-    L.part = o; o += 2u * IM_CWARPS * 16u * (uint32_t)cols * 4u;           // one 16-row tile per compute warp
+    // cols == 8 (M <= 2): a 16 x 8 tile of digit sums per compute warp; else one float per (warp, row, m)
+    L.part = o; o += 2u * IM_CWARPS * 16u * (uint32_t)(cols == 8 ? 8 : (cols == 16 ? 5 : 8)) * 4u;
     L.acc = o; o += (uint32_t)IM_RC * (uint32_t)rows * (uint32_t)(cols / 2) * 4u;
     L.total = o;
     return L;
 }
 
-// Row groups [lo, hi) of layer P that fall to CTA b: the layer's cta_count CTAs split its row groups evenly.
+// Row groups [lo, hi) of layer P that fall to CTA b: the layer's cta_count CTAs split its row groups evenly (the first
+// `rem` of them take one more); per and rem come from the host, so no division runs here.
 __device__ __forceinline__ void im_group_range(const ImProblem &P, int b, int &lo, int &hi)
 {
     lo = hi = 0;
     const int r = b - P.cta_begin;
     if (r < 0 || r >= P.cta_count) return;
-    lo = (int)((long long)P.groups * r / P.cta_count);
-    hi = (int)((long long)P.groups * (r + 1) / P.cta_count);
+    lo = r * P.per + min(r, P.rem);
+    hi = lo + P.per + (r < P.rem ? 1 : 0);
 }
 
 // TAB_MODE 0: tables gathered from global memory; 1: whole tables in shared memory; 2: the first tab_head entries in
@@ -208,7 +216,6 @@ gemv_imma_kernel(const __grid_constant__ ImBatch batch)
     constexpr int TRK = (NM == 1) ? 2 : 1;               // 16-row tiles per row group
     constexpr int ROWS = TRK * 16;
     constexpr int COLS = 8 * NM;
-    constexpr int TILE_INTS = 16 * COLS;                 // one compute warp's partial tile
     constexpr int KS = 16 / TRK;                         // K-slices of a part; warp w: slice w % KS, tile w / KS
     constexpr int SLICE = IM_PW / KS;                    // blocks per slice
     constexpr int BPL = SLICE / 4;                       // blocks per lane
@@ -222,8 +229,15 @@ gemv_imma_kernel(const __grid_constant__ ImBatch batch)
     uint32_t *s_planes = reinterpret_cast<uint32_t *>(smem + L.planes);
     uint32_t *s_tab = reinterpret_cast<uint32_t *>(smem + L.tab);
     unsigned char *s_ring = smem + L.ring;
-    int *s_part = reinterpret_cast<int *>(smem + L.part);
+    // Who recombines the three digit sums of a (K-slice, row, m): with M <= 2 the compute warps set the pace, so they
+    // hand over their raw 16 x 8 integer tiles and the epilogue warps recombine; with more rows of x the epilogue
+    // would fall behind, so each compute warp recombines its own sums and hands over one float per (row, m).
+    constexpr bool FPART = (NM > 1);
+    constexpr int TILE_INTS = 16 * COLS;                 // one compute warp's integer tile
+    float *s_part = reinterpret_cast<float *>(smem + L.part);
+    int *s_parti = reinterpret_cast<int *>(smem + L.part);
     float *s_acc = reinterpret_cast<float *>(smem + L.acc);
+    float *s_alpha = reinterpret_cast<float *>(smem + L.rowsc), *s_mu = s_alpha + IM_RC * 32;
     constexpr int ACC_M = COLS / 2;                      // floats per row of s_acc (>= MAXM)
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -310,6 +324,26 @@ gemv_imma_kernel(const __grid_constant__ ImBatch batch)
                 float sxtot[MAXM];                               // sum_k x[m, k] over the parts seen so far
 #pragma unroll
                 for (int m = 0; m < MAXM; ++m) sxtot[m] = 0.f;
+                // alpha / mu of this thread's row in every row group of the chunk go to shared memory once per chunk (each
+                // thread reads back only what it wrote, so no barrier is needed): the loads, a trip to DRAM, overlap the
+                // compute warps' fragment build instead of sitting in every iteration's chain
+                if (grp == 0) {
+                    unsigned short ab[IM_RC], mb[IM_RC];
+#pragma unroll
+                    for (int i = 0; i < IM_RC; ++i) {                // all loads in flight together
+                        const int n = (c0 + i) * ROWS + R;
+                        ab[i] = 0; mb[i] = 0;
+                        if (i < c1 - c0 && n < P.N) {
+                            ab[i] = __ldg(reinterpret_cast<const unsigned short *>(P.alpha) + n);
+                            if (P.mu) mb[i] = __ldg(reinterpret_cast<const unsigned short *>(P.mu) + n);
+                        }
+                    }
+#pragma unroll
+                    for (int i = 0; i < IM_RC; ++i) {
+                        s_alpha[i * ROWS + R] = __half2float(__ushort_as_half(ab[i]));
+                        s_mu[i * ROWS + R] = __half2float(__ushort_as_half(mb[i]));
+                    }
+                }
                 for (int j = 0; j < P.parts && ok; ++j, ++pc) {
                     const bool last = (j == P.parts - 1);
                     const ImScale *sc = s_scale + (size_t)(pc % IM_SLOTS) * IM_CWARPS * 8;
@@ -320,15 +354,8 @@ gemv_imma_kernel(const __grid_constant__ ImBatch batch)
                         const int buf = li & 1;
                         const int n = r * ROWS + R;
                         const bool live = (n < P.N) && (grp == 0);
-                        // alpha / mu of this row: the loads are issued here and first used after the wait below, so their
-                        // latency (a trip to DRAM) hides behind it
-                        unsigned short al_bits = 0, mu_bits = 0;
-                        if (last && live) {
-                            al_bits = __ldg(reinterpret_cast<const unsigned short *>(P.alpha) + n);
-                            if (P.mu) mu_bits = __ldg(reinterpret_cast<const unsigned short *>(P.mu) + n);
-                        }
                         if (!im_mbar_wait(bar_pfull(buf), (li >> 1) & 1, s_abort)) { ok = false; break; }
-                        const float al = __half2float(__ushort_as_half(al_bits)), mu = __half2float(__ushort_as_half(mu_bits));
+                        const float al = s_alpha[(r - c0) * ROWS + R], mu = s_mu[(r - c0) * ROWS + R];
                         if (r == c0) {
 #pragma unroll
                             for (int m = 0; m < MAXM; ++m)
@@ -338,29 +365,42 @@ gemv_imma_kernel(const __grid_constant__ ImBatch batch)
                             for (int m = 0; m < MAXM; ++m) sxtot[m] += sxp[m];
                         }
                         float *accrow = s_acc + ((size_t)(P.parts > 1 ? (r - c0) : 0) * ROWS + R) * ACC_M;
-                        // row R lies in tile R / 16, written by the compute warps (R / 16) * KS + slice
-                        const int *base = s_part + ((size_t)buf * IM_CWARPS + (R >> 4) * KS + grp * WPG) * TILE_INTS + (size_t)(R & 15) * COLS;
                         float dots[MAXM];
-#pragma unroll
-                        for (int m = 0; m < MAXM; ++m) dots[m] = 0.f;
-#pragma unroll
-                        for (int w = 0; w < WPG; ++w) {
-                            int pv[COLS];
-#pragma unroll
-                            for (int c4 = 0; c4 < COLS / 4; ++c4) {
-                                if (c4 * 4 < 3 * P.M) {                     // columns 3 m + d, m < M
-                                    const int4 q = *reinterpret_cast<const int4 *>(base + (size_t)w * TILE_INTS + c4 * 4);
-                                    pv[c4 * 4] = q.x; pv[c4 * 4 + 1] = q.y; pv[c4 * 4 + 2] = q.z; pv[c4 * 4 + 3] = q.w;
-                                } else {
-                                    pv[c4 * 4] = pv[c4 * 4 + 1] = pv[c4 * 4 + 2] = pv[c4 * 4 + 3] = 0;
-                                }
-                            }
+                        if constexpr (FPART) {
+                            // row R lies in tile R / 16; its K-slices' partial dot products sit side by side
+                            const float *base = s_part + ((((size_t)buf * TRK + (R >> 4)) * 16 + (R & 15)) * MAXM) * KS + grp * WPG;
 #pragma unroll
                             for (int m = 0; m < MAXM; ++m) {
+                                dots[m] = 0.f;
                                 if (m < P.M) {
-                                    // each digit sum is below 2^24 in magnitude, so the conversions are exact
-                                    const float T = ((float)pv[3 * m + 2] * 256.0f + (float)pv[3 * m + 1]) * 256.0f + (float)pv[3 * m];
-                                    dots[m] += T * sc[(grp * WPG + w) * 8 + m].inv;
+                                    const float4 q = *reinterpret_cast<const float4 *>(base + m * KS);
+                                    dots[m] = ((q.x + q.y) + q.z) + q.w;
+                                }
+                            }
+                        } else {
+                            // row R lies in tile R / 16, written by the compute warps (R / 16) * KS + slice
+                            const int *base = s_parti + ((size_t)buf * IM_CWARPS + (R >> 4) * KS + grp * WPG) * TILE_INTS + (size_t)(R & 15) * COLS;
+#pragma unroll
+                            for (int m = 0; m < MAXM; ++m) dots[m] = 0.f;
+#pragma unroll
+                            for (int w = 0; w < WPG; ++w) {
+                                int pv[COLS];
+#pragma unroll
+                                for (int c4 = 0; c4 < COLS / 4; ++c4) {
+                                    if (c4 * 4 < 3 * P.M) {                 // columns 3 m + d, m < M
+                                        const int4 q = *reinterpret_cast<const int4 *>(base + (size_t)w * TILE_INTS + c4 * 4);
+                                        pv[c4 * 4] = q.x; pv[c4 * 4 + 1] = q.y; pv[c4 * 4 + 2] = q.z; pv[c4 * 4 + 3] = q.w;
+                                    } else {
+                                        pv[c4 * 4] = pv[c4 * 4 + 1] = pv[c4 * 4 + 2] = pv[c4 * 4 + 3] = 0;
+                                    }
+                                }
+#pragma unroll
+                                for (int m = 0; m < MAXM; ++m) {
+                                    if (m < P.M) {
+                                        // each digit sum is below 2^24 in magnitude, so the conversions are exact
+                                        const float T = ((float)pv[3 * m + 2] * 256.0f + (float)pv[3 * m + 1]) * 256.0f + (float)pv[3 * m];
+                                        dots[m] += T * sc[(grp * WPG + w) * 8 + m].inv;
+                                    }
                                 }
                             }
                         }
@@ -571,11 +611,15 @@ gemv_imma_kernel(const __grid_constant__ ImBatch batch)
                     };
                     if (!load_indices()) { ok = false; break; }
                     for (int r = c0; r < c1; ++r, ++li) {
-                        int acc[NM][4], acc2[NM][4];                 // two chains: an MMA need not wait for the previous one
+                        constexpr int CH = 2;        // accumulation chains: an MMA need not wait for the previous one
+                        int accs[CH][NM][4];
+                        int (&acc)[NM][4] = accs[0];
 #pragma unroll
                         for (int nm = 0; nm < NM; ++nm)
 #pragma unroll
-                            for (int i = 0; i < 4; ++i) { acc[nm][i] = 0; acc2[nm][i] = 0; }
+                            for (int i = 0; i < 4; ++i)
+#pragma unroll
+                                for (int ch = 0; ch < CH; ++ch) accs[ch][nm][i] = 0;
                         if (ks * SLICE < pw) {                      // warp-uniform: the slice is not empty
 #pragma unroll
                             for (int e4 = 0; e4 < BPL; e4 += 4) {
@@ -599,7 +643,7 @@ gemv_imma_kernel(const __grid_constant__ ImBatch batch)
                                         const uint32_t ma = 0x01010101u << (2 * cp), mb = 0x01010101u << (2 * cp + 1);
 #pragma unroll
                                         for (int nm = 0; nm < NM; ++nm)
-                                            im_mma_u8s8((cp & 1) ? acc2[nm] : acc[nm], w0[e] & ma, w1[e] & ma, w0[e] & mb, w1[e] & mb,
+                                            im_mma_u8s8(accs[((e & 1) * 2 + (cp & 1)) % CH][nm], w0[e] & ma, w1[e] & ma, w0[e] & mb, w1[e] & mb,
                                                         breg[e4 + e][2 * cp][nm], breg[e4 + e][2 * cp + 1][nm]);
                                     }
                                 }
@@ -617,18 +661,45 @@ gemv_imma_kernel(const __grid_constant__ ImBatch batch)
                         // the next row group's indices are fetched while this one's MMAs drain (their codewords are in
                         // registers by now), so the barrier round trip is off the critical path
                         if (r + 1 < c1 && !load_indices()) { ok = false; break; }
+                        // likewise the wait for the partial-sum buffer: its round trip overlaps the MMAs' drain
+                        const int buf = li & 1;
+                        if (li >= 2 && !im_mbar_wait(bar_pempty(buf), ((li >> 1) & 1) ^ 1, s_abort)) { ok = false; break; }
 #pragma unroll
                         for (int nm = 0; nm < NM; ++nm)
 #pragma unroll
-                            for (int i = 0; i < 4; ++i) acc[nm][i] += acc2[nm][i];
-                        const int buf = li & 1;
-                        if (li >= 2 && !im_mbar_wait(bar_pempty(buf), ((li >> 1) & 1) ^ 1, s_abort)) { ok = false; break; }
-                        int *mine = s_part + ((size_t)buf * IM_CWARPS + warp) * TILE_INTS;
+                            for (int i = 0; i < 4; ++i)
 #pragma unroll
-                        for (int nm = 0; nm < NM; ++nm) {
-                            if (nm * 8 + 2 * t < 3 * M) {               // columns 3 m + d, m < M: the others are never read
-                                *reinterpret_cast<int2 *>(mine + sg * COLS + nm * 8 + 2 * t) = make_int2(acc[nm][0], acc[nm][1]);
-                                *reinterpret_cast<int2 *>(mine + (sg + 8) * COLS + nm * 8 + 2 * t) = make_int2(acc[nm][2], acc[nm][3]);
+                                for (int ch = 1; ch < CH; ++ch) acc[nm][i] += accs[ch][nm][i];
+                        if constexpr (FPART) {
+                            // The three digit sums of (row, m) sit in columns 3 m .. 3 m + 2, spread over the lanes of a quad:
+                            // they are brought together by shuffles, recombined (each is below 2^24 in magnitude, so the
+                            // conversions are exact), scaled by the slice's 2^-s and stored as one float per (row, m).
+                            float *mine = s_part + (((size_t)buf * TRK + rh) * 16) * MAXM * KS + ks;
+#pragma unroll
+                            for (int m = 0; m < MAXM; ++m) {
+                                if (m < M) {                                // warp-uniform
+                                    int dlo[3], dhi[3];
+#pragma unroll
+                                    for (int d = 0; d < 3; ++d) {
+                                        const int col = 3 * m + d;          // a constant once unrolled
+                                        const int src = (lane & ~3) | ((col & 7) >> 1);
+                                        dlo[d] = __shfl_sync(0xffffffffu, acc[col >> 3][col & 1], src);
+                                        dhi[d] = __shfl_sync(0xffffffffu, acc[col >> 3][2 + (col & 1)], src);
+                                    }
+                                    if (t == (m & 3)) {
+                                        const float inv = scale_out[m].inv;
+                                        const float Tlo = ((float)dlo[2] * 256.0f + (float)dlo[1]) * 256.0f + (float)dlo[0];
+                                        const float Thi = ((float)dhi[2] * 256.0f + (float)dhi[1]) * 256.0f + (float)dhi[0];
+                                        mine[(sg * MAXM + m) * KS] = Tlo * inv;
+                                        mine[((sg + 8) * MAXM + m) * KS] = Thi * inv;
+                                    }
+                                }
+                            }
+                        } else {
+                            int *mine = s_parti + ((size_t)buf * IM_CWARPS + warp) * TILE_INTS;
+                            if (2 * t < 3 * M) {                        // columns 3 m + d, m < M: the others are never read
+                                *reinterpret_cast<int2 *>(mine + sg * COLS + 2 * t) = make_int2(acc[0][0], acc[0][1]);
+                                *reinterpret_cast<int2 *>(mine + (sg + 8) * COLS + 2 * t) = make_int2(acc[0][2], acc[0][3]);
                             }
                         }
                         __syncwarp();
@@ -742,7 +813,12 @@ static int im_assign_ctas(ImBatch &b, int budget)
         ++b.p[best].cta_count; ++sum;
     }
     int begin = 0;
-    for (int i = 0; i < b.count; ++i) { b.p[i].cta_begin = begin; begin += b.p[i].cta_count; }
+    for (int i = 0; i < b.count; ++i) {
+        b.p[i].cta_begin = begin;
+        begin += b.p[i].cta_count;
+        b.p[i].per = b.p[i].groups / b.p[i].cta_count;
+        b.p[i].rem = b.p[i].groups % b.p[i].cta_count;
+    }
     return begin;
 }
 
