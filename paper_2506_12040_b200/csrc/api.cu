@@ -110,7 +110,8 @@ extern "C" int btc_last_cuda_error(void) { return g_last_cuda_error; }
 extern "C" size_t btc_codebook_packed_bytes(int Kc, int v)
 {
     if (v < 1 || v > 32 || Kc < 1 || Kc > 65536) return 0;
-    return (size_t)((Kc + 3) / 4 * 4) * 12;
+    // three sections of (Kc rounded up to 4) 32-bit words and one of (Kc rounded up to 8) 16-bit halves
+    return (size_t)((Kc + 3) / 4 * 4) * 12 + (size_t)((Kc + 7) / 8 * 8) * 2;
 }
 
 extern "C" size_t btc_linear_workspace_bytes(int M, int N, int K, int v, int Kc)

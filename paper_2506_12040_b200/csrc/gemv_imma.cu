@@ -57,6 +57,7 @@ struct ImProblem {
     const void *x;
     const uint16_t *idx;
     const uint32_t *tab;      // byte-lane codeword words [Kc]
+    const uint16_t *tab16;    // the same squeezed into 16 bits (v <= 16)
     const __half *alpha;
     const __half *mu;         // may be nullptr
     void *y;
@@ -207,7 +208,8 @@ __device__ __forceinline__ void im_group_range(const ImProblem &P, int b, int &l
 }
 
 // TAB_MODE 0: tables gathered from global memory; 1: whole tables in shared memory; 2: the first tab_head entries in
-// shared memory, the rest from global memory.
+// shared memory, the rest from global memory; 3: whole tables in shared memory as 16-bit halves (v <= 16; a table of
+// 65536 codewords then takes 128 KB), widened by `h | (h << 12)` after the gather.
 template <int NCLS, int NM, int TAB_MODE>
 __global__ void __launch_bounds__(IM_THREADS, 1)
 gemv_imma_kernel(const __grid_constant__ ImBatch batch)
@@ -278,9 +280,11 @@ gemv_imma_kernel(const __grid_constant__ ImBatch batch)
             if (tab_smem) {
                 if (ps > 0 && !im_mbar_wait(bar_tabfree, (ps - 1) & 1, s_abort)) break;
                 if (lane == 0) {
-                    const uint32_t bytes = (uint32_t)(min((P.Kc + 3) / 4 * 4, batch.tab_head) * 4);
+                    const uint32_t bytes = TAB_MODE == 3 ? (uint32_t)((P.Kc + 7) / 8 * 8 * 2)
+                                                         : (uint32_t)(min((P.Kc + 3) / 4 * 4, batch.tab_head) * 4);
                     im_mbar_expect_tx(bar_tabfull, bytes);
-                    im_bulk_g2s(im_smem_u32(s_tab), P.tab, bytes, bar_tabfull);
+                    im_bulk_g2s(im_smem_u32(s_tab), TAB_MODE == 3 ? static_cast<const void *>(P.tab16) : static_cast<const void *>(P.tab),
+                                bytes, bar_tabfull);
                 }
             }
             ++ps;
@@ -630,6 +634,11 @@ gemv_imma_kernel(const __grid_constant__ ImBatch batch)
                                     const uint32_t i0 = (e & 1) ? (pa >> 16) : (pa & 0xffffu);
                                     const uint32_t i1 = (e & 1) ? (pb >> 16) : (pb & 0xffffu);
                                     if (TAB_MODE == 1) { w0[e] = s_tab[i0]; w1[e] = s_tab[i1]; }
+                                    else if (TAB_MODE == 3) {
+                                        const uint32_t h0 = reinterpret_cast<const uint16_t *>(s_tab)[i0];
+                                        const uint32_t h1 = reinterpret_cast<const uint16_t *>(s_tab)[i1];
+                                        w0[e] = h0 | (h0 << 12); w1[e] = h1 | (h1 << 12);
+                                    }
                                     else if (TAB_MODE == 0) { w0[e] = __ldg(gtab + i0); w1[e] = __ldg(gtab + i1); }
                                     else {
                                         w0[e] = i0 < tab_head ? s_tab[i0] : __ldg(gtab + i0);
@@ -861,7 +870,7 @@ int launch_gemv_imma(const LinearArgs *problems, int count, cudaStream_t s)
     if (!enc) return BTC_ERR_UNSUPPORTED;
     ImBatch b = {};
     b.count = count;
-    int ncls_max = 0, m_max = 0, tab_max = 0;
+    int ncls_max = 0, m_max = 0, tab_max = 0, tab16_max = 0, v_max = 0;
     for (int i = 0; i < count; ++i) {
         const LinearArgs &a = problems[i];
         // covered: M <= 8, v a multiple of 4 up to 20, K/v a multiple of 8 (16-byte rows for the bulk copies)
@@ -877,6 +886,7 @@ int launch_gemv_imma(const LinearArgs *problems, int count, cudaStream_t s)
         p.x = a.x; p.idx = a.idx; p.alpha = a.alpha; p.mu = a.mu; p.y = a.y;
         const int Kc4 = (a.Kc + 3) / 4 * 4;
         p.tab = a.Cp + 2 * Kc4;                      // byte-lane words follow the two other forms
+        p.tab16 = reinterpret_cast<const uint16_t *>(a.Cp + 3 * (size_t)Kc4);
         p.M = a.M; p.N = a.N; p.K = a.K; p.v = a.v; p.Kc = a.Kc; p.Kb = a.Kb;
         p.x_dt = a.x_dt; p.y_dt = a.y_dt;
         p.parts = (a.Kb + IM_PW - 1) / IM_PW;
@@ -891,23 +901,32 @@ int launch_gemv_imma(const LinearArgs *problems, int count, cudaStream_t s)
         groups_total += p.groups;
         if (p.ncls > ncls_max) ncls_max = p.ncls;
         if (Kc4 * 4 > tab_max) tab_max = Kc4 * 4;
+        if ((a.Kc + 7) / 8 * 16 > tab16_max) tab16_max = (a.Kc + 7) / 8 * 16;
+        if (a.v > v_max) v_max = a.v;
     }
-    // the whole table in shared memory when it fits beside at least four index stages; else as much of its head as fits
+    // the whole table in shared memory when it fits beside at least four index stages; else, for v <= 16, as 16-bit
+    // halves beside at least two; else as much of its head as fits
     int mode = 1;
     b.tab_smem_bytes = tab_max;
     b.tab_head = tab_max / 4;
     if (im_smem_layout(tab_max, 8 * nm, rows, 4).total > 227u * 1024u) {
-        mode = 2;
-        int head_bytes = tab_max;
-        while (head_bytes > 0 && im_smem_layout(head_bytes, 8 * nm, rows, 4).total > 227u * 1024u) head_bytes -= 4096;
-        if (head_bytes <= 0) { mode = 0; head_bytes = 0; }
-        b.tab_smem_bytes = head_bytes;
-        b.tab_head = head_bytes / 4;
+        if (v_max <= 16 && im_smem_layout(tab16_max, 8 * nm, rows, 2).total <= 227u * 1024u) {
+            mode = 3;
+            b.tab_smem_bytes = tab16_max;
+        } else {
+            mode = 2;
+            int head_bytes = tab_max;
+            while (head_bytes > 0 && im_smem_layout(head_bytes, 8 * nm, rows, 4).total > 227u * 1024u) head_bytes -= 4096;
+            if (head_bytes <= 0) { mode = 0; head_bytes = 0; }
+            b.tab_smem_bytes = head_bytes;
+            b.tab_head = head_bytes / 4;
+        }
     }
     b.stages = IM_STAGES;
     while (b.stages > 2 && im_smem_layout(b.tab_smem_bytes, 8 * nm, rows, b.stages).total > 227u * 1024u) --b.stages;
     if (ncls_max <= 4) {
         if (mode == 1) return im_launch_nm<4, 1>(b, nm, groups_total, s);
+        if (mode == 3) return im_launch_nm<4, 3>(b, nm, groups_total, s);
         if (mode == 2) return im_launch_nm<4, 2>(b, nm, groups_total, s);
         return im_launch_nm<4, 0>(b, nm, groups_total, s);
     }

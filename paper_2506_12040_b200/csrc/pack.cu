@@ -27,7 +27,19 @@ __host__ __device__ inline uint32_t byte_lane_word(uint32_t pub, int v)
     return w;
 }
 
-// bit t of out[k] = (C[k][t] + 1) / 2, with C >= 0 read as +1; private words at out[Kc4 + k].
+// The byte-lane word squeezed into 16 bits for codebooks too large to sit in shared memory as 32-bit words
+// (v <= 16): nibble q of the result is the low nibble of byte {0, 2, 1, 3}[q] of the byte-lane word, so that
+// `h | (h << 12)` has the low nibble of every byte in place (the high nibbles carry leftovers, which the kernel's
+// masks never look at).  0 for v > 16.
+__host__ __device__ inline uint16_t byte_lane_half(uint32_t pub, int v)
+{
+    if (v > 16) return 0;
+    const uint32_t w = byte_lane_word(pub, v);
+    return (uint16_t)((w & 0xFu) | (((w >> 16) & 0xFu) << 4) | (((w >> 8) & 0xFu) << 8) | (((w >> 24) & 0xFu) << 12));
+}
+
+// bit t of out[k] = (C[k][t] + 1) / 2, with C >= 0 read as +1; private words at out[Kc4 + k], out[2 Kc4 + k] and, as
+// 16-bit halves, from out[3 Kc4].
 __global__ void pack_codebook_kernel(const int8_t *__restrict__ C, int Kc, int v, uint32_t *__restrict__ out)
 {
     const int k = blockIdx.x * blockDim.x + threadIdx.x;
@@ -40,6 +52,9 @@ __global__ void pack_codebook_kernel(const int8_t *__restrict__ C, int Kc, int v
     out[k] = w;
     out[Kc4 + k] = mma_layout_word(w, v);
     out[2 * Kc4 + k] = byte_lane_word(w, v);
+    uint16_t *half = reinterpret_cast<uint16_t *>(out + 3 * (size_t)Kc4);   // (Kc + 7) / 8 * 8 entries: a whole number of 16 bytes
+    half[k] = byte_lane_half(w, v);
+    if (k < (Kc + 7) / 8 * 8 - Kc4) half[Kc4 + k] = 0;
 }
 
 // One thread per (row, block): expands the centroid word into v int8 signs.
@@ -90,6 +105,9 @@ extern "C" int btc_codebook_pack_host(const int8_t *C, int Kc, int v, uint32_t *
         out[k] = w;
         out[Kc4 + k] = mma_layout_word(w, v);
         out[2 * Kc4 + k] = byte_lane_word(w, v);
+        uint16_t *half = reinterpret_cast<uint16_t *>(out + 3 * (size_t)Kc4);
+        half[k] = byte_lane_half(w, v);
+        if (k < (Kc + 7) / 8 * 8 - Kc4) half[Kc4 + k] = 0;
     }
     return BTC_OK;
 }

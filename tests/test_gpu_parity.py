@@ -64,6 +64,8 @@ SMALL = [
     (257, 1040, 16, 4096, 8, "uniform", False),
     (300, 2000, 20, 65536, 4, "zipf", False),
     (129, 4096, 16, 8192, 1, "uniform", True),
+    (150, 2048, 16, 65536, 1, "uniform", True),
+    (77, 1024, 16, 50000, 2, "zipf", False),
     (70, 11008, 16, 8192, 2, "uniform", False),
     (1000, 640, 20, 21619, 5, "zipf", True),
     (33, 72, 4, 9, 7, "uniform", False),
@@ -202,6 +204,24 @@ def test_gemv_batch_matches_oracle_and_single_calls():
             else:           # single calls with M > 2 take the fp16 bit-trick kernel
                 rel2, fwd2 = errors(single, oracle_y(L), L)
                 assert rel2 <= TOL_GEMV and fwd2 <= TOL_GEMV, (L.spec, M, rel2, fwd2)
+    assert btc.device_status() == 0
+
+
+@pytest.mark.parametrize("M", [1, 2, 4, 8])
+def test_gemv_batch_large_codebooks_16bit_table(M):
+    """Codebooks too large to sit in shared memory as 32-bit words (v <= 16): the decode kernel keeps them as 16-bit
+    halves.  65536 centroids at v = 16 is the codebook of all patterns; 40000 and a v = 12 layer ride in the same launch."""
+    shapes = [(200, 4096, 16, 65536, True, "uniform"), (130, 1024, 16, 40000, False, "zipf"), (64, 768, 12, 4096, False, "uniform"),
+              (300, 11008, 16, 65536, False, "uniform")]
+    Ls = [wl.make_layer(_spec(N, K, v, Kc, idx_dist=dist, with_mu=mu, outlier_frac=0.01), M, seed=900 + i)
+          for i, (N, K, v, Kc, mu, dist) in enumerate(shapes)]
+    ds = [to_device(L) for L in Ls]
+    outs = btc.linear_gemv_batch([dict(x=d["x"], idx=d["idx"], C_packed=d["Cp"], alpha=d["alpha"], mu=d["mu"], v=L.spec.v, Kc=L.spec.Kc)
+                                  for L, d in zip(Ls, ds)])
+    torch.cuda.synchronize()
+    for L, y in zip(Ls, outs):
+        rel, fwd = errors(y, oracle_y(L), L)
+        assert rel <= TOL_GEMV and fwd <= TOL_GEMV, (L.spec, M, rel, fwd)
     assert btc.device_status() == 0
 
 

@@ -82,7 +82,7 @@ def test_accounting_matches_closed_forms():
         assert abs(btc.bits_per_weight(N, K, v, Kc, sb, mode, cb)
                    - oracle.bits_per_weight(N, K, v, Kc, sb, mode, cb)) < 1e-15
     assert btc.lib.btc_bits_per_weight(1, 1, 40, 4, 0, 0, 0) == -1.0
-    assert btc.lib.btc_codebook_packed_bytes(8192, 16) == 8192 * 12
-    assert btc.lib.btc_codebook_packed_bytes(7133, 16) == 7136 * 12
+    assert btc.lib.btc_codebook_packed_bytes(8192, 16) == 8192 * 14
+    assert btc.lib.btc_codebook_packed_bytes(7133, 16) == 7136 * 14
     assert btc.lib.btc_codebook_packed_bytes(0, 16) == 0
     assert btc.linear_workspace_bytes(1, 4096, 4096, 15, 4096) == 0   # invalid shape: v does not divide K
