@@ -37,7 +37,7 @@ UNIT = "GB/s"
 CONFIG_ID = 2
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the fused step kernel, from the ncu capture summarised in
 # profiles/decode_imma_config2_M1_step.md (set to None whenever that kernel changes until it is captured again)
-TRAFFIC_BYTES_PER_LAUNCH = 25724416
+TRAFFIC_BYTES_PER_LAUNCH = 25726720
 
 
 def measured_peaks():
