@@ -315,3 +315,102 @@ def test_pins_catch_planted_mistakes():
     }
     for name, bad in mutants.items():
         assert np.abs(bad - y).max() > 1e-3 * np.abs(y).max(), name
+
+
+# ------------------------------------------------------------------ codebook construction (Section 4.1)
+
+def _read_kmeans_fixture():
+    vals = {"vec": [], "init": [], "C1": [], "C2": []}
+    with open(os.path.join(GOLDEN, "kmeans_tiny.txt")) as f:
+        for line in f:
+            line = line.strip()
+            if not line or line.startswith("#"):
+                continue
+            key, *rest = line.split()
+            nums = [int(t) for t in rest]
+            if key in vals:
+                vals[key].append(nums)
+            else:
+                vals[key] = nums
+    return vals
+
+
+def test_kmeans_hand_worked_example():
+    from oracle import codebook_kmeans as km
+    g = _read_kmeans_fixture()
+    B = np.array(g["vec"], dtype=np.int8)
+    c = g["c"][0]
+    C0, n_unique = km.initial_codebook(B, c)
+    assert n_unique == 5 and np.array_equal(C0, np.array(g["init"], dtype=np.int8))
+    z1 = km.e_step(B, C0)
+    assert z1.tolist() == g["z1"]
+    C1 = km.m_step(B, z1, C0)
+    assert np.array_equal(C1, np.array(g["C1"], dtype=np.int8))
+    z2 = km.e_step(B, C1)
+    assert z2.tolist() == g["z2"]
+    C2 = km.m_step(B, z2, C1)
+    assert np.array_equal(C2, np.array(g["C2"], dtype=np.int8))
+    C, z, iters, _ = km.optimize_codebook(B, c, max_iter=10)
+    assert iters == g["iterations"][0] and z.tolist() == g["z3"] and np.array_equal(C, C2)
+    assert km.total_hamming(B, C, z) == g["total_hamming"][0]
+    # stopping early by max_iter: one E-step and one M-step
+    C_a, z_a, it_a, _ = km.optimize_codebook(B, c, max_iter=1)
+    assert it_a == 1 and z_a.tolist() == g["z1"] and np.array_equal(C_a, C1)
+
+
+def test_kmeans_majority_vote_ties_and_empty_clusters():
+    from oracle import codebook_kmeans as km
+    B = np.array([[1, -1], [-1, 1]], dtype=np.int8)
+    C = km.m_step(B, np.array([0, 0]), np.array([[-1, -1], [1, -1]], dtype=np.int8))
+    assert C.tolist() == [[1, 1], [1, -1]]          # element means 0 -> +1; the empty cluster keeps its centroid
+
+
+def test_kmeans_single_centroid_is_the_bitwise_majority():
+    """c = 1 after one M-step: the centroid is the element-wise majority of all vectors (closed form)."""
+    from oracle import codebook_kmeans as km
+    rng = np.random.default_rng(5)
+    B = np.where(rng.random((501, 12)) < 0.4, 1, -1).astype(np.int8)
+    C, z, iters, _ = km.optimize_codebook(B, 1, max_iter=5)
+    assert np.array_equal(C[0], np.where(B.astype(np.int64).sum(axis=0) >= 0, 1, -1))
+    assert not z.any() and iters == 2
+
+
+def test_kmeans_e_step_equals_hamming_argmin_on_packed_words():
+    """||b - c||^2 = 4 d_H(b, c) (Section 4.1): the E-step's Euclidean argmin equals the argmin of
+    POPCNT(b xor c) on packed words, first index among equals."""
+    from oracle import codebook_kmeans as km
+    rng = np.random.default_rng(6)
+    v = 11
+    B = np.where(rng.random((300, v)) < 0.5, 1, -1).astype(np.int8)
+    C = np.where(rng.random((17, v)) < 0.5, 1, -1).astype(np.int8)
+    z = km.e_step(B, C)
+    bw, cw = km.pack_words(B), km.pack_words(C)
+    for i in range(B.shape[0]):
+        d = [bin(int(bw[i]) ^ int(cw[k])).count("1") for k in range(C.shape[0])]
+        assert z[i] == d.index(min(d))
+        assert ((B[i].astype(int) - C[z[i]].astype(int)) ** 2).sum() == 4 * min(d)
+
+
+def test_kmeans_objective_never_increases_and_few_distinct_vectors_are_kept_exactly():
+    from oracle import codebook_kmeans as km
+    rng = np.random.default_rng(7)
+    v, c = 10, 24
+    proto = np.where(rng.random((40, v)) < 0.5, 1, -1).astype(np.int8)
+    B = proto[rng.integers(0, 40, 4000)]
+    flip = rng.random(B.shape) < 0.03
+    B = np.where(flip, -B, B).astype(np.int8)
+    C = km.initial_codebook(B, c)[0]
+    prev = None
+    for _ in range(6):
+        z = km.e_step(B, C)
+        obj = km.total_hamming(B, C, z)
+        assert prev is None or obj <= prev          # the E-step cannot increase it ...
+        C = km.m_step(B, z, C)
+        obj2 = km.total_hamming(B, C, z)
+        assert obj2 <= obj                          # ... nor can the majority vote
+        prev = obj2
+    # at most c distinct vectors: the codebook is the set of distinct vectors and the loss is zero
+    few = proto[:c][rng.integers(0, c, 1000)]
+    C2, z2, iters, n_unique = km.optimize_codebook(few, c + 5, max_iter=10)
+    assert C2.shape[0] == n_unique <= c and km.total_hamming(few, C2, z2) == 0
+    assert len({tuple(r) for r in C2.tolist()}) == n_unique
