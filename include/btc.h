@@ -89,6 +89,29 @@ BTC_API int btc_codebook_pack(const int8_t *C_pm1, int Kc, int v, uint32_t *C_pa
 /* Same mapping with both pointers in HOST memory; runs on the calling thread, no GPU work. */
 BTC_API int btc_codebook_pack_host(const int8_t *C_pm1_host, int Kc, int v, uint32_t *C_packed_host);
 
+/* ---- codebook construction (offline; the step before the layer) -----------------------------
+ * Section 4.1 "Flash and Accurate Binary Codebook", steps (1)-(3), with the loop of the appendix
+ * Algorithm "Binary Codebook Optimization": the c most frequent distinct vectors are the initial
+ * centroids; E-step z_i = argmin_k d_H(b_i, c_k) (POPCNT of the XOR; ||b - c||^2 = 4 d_H); M-step
+ * c_k = element-wise majority of its vectors (ties -> +1; a cluster without vectors keeps its
+ * centroid); stop when an E-step changes no assignment, or after max_iter E-steps.
+ * Choices the paper leaves open: equally frequent vectors are ordered by their packed word,
+ * ascending; among equally near centroids the smallest index wins.
+ *   vecs      device, n uint32 words, bit t (LSB first) = (b_t + 1) / 2, bits >= v ignored
+ *   C_words   device, Kc uint32 words out: the centroids in the public packed form (what
+ *             btc_codebook_pack calls the first section); slots >= info[1] are 0
+ *   z         device, n uint16 out: the assignment of the last E-step that ran
+ *   info      device, 4 ints out: E-steps run; min(Kc, number of distinct vectors); number of
+ *             distinct vectors; 1 if the loop ended because nothing changed
+ *   workspace device, btc_codebook_kmeans_workspace_bytes(v, Kc) bytes, 256-byte aligned
+ * Integer arithmetic only: the result is unique.  Work is enqueued on `stream`, nothing is
+ * allocated, nothing synchronises (the loop is max_iter rounds of launches; rounds after the
+ * last one return at once).  v <= 16 (the steps run over the 2^v patterns); 16 < v <= 32 returns
+ * BTC_ERR_UNSUPPORTED.  1 <= Kc <= 65536, 1 <= n < 2^31, 1 <= max_iter <= 4096. */
+BTC_API size_t btc_codebook_kmeans_workspace_bytes(int v, int Kc);
+BTC_API int btc_codebook_kmeans(const uint32_t *vecs, size_t n, int v, int Kc, int max_iter, uint32_t *C_words,
+                                uint16_t *z, int *info, void *workspace, size_t workspace_bytes, void *stream);
+
 /* ---- the layer ---------------------------------------------------------------------------
  * y[m, n] = alpha_n * sum_j <x[m, j*v:(j+1)*v], C[idx[n, j]]>  (+ mu_n * sum_k x[m, k])
  *

@@ -83,23 +83,25 @@ def m_step(B_pm1: np.ndarray, z: np.ndarray, C_pm1: np.ndarray) -> np.ndarray:
     return C
 
 
-def optimize_codebook(B_pm1: np.ndarray, c: int, max_iter: int):
-    """Returns (C int8 [c_eff, v], z int64 [n], iterations run, number of distinct vectors)."""
+def optimize_codebook(B_pm1: np.ndarray, c: int, max_iter: int, with_flag: bool = False):
+    """Returns (C int8 [c_eff, v], z int64 [n], E-steps run, number of distinct vectors) and, with_flag, whether
+    the loop ended because an E-step changed no assignment."""
     B = np.asarray(B_pm1, dtype=np.int8)
     C, n_unique = initial_codebook(B, c)
     z = None
     iters = 0
+    converged = False
     for _ in range(max_iter):
         z_new = e_step(B, C)
         iters += 1
         if z is not None and np.array_equal(z_new, z):
-            z = z_new
+            converged = True
             break
         z = z_new
         C = m_step(B, z, C)
     if z is None:
         z = e_step(B, C)
-    return C, z, iters, n_unique
+    return (C, z, iters, n_unique, converged) if with_flag else (C, z, iters, n_unique)
 
 
 def total_hamming(B_pm1: np.ndarray, C_pm1: np.ndarray, z: np.ndarray) -> int:

@@ -21,6 +21,7 @@ EXPORTS = (
     "btc_version", "btc_status_string", "btc_last_cuda_error", "btc_codebook_packed_bytes",
     "btc_codebook_pack", "btc_codebook_pack_host", "btc_linear_workspace_bytes", "btc_linear_gemv",
     "btc_linear_gemm", "btc_linear_gemv_batch", "btc_linear_gemm_static_scratch", "btc_decode_pm1", "btc_validate_indices", "btc_bits_per_weight", "btc_device_status", "btc_device_status_reset", "btc_selftest_bounded_wait",
+    "btc_codebook_kmeans_workspace_bytes", "btc_codebook_kmeans",
 )
 
 
@@ -72,6 +73,9 @@ def _load() -> ctypes.CDLL:
     L.btc_validate_indices.argtypes = [vp, sz, ci, vp, vp]
     L.btc_device_status.argtypes = [ctypes.POINTER(ctypes.c_int)]
     L.btc_selftest_bounded_wait.argtypes = [vp]
+    L.btc_codebook_kmeans_workspace_bytes.restype = sz
+    L.btc_codebook_kmeans_workspace_bytes.argtypes = [ci, ci]
+    L.btc_codebook_kmeans.argtypes = [vp, sz, ci, ci, ci, vp, vp, vp, vp, sz, vp]
     L.btc_bits_per_weight.restype = ctypes.c_double
     L.btc_bits_per_weight.argtypes = [ci] * 7
     return L
@@ -259,6 +263,26 @@ def linear_gemm_static_scratch(x, idx, C_packed, alpha, v, Kc, mu=None, out=None
 def linear(x, idx, C_packed, alpha, v, Kc, **kw):
     """Routes by M the way a caller would: decode path up to 8 rows, tensor-core path above."""
     return (linear_gemv if x.shape[0] <= 8 else linear_gemm)(x, idx, C_packed, alpha, v, Kc, **kw)
+
+
+def codebook_kmeans(vecs: torch.Tensor, v: int, Kc: int, max_iter: int = 20, workspace: Optional[torch.Tensor] = None):
+    """btc_codebook_kmeans on n packed vectors (int32 words on the device, bit t = element t).  Returns
+    (C_words int32 [Kc], z int16 [n], info int32 [4] on the device: E-steps run, centroids in use, distinct
+    vectors, converged)."""
+    _dev(vecs, "vecs")
+    if vecs.dtype != torch.int32 or vecs.dim() != 1:
+        raise ValueError("vecs must be a 1-D int32 tensor of packed vectors")
+    need = int(lib.btc_codebook_kmeans_workspace_bytes(v, Kc))
+    if workspace is None:
+        workspace = torch.empty(max(need, 256), dtype=torch.uint8, device=vecs.device)
+    C = torch.empty(Kc, dtype=torch.int32, device=vecs.device)
+    z = torch.empty(vecs.numel(), dtype=torch.int16, device=vecs.device)
+    info = torch.empty(4, dtype=torch.int32, device=vecs.device)
+    st = lib.btc_codebook_kmeans(vecs.data_ptr(), vecs.numel(), v, Kc, max_iter, C.data_ptr(), z.data_ptr(), info.data_ptr(),
+                                 workspace.data_ptr(), workspace.numel(), _stream())
+    if st:
+        raise BtcError(st, "btc_codebook_kmeans")
+    return C, z, info
 
 
 def decode_pm1(idx, C_packed, v, Kc) -> torch.Tensor:
