@@ -423,6 +423,26 @@ def run_gpu(args):
                     "frac_measured": nbytes / t * 1e-9 / peaks["hbm_gbs"], "launches": len(launches), "finite": finite}
         details["config5_chain"] = {f"Kc{Kc}_{dn}": time_chain(Kc, dn)
                                     for (Kc, dn) in ((4096, "uniform"), (256, "uniform"), (65536, "uniform"), (4096, "zipf"))}
+        # ---- codebook construction: the blocks of a 4096 x 4096 sign matrix (v = 16), 8192 centroids
+        def time_kmeans(n=4096 * 4096 // 16, v=16, Kc=8192, max_iter=8):
+            words = torch.from_numpy(wl.make_sign_words(n, v, cfg["seed"] + 31).view(np.int32)).to(dev)
+            ws = torch.empty(int(btc.lib.btc_codebook_kmeans_workspace_bytes(v, Kc)), dtype=torch.uint8, device=dev)
+            ts = []
+            info = None
+            for _ in range(4):
+                e0 = torch.cuda.Event(enable_timing=True)
+                e1 = torch.cuda.Event(enable_timing=True)
+                e0.record()
+                C, z, info = btc.codebook_kmeans(words, v, Kc, max_iter, workspace=ws)
+                e1.record()
+                torch.cuda.synchronize()
+                ts.append(e0.elapsed_time(e1) * 1e-3)
+            t = float(np.median(ts[1:]))
+            it, k_eff, n_unique, conv = (int(a) for a in info.cpu().numpy())
+            return {"n": n, "v": v, "Kc": Kc, "max_iter": max_iter, "e_steps": it, "distinct_vectors": n_unique, "converged": bool(conv),
+                    "ms": t * 1e3, "pattern_centroid_pairs_per_e_step": float(n_unique) * k_eff,
+                    "note": "whole call timed (histogram, frequency ranking, E/M rounds, assignment); per-kernel times: profiles/"}
+        details["codebook_kmeans"] = time_kmeans()
         details["device_status"] = btc.device_status()
 
     # ---- end to end: host buffers in, host buffers out, through the same calls

@@ -13,6 +13,7 @@ from .gen import (  # noqa: F401
     make_layer,
     make_codebook_pm1,
     make_indices,
+    make_sign_words,
     make_alpha_f16,
     make_x,
     f32_to_bf16_bits,

@@ -133,6 +133,25 @@ def make_indices(N: int, Kb: int, Kc: int, dist: str, seed: int, stream: int = 1
     return idx.astype(np.uint16).reshape(N, Kb)
 
 
+def make_sign_words(n: int, v: int, seed: int, stream: int = 7, prototypes: int = 4096, flip: float = 0.06) -> np.ndarray:
+    """n packed v-bit sign vectors (uint32, bit t = element t) standing in for the blocks of a binarised weight
+    matrix: each is one of `prototypes` seeded patterns (picked with Zipf(1.1) frequencies) with every element
+    flipped independently with probability `flip`, which gives the skewed, clustered pattern histogram that a
+    codebook is built for.  prototypes = 0: independent fair signs."""
+    mask = np.uint64((1 << v) - 1)
+    if prototypes <= 0:
+        return (_u64(seed, stream, n) & mask).astype(np.uint32)
+    protos = _u64(seed, stream + 100, prototypes) & mask
+    w = np.arange(1, prototypes + 1, dtype=np.float64) ** -1.1
+    cdf = np.cumsum(w) / w.sum()
+    pick = np.minimum(np.searchsorted(cdf, _uniform01(seed, stream + 101, n), side="right"), prototypes - 1)
+    words = protos[pick]
+    for t in range(v):
+        f = _uniform01(seed, stream + 200 + t, n) < flip
+        words = words ^ (f.astype(np.uint64) << np.uint64(t))
+    return words.astype(np.uint32)
+
+
 def make_alpha_f16(N: int, seed: int, stream: int = 2, sigma: float = 0.02, scale: float = 1.0) -> np.ndarray:
     return (np.abs(_normal(seed, stream, N)) * sigma * scale).astype(np.float16)
 
