@@ -9,7 +9,8 @@
 // streams them, besides the final look-up of z) reduces every later step to at most 2^v weighted patterns:
 //   histogram       cnt[p]                                     n atomic adds
 //   initial order   rank(p) = #{q : (cnt[q], -q) > (cnt[p], -p)}  (frequency descending, packed word ascending);
-//                   pattern p becomes centroid rank(p) when rank(p) < c
+//                   pattern p becomes centroid rank(p) when rank(p) < c; counted among the patterns at least as
+//                   frequent as the c-th most frequent one (threshold by bisection, then a candidate list)
 //   E-step          one thread per occurring pattern, centroids broadcast from shared memory;
 //                   min over k of (POPCNT << 16 | k) is the nearest centroid with the smallest index among equals
 //   M-step          per occurring pattern: add cnt[p] to the vote counters of its cluster; then one thread per centroid
@@ -26,6 +27,8 @@ struct KmState {
     int kc_eff;       // min(c, number of distinct vectors)
     int n_unique;
     int changed;      // set by the E-step of the current round
+    unsigned thr;     // frequency of the c-th most frequent distinct vector (1 when there are fewer than c)
+    int n_cand;       // distinct vectors at least that frequent: the candidates for the initial codebook
 };
 
 struct KmWorkspace {
@@ -34,6 +37,8 @@ struct KmWorkspace {
     uint32_t *label;      // [2][P], E-step i writes half i & 1
     uint32_t *tot;        // [Kc]
     uint32_t *ones;       // [Kc][16]
+    uint32_t *cand_p;     // [P] candidate patterns (unordered) ...
+    uint32_t *cand_c;     // [P] ... and their frequencies
 };
 
 __host__ __device__ inline size_t km_align(size_t x) { return (x + 255) & ~(size_t)255; }
@@ -47,14 +52,17 @@ static KmWorkspace km_carve(void *ws, int v, int Kc)
     w.cnt = reinterpret_cast<uint32_t *>(p); p += km_align(P * 4);
     w.label = reinterpret_cast<uint32_t *>(p); p += km_align(2 * P * 4);
     w.tot = reinterpret_cast<uint32_t *>(p); p += km_align((size_t)Kc * 4);
-    w.ones = reinterpret_cast<uint32_t *>(p);
+    w.ones = reinterpret_cast<uint32_t *>(p); p += km_align((size_t)Kc * 16 * 4);
+    w.cand_p = reinterpret_cast<uint32_t *>(p); p += km_align(P * 4);
+    w.cand_c = reinterpret_cast<uint32_t *>(p);
     return w;
 }
 
 static size_t km_workspace_bytes(int v, int Kc)
 {
     const size_t P = (size_t)1 << v;
-    return km_align(sizeof(KmState)) + km_align(P * 4) + km_align(2 * P * 4) + km_align((size_t)Kc * 4) + km_align((size_t)Kc * 16 * 4);
+    return km_align(sizeof(KmState)) + km_align(P * 4) + km_align(2 * P * 4) + km_align((size_t)Kc * 4) + km_align((size_t)Kc * 16 * 4) +
+           2 * km_align(P * 4);
 }
 
 __global__ void km_hist_kernel(const uint32_t *__restrict__ vecs, size_t n, uint32_t mask, uint32_t *__restrict__ cnt)
@@ -64,36 +72,95 @@ __global__ void km_hist_kernel(const uint32_t *__restrict__ vecs, size_t n, uint
     for (; i < n; i += stride) atomicAdd(cnt + (vecs[i] & mask), 1u);
 }
 
-// Initial centroids: occurring pattern p goes to slot rank(p) if that is below c.  Keys (cnt, P - 1 - p) are distinct, so
-// the ranks are a permutation of 0 .. n_unique - 1.
+// Initial centroids: occurring pattern p goes to slot rank(p) if that is below c, where rank counts the patterns that
+// are more frequent, or as frequent with a smaller packed word.  Only patterns at least as frequent as the c-th most
+// frequent one can get a slot, and only those can rank before one another, so the ranking runs over that candidate
+// list (about c entries when frequencies differ, all occurring patterns when they do not) instead of all 2^v patterns.
 constexpr int KM_TILE = 2048;
-__global__ void __launch_bounds__(256)
-km_init_rank_kernel(const uint32_t *__restrict__ cnt, int P, int Kc, uint32_t *__restrict__ C, KmState *st)
+
+// One CTA: number of distinct vectors, and the largest threshold t with #{p : cnt[p] >= t} >= c (bisection over t).
+__global__ void __launch_bounds__(1024)
+km_threshold_kernel(const uint32_t *__restrict__ cnt, int P, int Kc, KmState *st)
 {
-    __shared__ uint32_t s_cnt[KM_TILE];
-    const int p = blockIdx.x * blockDim.x + threadIdx.x;
-    const uint32_t mine = (p < P) ? cnt[p] : 0u;
-    int rank = 0;
-    for (int q0 = 0; q0 < P; q0 += KM_TILE) {
+    __shared__ unsigned s_red[32];
+    __shared__ unsigned s_val;
+    auto block_sum = [&](unsigned v) -> unsigned {
+        for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
         __syncthreads();
-        for (int i = threadIdx.x; i < KM_TILE; i += blockDim.x) s_cnt[i] = (q0 + i < P) ? cnt[q0 + i] : 0u;
+        if ((threadIdx.x & 31) == 0) s_red[threadIdx.x >> 5] = v;
         __syncthreads();
-        if (mine) {
-            const int lim = min(KM_TILE, P - q0);
-            for (int i = 0; i < lim; ++i) {
-                const uint32_t c = s_cnt[i];
-                // q = q0 + i ranks before p when it is more frequent, or as frequent with a smaller packed word
-                rank += (c > mine || (c == mine && q0 + i < p)) ? 1 : 0;
-            }
+        if (threadIdx.x < 32) {
+            unsigned w = s_red[threadIdx.x];
+            for (int o = 16; o > 0; o >>= 1) w += __shfl_xor_sync(0xffffffffu, w, o);
+            if (threadIdx.x == 0) s_val = w;
+        }
+        __syncthreads();
+        return s_val;
+    };
+    auto count_ge = [&](unsigned t) -> unsigned {
+        unsigned c = 0;
+        for (int p = threadIdx.x; p < P; p += blockDim.x) c += (cnt[p] >= t) ? 1u : 0u;
+        return block_sum(c);
+    };
+    unsigned mx = 0;
+    for (int p = threadIdx.x; p < P; p += blockDim.x) mx = max(mx, cnt[p]);
+    for (int o = 16; o > 0; o >>= 1) mx = max(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+    __syncthreads();
+    if ((threadIdx.x & 31) == 0) s_red[threadIdx.x >> 5] = mx;
+    __syncthreads();
+    mx = 0;
+    for (int i = 0; i < 32; ++i) mx = max(mx, s_red[i]);
+    const unsigned n_unique = count_ge(1u);
+    unsigned lo = 1u, hi = max(mx, 1u);                     // invariant: count_ge(lo) >= min(c, n_unique)
+    if (n_unique > (unsigned)Kc) {
+        while (lo < hi) {
+            const unsigned mid = lo + (hi - lo + 1u) / 2u;
+            if (count_ge(mid) >= (unsigned)Kc) lo = mid; else hi = mid - 1u;
         }
     }
-    if (mine) {
-        atomicAdd(&st->n_unique, 1);
-        if (rank < Kc) C[rank] = (uint32_t)p;
+    if (threadIdx.x == 0) {
+        st->n_unique = (int)n_unique;
+        st->kc_eff = min(Kc, (int)n_unique);
+        st->thr = (n_unique > (unsigned)Kc) ? lo : 1u;
     }
 }
 
-__global__ void km_init_finish_kernel(int Kc, KmState *st) { st->kc_eff = min(Kc, st->n_unique); }
+__global__ void km_candidates_kernel(const uint32_t *__restrict__ cnt, int P, uint32_t *__restrict__ cand_p, uint32_t *__restrict__ cand_c, KmState *st)
+{
+    const int p = blockIdx.x * blockDim.x + threadIdx.x;
+    if (p >= P) return;
+    const uint32_t c = cnt[p];
+    if (c != 0u && c >= st->thr) {
+        const int pos = atomicAdd(&st->n_cand, 1);
+        cand_p[pos] = (uint32_t)p;
+        cand_c[pos] = c;
+    }
+}
+
+__global__ void __launch_bounds__(256)
+km_init_rank_kernel(const uint32_t *__restrict__ cand_p, const uint32_t *__restrict__ cand_c, int Kc, uint32_t *__restrict__ C, const KmState *st)
+{
+    __shared__ uint32_t s_p[KM_TILE], s_c[KM_TILE];
+    const int L = st->n_cand;
+    if ((int)(blockIdx.x * blockDim.x) >= L) return;        // (uniform over the block)
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    const bool live = i < L;
+    const uint32_t p = live ? cand_p[i] : 0u, mine = live ? cand_c[i] : 0u;
+    int rank = 0;
+    for (int q0 = 0; q0 < L; q0 += KM_TILE) {
+        __syncthreads();
+        for (int j = threadIdx.x; j < KM_TILE; j += blockDim.x) {
+            s_p[j] = (q0 + j < L) ? cand_p[q0 + j] : 0u;
+            s_c[j] = (q0 + j < L) ? cand_c[q0 + j] : 0u;
+        }
+        __syncthreads();
+        if (live) {
+            const int lim = min(KM_TILE, L - q0);
+            for (int j = 0; j < lim; ++j) rank += (s_c[j] > mine || (s_c[j] == mine && s_p[j] < p)) ? 1 : 0;
+        }
+    }
+    if (live && rank < Kc) C[rank] = p;
+}
 
 __global__ void __launch_bounds__(256)
 km_estep_kernel(const uint32_t *__restrict__ cnt, int P, const uint32_t *__restrict__ C, uint32_t *__restrict__ label, KmState *st)
@@ -209,8 +276,9 @@ extern "C" BTC_API int btc_codebook_kmeans(const uint32_t *vecs, size_t n, int v
     const unsigned nb = (unsigned)((n + 255) / 256 < 148 * 32 ? (n + 255) / 256 : 148 * 32);
     const unsigned pb = (unsigned)((P + 255) / 256), kb = (unsigned)((Kc + 255) / 256);
     km_hist_kernel<<<nb, 256, 0, s>>>(vecs, n, mask, w.cnt);
-    km_init_rank_kernel<<<pb, 256, 0, s>>>(w.cnt, P, Kc, C_words, w.st);
-    km_init_finish_kernel<<<1, 1, 0, s>>>(Kc, w.st);
+    km_threshold_kernel<<<1, 1024, 0, s>>>(w.cnt, P, Kc, w.st);
+    km_candidates_kernel<<<pb, 256, 0, s>>>(w.cnt, P, w.cand_p, w.cand_c, w.st);
+    km_init_rank_kernel<<<pb, 256, 0, s>>>(w.cand_p, w.cand_c, Kc, C_words, w.st);
     for (int it = 0; it < max_iter; ++it) {
         km_estep_kernel<<<pb, 256, 0, s>>>(w.cnt, P, C_words, w.label, w.st);
         km_round_kernel<<<1, 1, 0, s>>>(w.st);
