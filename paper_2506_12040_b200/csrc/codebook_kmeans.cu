@@ -28,7 +28,8 @@ struct KmState {
     int n_unique;
     int changed;      // set by the E-step of the current round
     unsigned thr;     // frequency of the c-th most frequent distinct vector (1 when there are fewer than c)
-    int n_cand;       // distinct vectors at least that frequent: the candidates for the initial codebook
+    int n_cand;       // distinct vectors more frequent than that (fewer than c): ranked pairwise; the ones exactly that
+                      // frequent follow them in the order of their packed words
 };
 
 struct KmWorkspace {
@@ -74,8 +75,9 @@ __global__ void km_hist_kernel(const uint32_t *__restrict__ vecs, size_t n, uint
 
 // Initial centroids: occurring pattern p goes to slot rank(p) if that is below c, where rank counts the patterns that
 // are more frequent, or as frequent with a smaller packed word.  Only patterns at least as frequent as the c-th most
-// frequent one can get a slot, and only those can rank before one another, so the ranking runs over that candidate
-// list (about c entries when frequencies differ, all occurring patterns when they do not) instead of all 2^v patterns.
+// frequent one can get a slot.  Those strictly more frequent (fewer than c) are ranked against one another; those
+// exactly as frequent (possibly many: frequencies of rare patterns tie) come after them in word order, which is a
+// prefix count, not a comparison of pairs.
 constexpr int KM_TILE = 2048;
 
 // One CTA: number of distinct vectors, and the largest threshold t with #{p : cnt[p] >= t} >= c (bisection over t).
@@ -130,36 +132,64 @@ __global__ void km_candidates_kernel(const uint32_t *__restrict__ cnt, int P, ui
     const int p = blockIdx.x * blockDim.x + threadIdx.x;
     if (p >= P) return;
     const uint32_t c = cnt[p];
-    if (c != 0u && c >= st->thr) {
+    if (c > st->thr) {                                      // strictly more frequent than the c-th: fewer than c of them
         const int pos = atomicAdd(&st->n_cand, 1);
         cand_p[pos] = (uint32_t)p;
         cand_c[pos] = c;
     }
 }
 
-__global__ void __launch_bounds__(256)
+// (frequency, word) of a candidate as one key: larger key = earlier slot.
+__device__ __forceinline__ unsigned long long km_key(uint32_t c, uint32_t p) { return ((unsigned long long)c << 32) | (0xffffffffu - p); }
+
+constexpr int KM_RANK_THREADS = 64;                         // small blocks: a few thousand candidates should still fill the SMs
+__global__ void __launch_bounds__(KM_RANK_THREADS)
 km_init_rank_kernel(const uint32_t *__restrict__ cand_p, const uint32_t *__restrict__ cand_c, int Kc, uint32_t *__restrict__ C, const KmState *st)
 {
-    __shared__ uint32_t s_p[KM_TILE], s_c[KM_TILE];
+    __shared__ __align__(16) unsigned long long s_key[KM_TILE];
     const int L = st->n_cand;
     if ((int)(blockIdx.x * blockDim.x) >= L) return;        // (uniform over the block)
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
     const bool live = i < L;
-    const uint32_t p = live ? cand_p[i] : 0u, mine = live ? cand_c[i] : 0u;
+    const uint32_t p = live ? cand_p[i] : 0u;
+    const unsigned long long mine = live ? km_key(cand_c[i], p) : ~0ull;
     int rank = 0;
     for (int q0 = 0; q0 < L; q0 += KM_TILE) {
         __syncthreads();
-        for (int j = threadIdx.x; j < KM_TILE; j += blockDim.x) {
-            s_p[j] = (q0 + j < L) ? cand_p[q0 + j] : 0u;
-            s_c[j] = (q0 + j < L) ? cand_c[q0 + j] : 0u;
-        }
+        for (int j = threadIdx.x; j < KM_TILE; j += blockDim.x)
+            s_key[j] = (q0 + j < L) ? km_key(cand_c[q0 + j], cand_p[q0 + j]) : 0ull;     // (key 0 ranks before nothing)
         __syncthreads();
-        if (live) {
-            const int lim = min(KM_TILE, L - q0);
-            for (int j = 0; j < lim; ++j) rank += (s_c[j] > mine || (s_c[j] == mine && s_p[j] < p)) ? 1 : 0;
-        }
+#pragma unroll 8
+        for (int j = 0; j < KM_TILE; ++j) rank += (s_key[j] > mine) ? 1 : 0;
     }
     if (live && rank < Kc) C[rank] = p;
+}
+
+// The patterns exactly as frequent as the c-th most frequent one follow the strictly more frequent ones in the order
+// of their packed words: rank = n_cand + (number of such patterns with a smaller word), a prefix count over p.
+__global__ void __launch_bounds__(1024)
+km_ties_kernel(const uint32_t *__restrict__ cnt, int P, int Kc, uint32_t *__restrict__ C, const KmState *st)
+{
+    __shared__ int s_off[1024];
+    const unsigned thr = st->thr;
+    const int per = (P + 1023) / 1024;
+    const int p0 = threadIdx.x * per, p1 = min(P, p0 + per);
+    int mine = 0;
+    for (int p = p0; p < p1; ++p) mine += (cnt[p] == thr) ? 1 : 0;
+    s_off[threadIdx.x] = mine;
+    __syncthreads();
+    for (int o = 1; o < 1024; o <<= 1) {                    // inclusive scan
+        const int add = (threadIdx.x >= o) ? s_off[threadIdx.x - o] : 0;
+        __syncthreads();
+        s_off[threadIdx.x] += add;
+        __syncthreads();
+    }
+    int rank = st->n_cand + s_off[threadIdx.x] - mine;
+    for (int p = p0; p < p1; ++p)
+        if (cnt[p] == thr) {
+            if (rank < Kc) C[rank] = (uint32_t)p;
+            ++rank;
+        }
 }
 
 __global__ void __launch_bounds__(256)
@@ -278,7 +308,8 @@ extern "C" BTC_API int btc_codebook_kmeans(const uint32_t *vecs, size_t n, int v
     km_hist_kernel<<<nb, 256, 0, s>>>(vecs, n, mask, w.cnt);
     km_threshold_kernel<<<1, 1024, 0, s>>>(w.cnt, P, Kc, w.st);
     km_candidates_kernel<<<pb, 256, 0, s>>>(w.cnt, P, w.cand_p, w.cand_c, w.st);
-    km_init_rank_kernel<<<pb, 256, 0, s>>>(w.cand_p, w.cand_c, Kc, C_words, w.st);
+    km_init_rank_kernel<<<(unsigned)((P + KM_RANK_THREADS - 1) / KM_RANK_THREADS), KM_RANK_THREADS, 0, s>>>(w.cand_p, w.cand_c, Kc, C_words, w.st);
+    km_ties_kernel<<<1, 1024, 0, s>>>(w.cnt, P, Kc, C_words, w.st);
     for (int it = 0; it < max_iter; ++it) {
         km_estep_kernel<<<pb, 256, 0, s>>>(w.cnt, P, C_words, w.label, w.st);
         km_round_kernel<<<1, 1, 0, s>>>(w.st);
