@@ -225,6 +225,37 @@ def test_gemv_batch_large_codebooks_16bit_table(M):
     assert btc.device_status() == 0
 
 
+@pytest.mark.parametrize("Kc,dist", [(4096, "uniform"), (256, "uniform"), (65536, "uniform"), (4096, "zipf")])
+def test_chained_decode_blocks_with_teacher_forcing(Kc, dist):
+    """The dependent decode chain in the launch grouping the benchmark times ({q,k,v}, o, {gate,up}, down; fp16
+    outputs feed the next launch), two blocks at full layer sizes: every layer's output against the oracle evaluated
+    on the fp16 activations the chain actually handed to that layer."""
+    cfg5 = wl.config_layers(5, Kc=Kc, idx_dist=dist)
+    sp = cfg5["layers"]
+    Ls = [wl.make_layer(s5, 1, cfg5["seed"], i) for i, s5 in enumerate(sp)]
+    ds = [to_device(L) for L in Ls]
+    lay = [dict(idx=d["idx"], C_packed=d["Cp"], alpha=d["alpha"], v=L.spec.v, Kc=L.spec.Kc) for L, d in zip(Ls, ds)]
+    h = ds[0]["x"][:1].clone()
+    f16 = lambda n: torch.empty((1, n), dtype=torch.float16, device="cuda")
+    for blk in range(2):
+        qkv = [f16(4096) for _ in range(3)]
+        o_out, gu, nxt = f16(4096), [f16(11008) for _ in range(2)], f16(4096)
+        steps = [([0, 1, 2], h, qkv), ([3], qkv[0], [o_out]), ([4, 5], o_out, gu), ([6], gu[0], [nxt])]
+        for ids, xin, outs in steps:
+            btc.GemvBatch([dict(x=xin, out=o, **lay[i]) for i, o in zip(ids, outs)]).run()
+            torch.cuda.synchronize()
+            x64 = xin.double().cpu().numpy()
+            assert np.isfinite(x64).all()
+            for i, o in zip(ids, outs):
+                want = oracle.linear(x64, Ls[i].idx, Ls[i].C_pm1, Ls[i].alpha, None)
+                got = o.double().cpu().numpy()
+                # the output is the fp32 result rounded to fp16: half an fp16 ulp on top of the decode tolerance
+                tol = TOL_GEMV * np.abs(want).max() + 2.0 ** -11 * np.abs(want)
+                assert (np.abs(got - want) <= tol).all(), (Kc, dist, blk, i, float(np.abs(got - want).max()), float(np.abs(want).max()))
+        h = nxt
+    assert btc.device_status() == 0
+
+
 # ------------------------------------------------------------------ online activation transform
 
 @pytest.mark.parametrize("path,M,k1,k2", [("gemv", 2, 32, 32), ("gemv", 1, 64, 64), ("gemm", 96, 16, 64), ("gemv", 8, 8, 40)])
