@@ -106,7 +106,7 @@ BTC_API int btc_codebook_pack_host(const int8_t *C_pm1_host, int Kc, int v, uint
  *   workspace device, btc_codebook_kmeans_workspace_bytes(v, Kc) bytes, 256-byte aligned
  * Integer arithmetic only: the result is unique.  Work is enqueued on `stream`, nothing is
  * allocated, nothing synchronises (the loop is max_iter rounds of launches; rounds after the
- * last one return at once).  v <= 16 (the steps run over the 2^v patterns); 16 < v <= 32 returns
+ * last one return at once).  v <= 20 (the steps keep tables of 2^v entries); 20 < v <= 32 returns
  * BTC_ERR_UNSUPPORTED.  1 <= Kc <= 65536, 1 <= n < 2^31, 1 <= max_iter <= 4096. */
 BTC_API size_t btc_codebook_kmeans_workspace_bytes(int v, int Kc);
 BTC_API int btc_codebook_kmeans(const uint32_t *vecs, size_t n, int v, int Kc, int max_iter, uint32_t *C_words,

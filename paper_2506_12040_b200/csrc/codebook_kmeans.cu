@@ -4,7 +4,8 @@
 //   M-step  c_k = element-wise majority of the vectors assigned to k  (ties -> +1; an empty cluster keeps its centroid)
 // until no assignment changes or max_iter E-steps have run.
 //
-// Everything is done in the space of the 2^v possible patterns (v <= 16, so at most 65536 of them), not per vector:
+// Everything is done in the space of the 2^v possible patterns (v <= 20: the paper's range; 65536 of them at v = 16),
+// not per vector:
 // identical vectors have identical nearest centroids, so one histogram pass over the n vectors (the only pass that
 // streams them, besides the final look-up of z) reduces every later step to at most 2^v weighted patterns:
 //   histogram       cnt[p]                                     n atomic adds
@@ -20,6 +21,9 @@
 #include "btc_internal.cuh"
 
 namespace btc {
+
+constexpr int KM_VMAX = 20;                  // longest vector: the steps keep tables of 2^v entries
+constexpr int KM_VMAX_SLOTS = 32;            // vote counters per centroid
 
 struct KmState {
     int done;         // 1: assignments unchanged in an E-step (the loop has ended)
@@ -37,7 +41,7 @@ struct KmWorkspace {
     uint32_t *cnt;        // [P]
     uint32_t *label;      // [2][P], E-step i writes half i & 1
     uint32_t *tot;        // [Kc]
-    uint32_t *ones;       // [Kc][16]
+    uint32_t *ones;       // [Kc][KM_VMAX_SLOTS]
     uint32_t *cand_p;     // [P] candidate patterns (unordered) ...
     uint32_t *cand_c;     // [P] ... and their frequencies
 };
@@ -53,7 +57,7 @@ static KmWorkspace km_carve(void *ws, int v, int Kc)
     w.cnt = reinterpret_cast<uint32_t *>(p); p += km_align(P * 4);
     w.label = reinterpret_cast<uint32_t *>(p); p += km_align(2 * P * 4);
     w.tot = reinterpret_cast<uint32_t *>(p); p += km_align((size_t)Kc * 4);
-    w.ones = reinterpret_cast<uint32_t *>(p); p += km_align((size_t)Kc * 16 * 4);
+    w.ones = reinterpret_cast<uint32_t *>(p); p += km_align((size_t)Kc * KM_VMAX_SLOTS * 4);
     w.cand_p = reinterpret_cast<uint32_t *>(p); p += km_align(P * 4);
     w.cand_c = reinterpret_cast<uint32_t *>(p);
     return w;
@@ -62,7 +66,7 @@ static KmWorkspace km_carve(void *ws, int v, int Kc)
 static size_t km_workspace_bytes(int v, int Kc)
 {
     const size_t P = (size_t)1 << v;
-    return km_align(sizeof(KmState)) + km_align(P * 4) + km_align(2 * P * 4) + km_align((size_t)Kc * 4) + km_align((size_t)Kc * 16 * 4) +
+    return km_align(sizeof(KmState)) + km_align(P * 4) + km_align(2 * P * 4) + km_align((size_t)Kc * 4) + km_align((size_t)Kc * KM_VMAX_SLOTS * 4) +
            2 * km_align(P * 4);
 }
 
@@ -246,7 +250,7 @@ __global__ void km_vote_kernel(const uint32_t *__restrict__ cnt, int P, int v, c
     const uint32_t k = label[(size_t)((st->iters - 1) & 1) * P + p];     // the E-step just counted wrote half (iters - 1) & 1
     atomicAdd(tot + k, c);
     for (int t = 0; t < v; ++t)
-        if ((p >> t) & 1) atomicAdd(ones + (size_t)k * 16 + t, c);
+        if ((p >> t) & 1) atomicAdd(ones + (size_t)k * KM_VMAX_SLOTS + t, c);
 }
 
 __global__ void km_update_kernel(int v, uint32_t *__restrict__ C, uint32_t *__restrict__ tot, uint32_t *__restrict__ ones, const KmState *st)
@@ -258,9 +262,9 @@ __global__ void km_update_kernel(int v, uint32_t *__restrict__ C, uint32_t *__re
     if (n) {
         uint32_t w = 0;
         for (int t = 0; t < v; ++t) {
-            const uint32_t o = ones[(size_t)k * 16 + t];
+            const uint32_t o = ones[(size_t)k * KM_VMAX_SLOTS + t];
             if (o >= n - o) w |= 1u << t;                   // at least as many +1 as -1: sign(0) = +1
-            ones[(size_t)k * 16 + t] = 0;
+            ones[(size_t)k * KM_VMAX_SLOTS + t] = 0;
         }
         C[k] = w;
         tot[k] = 0;
@@ -283,7 +287,7 @@ using namespace btc;
 
 extern "C" BTC_API size_t btc_codebook_kmeans_workspace_bytes(int v, int Kc)
 {
-    if (v < 1 || v > 16 || Kc < 1 || Kc > 65536) return 0;
+    if (v < 1 || v > KM_VMAX || Kc < 1 || Kc > 65536) return 0;
     return km_workspace_bytes(v, Kc);
 }
 
@@ -292,7 +296,7 @@ extern "C" BTC_API int btc_codebook_kmeans(const uint32_t *vecs, size_t n, int v
 {
     if (!vecs || !C_words || !z || !info || !workspace) return BTC_ERR_NULL;
     if (Kc < 1 || Kc > 65536 || n < 1 || n > 0x7fffffffull || max_iter < 1 || max_iter > 4096 || v < 1 || v > 32) return BTC_ERR_SHAPE;
-    if (v > 16) return BTC_ERR_UNSUPPORTED;                  // the pattern-space steps keep 2^v entries
+    if (v > KM_VMAX) return BTC_ERR_UNSUPPORTED;             // the pattern-space steps keep 2^v entries
     if (workspace_bytes < km_workspace_bytes(v, Kc)) return BTC_ERR_WORKSPACE;
     if (reinterpret_cast<uintptr_t>(workspace) % 256) return BTC_ERR_ALIGN;
     cudaStream_t s = (cudaStream_t)stream;

@@ -46,6 +46,8 @@ CASES = [
     (2000, 9, 50, 10, "few"),            # fewer distinct vectors than centroids
     (1, 5, 3, 4, "iid"),
     (70000, 13, 5000, 6, "noisy"),       # ragged: many tiles of centroids and patterns
+    (30000, 20, 700, 8, "noisy"),        # the longest vectors of the paper's range
+    (9000, 18, 3000, 5, "iid"),
 ]
 
 
@@ -81,7 +83,7 @@ def test_kmeans_feeds_the_layer():
 def test_kmeans_argument_errors():
     w = torch.zeros(16, dtype=torch.int32, device="cuda")
     with pytest.raises(btc.BtcError):
-        btc.codebook_kmeans(w, 20, 16, 5)            # v > 16: unsupported
+        btc.codebook_kmeans(w, 24, 16, 5)            # v > 20: unsupported
     with pytest.raises(btc.BtcError):
         btc.codebook_kmeans(w, 8, 0, 5)
     with pytest.raises(btc.BtcError):
