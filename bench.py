@@ -259,6 +259,20 @@ def run_gpu(args):
                "frac_of_nominal": achieved / 8000.0}
 
     if rank == 0 and not args.quick:
+        # ---- one isolated launch of the step (no graph, L2 flushed by writing a buffer larger than L2 before it)
+        flush = torch.empty(2 * l2, dtype=torch.uint8, device=dev)
+        iso = []
+        for k in range(12):
+            flush.zero_()
+            e0 = torch.cuda.Event(enable_timing=True)
+            e1 = torch.cuda.Event(enable_timing=True)
+            e0.record()
+            step1(k % R)
+            e1.record()
+            torch.cuda.synchronize()
+            iso.append(e0.elapsed_time(e1) * 1e3)
+        details["isolated_step_us_M1"] = float(np.median(iso[2:]))
+        del flush
         # ---- per shape, M in {1, 8}, each over its own rotating sets
         def time_shape(i, M, reps=200):
             s = specs[i]
