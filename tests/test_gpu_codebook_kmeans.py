@@ -48,6 +48,9 @@ CASES = [
     (70000, 13, 5000, 6, "noisy"),       # ragged: many tiles of centroids and patterns
     (30000, 20, 700, 8, "noisy"),        # the longest vectors of the paper's range
     (9000, 18, 3000, 5, "iid"),
+    (100, 1, 2, 3, "iid"),               # one element per vector: two patterns
+    (1000, 6, 1, 5, "noisy"),            # a single centroid: the bitwise majority
+    (500, 16, 65536, 3, "iid"),          # the largest codebook, far more slots than vectors
 ]
 
 
