@@ -313,6 +313,15 @@ def run_gpu(args):
             for M in (1, 8):
                 details.setdefault(f"per_shape_M{M}", {})[f"{s.N}x{s.K}"] = time_shape(i, M)
 
+        # ---- the whole step (one fused launch) with more rows of x
+        step_m = {}
+        for M in (2, 4, 8):
+            stepM, _, _ = make_runner(M)
+            tM = time_steps(stepM, 60, 5) / 60
+            bM = sum(algorithmic_bytes(s, M) for s in specs)
+            step_m[f"M{M}"] = {"us": tM * 1e6, "GBps": bM / tM * 1e-9, "frac_measured": bM / tM * 1e-9 / peaks["hbm_gbs"]}
+        details["step_by_M"] = step_m
+
         # ---- tensor-core path, config 4 shapes, with a cuBLAS fp16 GEMM of the same shape as context
         gem = {}
         c4 = wl.CONFIGS[4]
