@@ -123,7 +123,9 @@ BTC_API int btc_codebook_kmeans(const uint32_t *vecs, size_t n, int v, int Kc, i
  *   y        [M, N] row-major, y_dtype = BTC_F32 (also BTC_F16 / BTC_BF16, rounded to nearest)
  *   workspace / workspace_bytes: scratch of at least btc_linear_workspace_bytes(...) bytes,
  *            256-byte aligned; may be NULL when that function returns 0.  Contents are
- *            undefined afterwards; concurrent calls need distinct workspaces.
+ *            undefined afterwards; concurrent calls need distinct workspaces.  For a layer with
+ *            few 128-row tiles and a long K (v = 16) the size includes room for the partial sums
+ *            of a K split over the idle SMs, added in a fixed order by a second small kernel.
  *
  * btc_linear_gemv: the decode path, 1 <= M <= 8, built on the identity <x, c> = 2 * sum_{bit=1} x - sum x.
  *   M <= 2: x is quantised per K-slice to a block-fixed-point integer (2^-20 of the slice's largest magnitude
@@ -188,9 +190,9 @@ BTC_API int btc_linear_gemv_batch(const btc_linear_problem *problems, int count,
  * the library holds that array until the process exits.
  *
  * Arguments are those of btc_linear_gemm without workspace / workspace_bytes.  Differences:
- *   - Needs btc_linear_workspace_bytes(M, N, K, v, Kc) <= BTC_STATIC_SCRATCH_BYTES, i.e.
- *     M <= BTC_STATIC_SCRATCH_BYTES / 4 rows of x; larger M returns BTC_ERR_WORKSPACE and nothing
- *     is launched.  T must be NULL (the transform needs M*K*2 bytes more): BTC_ERR_UNSUPPORTED.
+ *   - Needs 4*M <= BTC_STATIC_SCRATCH_BYTES, i.e. M <= BTC_STATIC_SCRATCH_BYTES / 4 rows of x;
+ *     larger M returns BTC_ERR_WORKSPACE and nothing is launched.  K is never split here (the
+ *     array has no room for partial sums).  T must be NULL (the transform needs M*K*2 bytes more): BTC_ERR_UNSUPPORTED.
  *   - The first call on each device looks up the array's device address (no allocation, no
  *     launch) and caches it; make that first call outside any stream capture.  The device that is
  *     current at the call is the one used, as for every other entry point.

@@ -36,7 +36,10 @@ static int run_linear(Path path, const void *x, int x_dt, const uint16_t *idx, c
     if (rc != BTC_OK) return rc;
     if (mu && !aligned(mu, 2)) return BTC_ERR_ALIGN;
     if (path == PATH_GEMV && M > 8) return BTC_ERR_SHAPE;
-    const size_t need = btc_linear_workspace_bytes(M, N, K, v, Kc);
+    // (btc_linear_workspace_bytes may ask for more: room for a K split, which the kernels do without when it is missing)
+    size_t need = (M <= 8) ? gemv_decode_workspace_bytes(M, N, K, v, Kc) : 0;
+    if (gemm_tcgen05_workspace_min(M) > need) need = gemm_tcgen05_workspace_min(M);
+    need = (need + 255) / 256 * 256;
     const size_t xt_bytes = T ? (((size_t)M * K * 2 + 255) / 256) * 256 : 0;
     if (need + xt_bytes > 0) {
         if (!ws || ws_bytes < need + xt_bytes) return BTC_ERR_WORKSPACE;

@@ -38,7 +38,8 @@ size_t gemv_decode_workspace_bytes(int M, int N, int K, int v, int Kc);
 
 // gemm_tcgen05.cu: tensor-core path.  Same UNSUPPORTED convention.
 int launch_gemm_tcgen05(const LinearArgs &a, cudaStream_t s);
-size_t gemm_tcgen05_workspace_bytes(int M, int N, int K, int v, int Kc);
+size_t gemm_tcgen05_workspace_bytes(int M, int N, int K, int v, int Kc);   // with room for a K split where one pays
+size_t gemm_tcgen05_workspace_min(int M);                                 // what the kernels cannot do without
 
 // gemv_imma.cu: integer-MMA decode path; runs up to IM_MAXP independent layers (M <= 8 each) in one launch.
 // Returns BTC_ERR_UNSUPPORTED when a shape is outside what it covers (nothing is launched then).

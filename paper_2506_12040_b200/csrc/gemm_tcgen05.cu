@@ -304,6 +304,11 @@ struct Gemm2Params {
     int tab_bytes;           // > 0: table staged in shared memory
 };
 
+struct SplitArgs {
+    int split_tiles;         // k tiles (a multiple of 16: whole index tiles) per CTA along grid.z
+    float *part;             // raw partial sums [grid.z][M][N]
+};
+
 __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar) {
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                  ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
@@ -342,9 +347,11 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32
 }
 __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
-template <int BM, int STAGES, int KS>
+// SPLIT: the CTAs of a tile share K along grid.z and leave raw partial sums in p.part (a separate instantiation, so
+// that the unsplit kernel carries none of it).
+template <int BM, int STAGES, int KS, bool SPLIT>
 __global__ void __launch_bounds__(G2_THREADS, 1)
-gemm_v16t_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_i, const Gemm2Params p)
+gemm_v16t_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_i, const Gemm2Params p, const SplitArgs sp)
 {
     constexpr uint32_t B_BYTES = BM * G_BK * 2;                    // one x tile (64 k); a stage holds KS of them
     constexpr uint32_t STAGE_BYTES = KS * B_BYTES;
@@ -371,7 +378,9 @@ gemm_v16t_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
     const LinearArgs &a = p.a;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int n0 = blockIdx.x * G_BN, m0 = blockIdx.y * BM;
-    const int KT = p.k_tiles;
+    // a CTA covers the k tiles [kt_first, kt_first + KT): all of them, or its share along grid.z (whole index tiles)
+    const int kt_first = SPLIT ? blockIdx.z * sp.split_tiles : 0;
+    const int KT = SPLIT ? min(sp.split_tiles, p.k_tiles - kt_first) : p.k_tiles;
     const int NS = (KT + KS - 1) / KS;                              // stages' worth of k steps
     const bool is_bf16 = (a.x_dt == BTC_BF16);
     auto bar_full = [&](int s) { return smem_u32(bars + s); };
@@ -407,14 +416,14 @@ gemm_v16t_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                     const int it = kt0 >> 4, ib = it & 1;
                     if (it >= 2 && !mbar_wait(bar_empty_i(ib), ((it >> 1) & 1) ^ 1, s_abort)) break;
                     mbar_expect_tx(bar_full_i(ib), G2_IDX_BYTES);
-                    tma_load_2d(smem_u32(s_idx + (size_t)ib * G2_IDX_BYTES), &tmap_i, it * 64, n0, bar_full_i(ib));
+                    tma_load_2d(smem_u32(s_idx + (size_t)ib * G2_IDX_BYTES), &tmap_i, (kt_first >> 4) * 64 + it * 64, n0, bar_full_i(ib));
                 }
                 const int s = ks % STAGES;
                 if (ks >= STAGES && !mbar_wait(bar_empty(s), ((ks / STAGES) & 1) ^ 1, s_abort)) break;
                 mbar_expect_tx(bar_full(s), STAGE_BYTES);
 #pragma unroll
                 for (int j = 0; j < KS; ++j)             // (a box past K arrives as zeros)
-                    tma_load_2d(smem_base + s * STAGE_BYTES + j * B_BYTES, &tmap_x, (kt0 + j) * G_BK, m0, bar_full(s));
+                    tma_load_2d(smem_base + s * STAGE_BYTES + j * B_BYTES, &tmap_x, (kt_first + kt0 + j) * G_BK, m0, bar_full(s));
             }
         }
     } else if (warp == 1 || (NACC == 2 && warp == 3)) {
@@ -516,9 +525,13 @@ gemm_v16t_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                     for (int i = 0; i < 32; ++i) {
                         const int m = m0 + c0 + i;
                         if (m < a.M) {
-                            float y = al * __uint_as_float(rr[i]);
-                            if (a.mu) y += mu * p.sumx[m];
-                            store_from_float(a.y, a.y_dt, (size_t)m * a.N + nrow, y);
+                            if (SPLIT) {                           // K split: the reduce kernel applies alpha and mu
+                                sp.part[((size_t)blockIdx.z * a.M + m) * a.N + nrow] = __uint_as_float(rr[i]);
+                            } else {
+                                float y = al * __uint_as_float(rr[i]);
+                                if (a.mu) y += mu * p.sumx[m];
+                                store_from_float(a.y, a.y_dt, (size_t)m * a.N + nrow, y);
+                            }
                         }
                     }
                 }
@@ -532,6 +545,21 @@ gemm_v16t_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
         __syncthreads();
     }
     if (warp == 2) tmem_dealloc(tmem_d, 512);
+}
+
+// y = alpha * (sum of the K splits' partial sums, in split order) + mu * sum_k x.
+__global__ void splitk_reduce_kernel(const float *__restrict__ part, int splits, int M, int N, const __half *__restrict__ alpha,
+                                     const __half *__restrict__ mu, const float *__restrict__ sumx, void *__restrict__ y, int y_dt)
+{
+    const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const size_t MN = (size_t)M * N;
+    if (i >= MN) return;
+    const int n = (int)(i % N), m = (int)(i / N);
+    float acc = 0.f;
+    for (int z = 0; z < splits; ++z) acc += part[(size_t)z * MN + i];
+    float v = __half2float(alpha[n]) * acc;
+    if (mu) v += __half2float(mu[n]) * sumx[m];
+    store_from_float(y, y_dt, i, v);
 }
 
 // ------------------------------------------------------------------------------------ host side
@@ -565,22 +593,58 @@ static int launch_cfg(const CUtensorMap &tm, const GemmParams &p, cudaStream_t s
     return cuda_check_launch();
 }
 
-template <int BM, int STAGES, int KS>
-static int launch_v16t(const CUtensorMap &tm, const CUtensorMap &ti, const Gemm2Params &p, cudaStream_t s)
+template <int BM, int STAGES, int KS, bool SPLIT>
+static int launch_v16t(const CUtensorMap &tm, const CUtensorMap &ti, const Gemm2Params &p, const SplitArgs &sp, cudaStream_t s)
 {
     const size_t smem = (size_t)STAGES * KS * (BM * G_BK * 2) + 1024 + 2 * G2_IDX_BYTES + ((p.tab_bytes + 15) & ~15) +
                         (2 * STAGES + 6) * 8 + 16;
-    auto kern = gemm_v16t_kernel<BM, STAGES, KS>;
+    auto kern = gemm_v16t_kernel<BM, STAGES, KS, SPLIT>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return cuda_fail(e);
-    dim3 grid((p.a.N + G_BN - 1) / G_BN, (p.a.M + BM - 1) / BM);
-    kern<<<grid, G2_THREADS, smem, s>>>(tm, ti, p);
+    dim3 grid((p.a.N + G_BN - 1) / G_BN, (p.a.M + BM - 1) / BM, SPLIT ? (p.k_tiles + sp.split_tiles - 1) / sp.split_tiles : 1);
+    kern<<<grid, G2_THREADS, smem, s>>>(tm, ti, p, sp);
     return cuda_check_launch();
 }
 
-size_t gemm_tcgen05_workspace_bytes(int M, int, int, int, int)
+// K splits for a launch of `tiles` CTAs over `k_tiles` k tiles: as many as keep the grid within the SM count, each a
+// whole number of index tiles (16 k tiles) and at least two of them long.  Returns k tiles per split.
+static int splitk_tiles(int tiles, int k_tiles, int *splits)
+{
+    *splits = 1;
+    if (tiles > 74 || k_tiles < 64) return k_tiles;
+    int want = 148 / tiles;
+    if (want > 8) want = 8;
+    int per = ((k_tiles + want - 1) / want + 15) / 16 * 16;
+    if (per < 32) per = 32;
+    const int n = (k_tiles + per - 1) / per;
+    if (n < 2) return k_tiles;
+    *splits = n;
+    return per;
+}
+
+// Tile width in rows of x for a (M, N) problem: 256 when that still gives enough tiles to fill the machine.
+static int gemm_bm(int M, int N)
+{
+    return (M > 128 && (long long)((M + 255) / 256) * ((N + 127) / 128) >= 120) ? 256 : 128;
+}
+
+size_t gemm_tcgen05_workspace_min(int M)
 {
     return M > 8 ? (size_t)M * sizeof(float) : 0;   // row sums of x for the mean term
+}
+
+// The minimum plus, where the launch would otherwise leave most SMs idle (v = 16, few tiles, long K), room for the
+// partial sums of a K split.  With less than this (but at least the minimum) the kernels run without the split.
+size_t gemm_tcgen05_workspace_bytes(int M, int N, int K, int v, int)
+{
+    size_t w = gemm_tcgen05_workspace_min(M);
+    if (M > 8 && v == 16 && (K / v) % 8 == 0) {
+        const int BM = gemm_bm(M, N);
+        int splits = 1;
+        splitk_tiles(((N + 127) / 128) * ((M + BM - 1) / BM), (K + G_BK - 1) / G_BK, &splits);
+        if (splits > 1) w = ((w + 255) & ~(size_t)255) + (size_t)splits * M * N * sizeof(float);
+    }
+    return w;
 }
 
 int launch_gemm_tcgen05(const LinearArgs &a, cudaStream_t s)
@@ -589,7 +653,7 @@ int launch_gemm_tcgen05(const LinearArgs &a, cudaStream_t s)
     if (a.K % 8) return BTC_ERR_UNSUPPORTED;                   // TMA row pitch must be a multiple of 16 bytes
     encode_tiled_fn enc = get_encode();
     if (!enc) return BTC_ERR_UNSUPPORTED;
-    const int BM = (a.M > 128 && (long long)((a.M + 255) / 256) * ((a.N + 127) / 128) >= 120) ? 256 : 128;
+    const int BM = gemm_bm(a.M, a.N);
 
     CUtensorMap tm;
     const cuuint64_t dims[2] = {(cuuint64_t)a.K, (cuuint64_t)a.M};
@@ -629,8 +693,26 @@ int launch_gemm_tcgen05(const LinearArgs &a, cudaStream_t s)
             // shared memory holds only x tiles (4 stages of 32 KB either way), index tiles and the table
             const size_t fixed_t = (size_t)4 * (256 * G_BK * 2) + 1024 + 2 * G2_IDX_BYTES + 512;
             q.tab_bytes = (fixed_t + (size_t)Kc4 * 4 <= 227u * 1024u) ? Kc4 * 4 : 0;
-            if (BM == 256) return launch_v16t<256, 4, 1>(tm, ti, q, s);
-            return launch_v16t<128, 4, 2>(tm, ti, q, s);
+            // few tiles and a long K: split K over the idle SMs when the caller's workspace has room for the partial sums
+            SplitArgs sp = {q.k_tiles, nullptr};
+            int splits = 1;
+            const int per = splitk_tiles(((a.N + 127) / 128) * ((a.M + BM - 1) / BM), q.k_tiles, &splits);
+            if (splits > 1) {
+                const size_t off = (gemm_tcgen05_workspace_min(a.M) + 255) & ~(size_t)255;
+                const size_t need = off + (size_t)splits * a.M * a.N * sizeof(float);
+                if (a.workspace && a.workspace_bytes >= need && reinterpret_cast<uintptr_t>(a.workspace) % 16 == 0) {
+                    sp.split_tiles = per;
+                    sp.part = reinterpret_cast<float *>(static_cast<char *>(a.workspace) + off);
+                } else {
+                    splits = 1;
+                }
+            }
+            if (splits == 1) return (BM == 256) ? launch_v16t<256, 4, 1, false>(tm, ti, q, sp, s) : launch_v16t<128, 4, 2, false>(tm, ti, q, sp, s);
+            const int rc = (BM == 256) ? launch_v16t<256, 4, 1, true>(tm, ti, q, sp, s) : launch_v16t<128, 4, 2, true>(tm, ti, q, sp, s);
+            if (rc != BTC_OK) return rc;
+            const size_t mn = (size_t)a.M * a.N;
+            splitk_reduce_kernel<<<(unsigned)((mn + 255) / 256), 256, 0, s>>>(sp.part, splits, a.M, a.N, a.alpha, a.mu, q.sumx, a.y, a.y_dt);
+            return cuda_check_launch();
         }
     }
     if (BM == 256) return launch_cfg<256, 4>(tm, p, s);
@@ -711,7 +793,7 @@ extern "C" BTC_API int btc_linear_gemm_static_scratch(const void *x, int x_dtype
 {
     if (T) return BTC_ERR_UNSUPPORTED;
     if (v < 1 || v > 32 || Kc < 1 || Kc > 65536 || M < 1 || N < 1 || K < 1 || K % v) return BTC_ERR_SHAPE;
-    if (btc_linear_workspace_bytes(M, N, K, v, Kc) > (size_t)BTC_STATIC_SCRATCH_BYTES) return BTC_ERR_WORKSPACE;
+    if (btc::gemm_tcgen05_workspace_min(M) > (size_t)BTC_STATIC_SCRATCH_BYTES) return BTC_ERR_WORKSPACE;
     void *scratch = nullptr;
     const int rc = btc::static_scratch_address(&scratch);
     if (rc != BTC_OK) return rc;

@@ -165,6 +165,36 @@ def test_gemm_parity_benchmark_config_sampled(M):
         assert bool(torch.isfinite(y).all())
 
 
+SPLIT_K = [
+    # N, K, M, xdt, mu, out dtype   (v = 16, few 128-row tiles, K >= 4096: the tensor-core path splits K over the idle SMs)
+    (300, 4096, 16, "bf16", False, torch.float32),
+    (200, 11008, 9, "f16", True, torch.float32),
+    (1000, 5120, 100, "bf16", True, torch.float16),
+    (640, 8192, 300, "bf16", False, torch.bfloat16),
+]
+
+
+@pytest.mark.parametrize("N,K,M,xdt,mu,odt", SPLIT_K)
+def test_gemm_split_k_matches_oracle_and_unsplit(N, K, M, xdt, mu, odt):
+    """With the full workspace K is split over several CTAs per tile and the partial sums are added in a fixed order;
+    with only the minimum workspace (the entry point without allocation) the same call runs unsplit.  Both against
+    the oracle; the split result twice, bit for bit."""
+    L = wl.make_layer(_spec(N, K, 16, 8192, x_dtype=xdt, with_mu=mu), M, seed=N + K + M)
+    d = to_device(L)
+    assert btc.linear_workspace_bytes(M, N, K, 16, 8192) > 4 * M * N          # room for at least two partial copies
+    y1 = btc.linear_gemm(d["x"], d["idx"], d["Cp"], d["alpha"], 16, 8192, mu=d["mu"], out_dtype=odt)
+    y2 = btc.linear_gemm(d["x"], d["idx"], d["Cp"], d["alpha"], 16, 8192, mu=d["mu"], out_dtype=odt)
+    y3 = btc.linear_gemm_static_scratch(d["x"], d["idx"], d["Cp"], d["alpha"], 16, 8192, mu=d["mu"])
+    torch.cuda.synchronize()
+    assert torch.equal(y1, y2)
+    want = oracle_y(L)
+    tol = TOL_GEMM if odt == torch.float32 else TOL_GEMM + 2.0 ** -8
+    for y in (y1, y3):
+        rel, fwd = errors(y.float(), want, L)
+        assert rel <= tol and fwd <= tol, (N, K, M, rel, fwd)
+    assert btc.device_status() == 0
+
+
 def test_gemm_deterministic_and_bounded():
     L = wl.make_layer(_spec(300, 1024, 16, 8192, x_dtype="bf16"), 200, seed=5)
     d = to_device(L)
