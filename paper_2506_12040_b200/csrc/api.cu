@@ -75,7 +75,10 @@ static int run_linear(Path path, const void *x, int x_dt, const uint16_t *idx, c
             rc = launch_gemv_imma(&a, 1, s);
             if (rc == BTC_ERR_UNSUPPORTED) rc = launch_gemv_decode(a, s);
         } else {
-            rc = launch_gemv_decode(a, s);
+            // (a very long K with few row tiles: the tensor-core launch with K split over the SMs, when the workspace has
+            // room for its partial sums)
+            if (gemm_tcgen05_small_m_pays(M, N, K, v)) rc = launch_gemm_tcgen05(a, s, true);
+            if (rc == BTC_ERR_UNSUPPORTED) rc = launch_gemv_decode(a, s);
             if (rc == BTC_ERR_UNSUPPORTED) rc = launch_gemv_imma(&a, 1, s);
         }
     }

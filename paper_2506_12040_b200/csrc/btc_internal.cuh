@@ -37,7 +37,8 @@ int launch_gemv_decode(const LinearArgs &a, cudaStream_t s);
 size_t gemv_decode_workspace_bytes(int M, int N, int K, int v, int Kc);
 
 // gemm_tcgen05.cu: tensor-core path.  Same UNSUPPORTED convention.
-int launch_gemm_tcgen05(const LinearArgs &a, cudaStream_t s);
+int launch_gemm_tcgen05(const LinearArgs &a, cudaStream_t s, bool small_m = false);   // small_m: also 5 <= M <= 8 where it pays
+bool gemm_tcgen05_small_m_pays(int M, int N, int K, int v);
 size_t gemm_tcgen05_workspace_bytes(int M, int N, int K, int v, int Kc);   // with room for a K split where one pays
 size_t gemm_tcgen05_workspace_min(int M);                                 // what the kernels cannot do without
 

@@ -633,12 +633,25 @@ size_t gemm_tcgen05_workspace_min(int M)
     return M > 8 ? (size_t)M * sizeof(float) : 0;   // row sums of x for the mean term
 }
 
+// 5 <= M <= 8 with few tiles and a very long K (the 11008-wide down projection): the split tensor-core launch beats
+// the fp16 decode kernel (measured 17 us against 30 us for 4096 x 11008), so the decode entry point tries it first.
+bool gemm_tcgen05_small_m_pays(int M, int N, int K, int v)
+{
+    if (M < 5 || M > 8 || v != 16 || K % 16 || (K / v) % 8) return false;
+    int splits = 1;
+    const int k_tiles = (K + G_BK - 1) / G_BK;
+    splitk_tiles((N + 127) / 128, k_tiles, &splits);
+    return splits > 1 && k_tiles >= 128;
+}
+
 // The minimum plus, where the launch would otherwise leave most SMs idle (v = 16, few tiles, long K), room for the
 // partial sums of a K split.  With less than this (but at least the minimum) the kernels run without the split.
 size_t gemm_tcgen05_workspace_bytes(int M, int N, int K, int v, int)
 {
     size_t w = gemm_tcgen05_workspace_min(M);
-    if (M > 8 && v == 16 && (K / v) % 8 == 0) {
+    const bool small = gemm_tcgen05_small_m_pays(M, N, K, v);
+    if (small) w = (size_t)M * sizeof(float);
+    if ((M > 8 || small) && v == 16 && (K / v) % 8 == 0) {
         const int BM = gemm_bm(M, N);
         int splits = 1;
         splitk_tiles(((N + 127) / 128) * ((M + BM - 1) / BM), (K + G_BK - 1) / G_BK, &splits);
@@ -647,9 +660,12 @@ size_t gemm_tcgen05_workspace_bytes(int M, int N, int K, int v, int)
     return w;
 }
 
-int launch_gemm_tcgen05(const LinearArgs &a, cudaStream_t s)
+int launch_gemm_tcgen05(const LinearArgs &a, cudaStream_t s, bool small_m)
 {
-    if (a.M <= 8) return BTC_ERR_UNSUPPORTED;                  // the decode path is the better kernel there
+    if (a.M <= 8 && !small_m) return BTC_ERR_UNSUPPORTED;      // the decode path is the better kernel there
+    if (a.M <= 8 && (!gemm_tcgen05_small_m_pays(a.M, a.N, a.K, a.v) || !a.workspace ||
+                     a.workspace_bytes < gemm_tcgen05_workspace_bytes(a.M, a.N, a.K, a.v, a.Kc)))
+        return BTC_ERR_UNSUPPORTED;                            // (only with room for the K split)
     if (a.K % 8) return BTC_ERR_UNSUPPORTED;                   // TMA row pitch must be a multiple of 16 bytes
     encode_tiled_fn enc = get_encode();
     if (!enc) return BTC_ERR_UNSUPPORTED;
@@ -698,7 +714,7 @@ int launch_gemm_tcgen05(const LinearArgs &a, cudaStream_t s)
             int splits = 1;
             const int per = splitk_tiles(((a.N + 127) / 128) * ((a.M + BM - 1) / BM), q.k_tiles, &splits);
             if (splits > 1) {
-                const size_t off = (gemm_tcgen05_workspace_min(a.M) + 255) & ~(size_t)255;
+                const size_t off = ((size_t)a.M * sizeof(float) + 255) & ~(size_t)255;   // (row sums of x come first)
                 const size_t need = off + (size_t)splits * a.M * a.N * sizeof(float);
                 if (a.workspace && a.workspace_bytes >= need && reinterpret_cast<uintptr_t>(a.workspace) % 16 == 0) {
                     sp.split_tiles = per;

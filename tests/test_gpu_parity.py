@@ -66,6 +66,8 @@ SMALL = [
     (129, 4096, 16, 8192, 1, "uniform", True),
     (150, 2048, 16, 65536, 1, "uniform", True),
     (77, 1024, 16, 50000, 2, "zipf", False),
+    (300, 8192, 16, 8192, 8, "uniform", True),      # few row tiles, very long K: the split tensor-core launch
+    (1000, 11008, 16, 4096, 5, "uniform", False),
     (70, 11008, 16, 8192, 2, "uniform", False),
     (1000, 640, 20, 21619, 5, "zipf", True),
     (33, 72, 4, 9, 7, "uniform", False),
