@@ -282,9 +282,11 @@ def run_gpu(args):
             # same-shape layers of other slots double the number of distinct index copies
             same = [j for j, t in enumerate(specs) if (t.N, t.K) == (s.N, s.K)]
 
+            ws1 = torch.empty(max(256, btc.linear_workspace_bytes(M, s.N, s.K, s.v, s.Kc)), dtype=torch.uint8, device=dev)
+
             def one(k):
                 d = sets[rr[k % R]][same[(k // R) % len(same)]]
-                btc.linear_gemv(x, d["idx"], d["Cp"], d["alpha"], s.v, s.Kc, out=outs[k % R])
+                btc.linear_gemv(x, d["idx"], d["Cp"], d["alpha"], s.v, s.Kc, out=outs[k % R], workspace=ws1)
             stream = torch.cuda.Stream(device=dev)
             with torch.cuda.stream(stream):
                 for k in range(5):
