@@ -403,6 +403,7 @@ gemm_v16t_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_d = *s_tmem;
+    if (SPLIT) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the reduce kernel may take its place early
 
     if (warp == 0) {
         if (lane == 0) {
@@ -551,6 +552,9 @@ gemm_v16t_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
 __global__ void splitk_reduce_kernel(const float *__restrict__ part, int splits, int M, int N, const __half *__restrict__ alpha,
                                      const __half *__restrict__ mu, const float *__restrict__ sumx, void *__restrict__ y, int y_dt)
 {
+    // launched with programmatic stream serialisation: the blocks are resident before the split kernel has finished, and
+    // wait here until all of it has completed and its partial sums are visible
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     const size_t MN = (size_t)M * N;
     if (i >= MN) return;
@@ -727,8 +731,18 @@ int launch_gemm_tcgen05(const LinearArgs &a, cudaStream_t s, bool small_m)
             const int rc = (BM == 256) ? launch_v16t<256, 4, 1, true>(tm, ti, q, sp, s) : launch_v16t<128, 4, 2, true>(tm, ti, q, sp, s);
             if (rc != BTC_OK) return rc;
             const size_t mn = (size_t)a.M * a.N;
-            splitk_reduce_kernel<<<(unsigned)((mn + 255) / 256), 256, 0, s>>>(sp.part, splits, a.M, a.N, a.alpha, a.mu, q.sumx, a.y, a.y_dt);
-            return cuda_check_launch();
+            cudaLaunchConfig_t cfg = {};
+            cfg.gridDim = dim3((unsigned)((mn + 255) / 256));
+            cfg.blockDim = dim3(256);
+            cfg.stream = s;
+            cudaLaunchAttribute at[1];
+            at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+            at[0].val.programmaticStreamSerializationAllowed = 1;
+            cfg.attrs = at;
+            cfg.numAttrs = 1;
+            const float *part = sp.part;
+            const cudaError_t e = cudaLaunchKernelEx(&cfg, splitk_reduce_kernel, part, splits, a.M, a.N, a.alpha, a.mu, q.sumx, a.y, a.y_dt);
+            return e == cudaSuccess ? BTC_OK : cuda_fail(e);
         }
     }
     if (BM == 256) return launch_cfg<256, 4>(tm, p, s);
