@@ -103,9 +103,23 @@ km_threshold_kernel(const uint32_t *__restrict__ cnt, int P, int Kc, KmState *st
         __syncthreads();
         return s_val;
     };
+    // up to 65536 patterns (v <= 16) the thread's 64 frequencies stay in registers over the bisection
+    constexpr int KEEP = 64;
+    const bool kept = P <= KEEP * 1024;
+    uint32_t mine[KEEP];
+#pragma unroll
+    for (int i = 0; i < KEEP; ++i) {
+        const int p = threadIdx.x + i * 1024;
+        mine[i] = (kept && p < P) ? cnt[p] : 0u;
+    }
     auto count_ge = [&](unsigned t) -> unsigned {
         unsigned c = 0;
-        for (int p = threadIdx.x; p < P; p += blockDim.x) c += (cnt[p] >= t) ? 1u : 0u;
+        if (kept) {
+#pragma unroll
+            for (int i = 0; i < KEEP; ++i) c += (mine[i] >= t) ? 1u : 0u;
+        } else {
+            for (int p = threadIdx.x; p < P; p += blockDim.x) c += (cnt[p] >= t) ? 1u : 0u;
+        }
         return block_sum(c);
     };
     unsigned mx = 0;
