@@ -188,26 +188,32 @@ km_init_rank_kernel(const uint32_t *__restrict__ cand_p, const uint32_t *__restr
 __global__ void __launch_bounds__(1024)
 km_ties_kernel(const uint32_t *__restrict__ cnt, int P, int Kc, uint32_t *__restrict__ C, const KmState *st)
 {
-    __shared__ int s_off[1024];
+    // each warp takes a contiguous range of patterns and walks it 32 at a time (coalesced); the order inside a step comes
+    // from a ballot, the order of the warps from a prefix over their totals
+    __shared__ int s_tot[32];
     const unsigned thr = st->thr;
-    const int per = (P + 1023) / 1024;
-    const int p0 = threadIdx.x * per, p1 = min(P, p0 + per);
-    int mine = 0;
-    for (int p = p0; p < p1; ++p) mine += (cnt[p] == thr) ? 1 : 0;
-    s_off[threadIdx.x] = mine;
-    __syncthreads();
-    for (int o = 1; o < 1024; o <<= 1) {                    // inclusive scan
-        const int add = (threadIdx.x >= o) ? s_off[threadIdx.x - o] : 0;
-        __syncthreads();
-        s_off[threadIdx.x] += add;
-        __syncthreads();
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int seg = (((P + 31) / 32) + 31) & ~31;           // patterns per warp, a multiple of 32
+    const int p_begin = warp * seg;
+    int total = 0;
+    for (int q = p_begin; q < p_begin + seg; q += 32) {
+        const int p = q + lane;
+        total += __popc(__ballot_sync(0xffffffffu, p < P && cnt[p] == thr));
     }
-    int rank = st->n_cand + s_off[threadIdx.x] - mine;
-    for (int p = p0; p < p1; ++p)
-        if (cnt[p] == thr) {
-            if (rank < Kc) C[rank] = (uint32_t)p;
-            ++rank;
+    if (lane == 0) s_tot[warp] = total;
+    __syncthreads();
+    int rank = st->n_cand;
+    for (int w = 0; w < warp; ++w) rank += s_tot[w];
+    for (int q = p_begin; q < p_begin + seg; q += 32) {
+        const int p = q + lane;
+        const bool tie = p < P && cnt[p] == thr;
+        const unsigned b = __ballot_sync(0xffffffffu, tie);
+        if (tie) {
+            const int r = rank + __popc(b & ((1u << lane) - 1u));
+            if (r < Kc) C[r] = (uint32_t)p;
         }
+        rank += __popc(b);
+    }
 }
 
 __global__ void __launch_bounds__(256)
