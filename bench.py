@@ -363,6 +363,31 @@ def run_gpu(args):
                 gem[f"M{M}_{s.N}x{s.K}"] = res
         details["gemm"] = gem
 
+        # ---- tensor-core path at small M (one 128-row x tile: few CTAs unless K is split over the SMs), same protocol
+        small = {}
+        for li, s in enumerate(c4["layers"]):
+            d = dev_layer(wl.make_layer(s, 1, c4["seed"], li))
+            for M in (16, 128):
+                xb = torch.from_numpy(wl.make_x(M, s.K, "bf16", c4["seed"], 16 * li + 5).view(np.int16)).to(dev).view(torch.bfloat16)
+                y = torch.empty((M, s.N), dtype=torch.float32, device=dev)
+                wsm = torch.empty(max(256, btc.linear_workspace_bytes(M, s.N, s.K, s.v, s.Kc)), dtype=torch.uint8, device=dev)
+                for _ in range(3):
+                    btc.linear_gemm(xb, d["idx"], d["Cp"], d["alpha"], s.v, s.Kc, out=y, workspace=wsm)
+                ts = []
+                for _ in range(7):
+                    flush.zero_()
+                    e0 = torch.cuda.Event(enable_timing=True)
+                    e1 = torch.cuda.Event(enable_timing=True)
+                    e0.record()
+                    btc.linear_gemm(xb, d["idx"], d["Cp"], d["alpha"], s.v, s.Kc, out=y, workspace=wsm)
+                    e1.record()
+                    torch.cuda.synchronize()
+                    ts.append(e0.elapsed_time(e1) * 1e3)
+                us = float(np.median(ts))
+                small[f"M{M}_{s.N}x{s.K}"] = {"us": us, "TFLOPs": 2.0 * M * s.N * s.K / us * 1e-6,
+                                              "workspace_bytes": int(wsm.numel())}
+        details["gemm_small_M"] = small
+
         # ---- configs 1 and 3: single layers at M = 1 (config 3: v = 20, 65536 centroids gathered from L1/L2, Zipf indices)
         def time_single(spec, seed, lid, M, copies=24, reps=96):
             L = wl.make_layer(spec, M, seed, lid)

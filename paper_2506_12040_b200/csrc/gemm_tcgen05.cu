@@ -611,7 +611,7 @@ static int launch_v16t(const CUtensorMap &tm, const CUtensorMap &ti, const Gemm2
 }
 
 // K splits for a launch of `tiles` CTAs over `k_tiles` k tiles: as many as keep the grid within the SM count, each a
-// whole number of index tiles (16 k tiles) and at least two of them long.  Returns k tiles per split.
+// whole number of index tiles (16 k tiles).  Returns k tiles per split.
 static int splitk_tiles(int tiles, int k_tiles, int *splits)
 {
     *splits = 1;
@@ -619,7 +619,7 @@ static int splitk_tiles(int tiles, int k_tiles, int *splits)
     int want = 148 / tiles;
     if (want > 8) want = 8;
     int per = ((k_tiles + want - 1) / want + 15) / 16 * 16;
-    if (per < 32) per = 32;
+    if (per < 16) per = 16;
     const int n = (k_tiles + per - 1) / per;
     if (n < 2) return k_tiles;
     *splits = n;
@@ -637,7 +637,7 @@ size_t gemm_tcgen05_workspace_min(int M)
     return M > 8 ? (size_t)M * sizeof(float) : 0;   // row sums of x for the mean term
 }
 
-// 5 <= M <= 8 with few tiles and a very long K (the 11008-wide down projection): the split tensor-core launch beats
+// 5 <= M <= 8 with few tiles and a long K (above all the 11008-wide down projection): the split tensor-core launch beats
 // the fp16 decode kernel (measured 17 us against 30 us for 4096 x 11008), so the decode entry point tries it first.
 bool gemm_tcgen05_small_m_pays(int M, int N, int K, int v)
 {
@@ -645,7 +645,7 @@ bool gemm_tcgen05_small_m_pays(int M, int N, int K, int v)
     int splits = 1;
     const int k_tiles = (K + G_BK - 1) / G_BK;
     splitk_tiles((N + 127) / 128, k_tiles, &splits);
-    return splits > 1 && k_tiles >= 128;
+    return splits > 1 && (k_tiles >= 128 || (k_tiles >= 64 && M >= 6));   // (4096 x 4096 at M = 8: 10 us against 12.5 us)
 }
 
 // The minimum plus, where the launch would otherwise leave most SMs idle (v = 16, few tiles, long K), room for the
