@@ -193,8 +193,9 @@ BTC_API int btc_linear_gemv_batch(const btc_linear_problem *problems, int count,
  *
  * Arguments are those of btc_linear_gemm without workspace / workspace_bytes.  Differences:
  *   - Needs 4*M <= BTC_STATIC_SCRATCH_BYTES, i.e. M <= BTC_STATIC_SCRATCH_BYTES / 4 rows of x;
- *     larger M returns BTC_ERR_WORKSPACE and nothing is launched.  K is never split here (the
- *     array has no room for partial sums).  T must be NULL (the transform needs M*K*2 bytes more): BTC_ERR_UNSUPPORTED.
+ *     larger M returns BTC_ERR_WORKSPACE and nothing is launched.  K is never split here: only the
+ *     bytes of the row sums are handed to the kernels, so no partial sums of y ever sit in the
+ *     array.  T must be NULL (the transform needs M*K*2 bytes more): BTC_ERR_UNSUPPORTED.
  *   - The first call on each device looks up the array's device address (no allocation, no
  *     launch) and caches it; make that first call outside any stream capture.  The device that is
  *     current at the call is the one used, as for every other entry point.

@@ -827,6 +827,9 @@ extern "C" BTC_API int btc_linear_gemm_static_scratch(const void *x, int x_dtype
     void *scratch = nullptr;
     const int rc = btc::static_scratch_address(&scratch);
     if (rc != BTC_OK) return rc;
+    // Only the part the kernels cannot do without is handed on (the row sums of x), so that no launch below ever
+    // takes the K split and parks partial sums of y in the shared array.
+    const size_t usable = (btc::gemm_tcgen05_workspace_min(M) + 255) / 256 * 256;
     return btc_linear_gemm(x, x_dtype, idx, C_packed, alpha, mu, nullptr, y, y_dtype, M, N, K, v, Kc, scratch,
-                           (size_t)BTC_STATIC_SCRATCH_BYTES, stream);
+                           usable, stream);
 }

@@ -152,8 +152,13 @@ def make_sign_words(n: int, v: int, seed: int, stream: int = 7, prototypes: int 
     return words.astype(np.uint32)
 
 
-def make_alpha_f16(N: int, seed: int, stream: int = 2, sigma: float = 0.02, scale: float = 1.0) -> np.ndarray:
-    return (np.abs(_normal(seed, stream, N)) * sigma * scale).astype(np.float16)
+def make_alpha_f16(N: int, seed: int, stream: int = 2, sigma: float = 0.02, scale: float = 1.0,
+                   signed: bool = False) -> np.ndarray:
+    """|N(0, sigma^2)| * scale as fp16; with signed=True the draw keeps its sign."""
+    a = _normal(seed, stream, N)
+    if not signed:
+        a = np.abs(a)
+    return (a * sigma * scale).astype(np.float16)
 
 
 def make_mu_f16(N: int, seed: int, stream: int = 5, sigma: float = 0.002) -> np.ndarray:
@@ -190,6 +195,7 @@ class LayerSpec:
     x_dtype: str = "f16"
     outlier_frac: float = 0.0
     alpha_scale: float = 1.0      # multiplies the 0.02 sigma (unit-gain chains use 1/(0.02*sqrt(K)))
+    alpha_signed: bool = False    # N(0, sigma^2) instead of |N(0, sigma^2)| (chains: keeps the activations zero-mean)
     with_mu: bool = False
 
     @property
@@ -222,7 +228,7 @@ def make_layer(spec: LayerSpec, M: int, seed: int, layer_id: int = 0,
     s0 = 16 * layer_id
     C = make_codebook_pm1(spec.Kc, spec.v, seed, s0 + 0)
     idx = make_indices(spec.N, spec.Kb, spec.Kc, spec.idx_dist, seed, s0 + 1)
-    alpha = make_alpha_f16(spec.N, seed, s0 + 2, scale=spec.alpha_scale)
+    alpha = make_alpha_f16(spec.N, seed, s0 + 2, scale=spec.alpha_scale, signed=spec.alpha_signed)
     x = make_x(M, spec.K, spec.x_dtype, seed, s0 + 3, spec.outlier_frac)
     mu = make_mu_f16(spec.N, seed, s0 + 5) if spec.with_mu else None
     return LayerData(spec, M, C, idx, alpha, x, mu)
@@ -257,14 +263,20 @@ CONFIGS: Dict[int, dict] = {
 
 def config_layers(config: int, Kc: Optional[int] = None, idx_dist: Optional[str] = None) -> dict:
     """Layer list of one benchmark config.  Config 5 is the 32-layer decode chain
-    (7 projections per layer, v=16) with unit-RMS-gain scales so that a chain of
-    224 linears stays inside fp16 range; Kc and the index distribution are swept."""
+    (7 projections per layer, v=16); Kc and the index distribution are swept.  So that a
+    chain of 224 linears with nothing between them stays inside fp16 range for every
+    point of the sweep, its scales have unit RMS gain (sigma = 1/sqrt(K)) and keep the
+    sign of their normal draw: with all-positive scales every output carries the same
+    multiple of the common component <x, mean centroid>, the next layer's input has a
+    non-zero mean, and that mode grows from layer to layer (with few centroids or Zipf
+    indices the mean centroid is far from zero); with signed scales the activations stay
+    zero-mean and uncorrelated, and the expected gain of a layer is exactly one."""
     if config in CONFIGS:
         return CONFIGS[config]
     if config == 5:
         kc = 4096 if Kc is None else Kc
         dist = idx_dist or "uniform"
         one = _llama7b(16, kc, idx_dist=dist)
-        one = [replace(s, alpha_scale=1.0 / (0.02 * math.sqrt(s.K))) for s in one]
+        one = [replace(s, alpha_scale=1.0 / (0.02 * math.sqrt(s.K)), alpha_signed=True) for s in one]
         return {"layers": one, "n_blocks": 32, "M": (1,), "seed": 42 + 5000}
     raise KeyError(config)
