@@ -35,9 +35,28 @@ import workloads as wl  # noqa: E402
 METRIC = "effective HBM GB/s at M=1 (us/layer and TFLOP/s at M=2048 in details)"
 UNIT = "GB/s"
 CONFIG_ID = 2
-# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the fused step kernel, from the ncu capture summarised in
-# profiles/decode_imma_config2_M1_step.md (set to None whenever that kernel changes until it is captured again)
-TRAFFIC_BYTES_PER_LAUNCH = 25726720
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the fused step kernel come from the ncu capture recorded in
+# profiles/decode_step_traffic.json, which also holds the SHA-256 of the kernel source it was taken on; when the source
+# has changed since, the figure no longer describes the kernel that is timed and `traffic` is reported as null.
+TRAFFIC_RECORD = os.path.join(ROOT, "profiles", "decode_step_traffic.json")
+KERNEL_SOURCE = os.path.join(ROOT, "paper_2506_12040_b200", "csrc", "gemv_imma.cu")
+
+
+def kernel_source_sha256() -> str:
+    import hashlib
+    with open(KERNEL_SOURCE, "rb") as f:
+        return hashlib.sha256(f.read()).hexdigest()
+
+
+def recorded_traffic():
+    """(bytes per launch or None, note)."""
+    if not os.path.exists(TRAFFIC_RECORD):
+        return None, "no capture recorded"
+    with open(TRAFFIC_RECORD) as f:
+        rec = json.load(f)
+    if rec.get("kernel_source_sha256") != kernel_source_sha256():
+        return None, "kernel source changed since the capture of " + str(rec.get("captured"))
+    return int(rec["dram_bytes_read"]) + int(rec["dram_bytes_write"]), "ncu capture of " + str(rec.get("captured"))
 
 
 def measured_peaks():
@@ -211,7 +230,9 @@ def run_gpu(args):
             batches[r].run()
         return step, outs, xs
 
-    def time_steps(step, steps, warmup):
+    def time_steps(step, steps, warmup, replays=25):
+        """One CUDA graph of `steps` steps, replayed `replays` times; every replay is bracketed by CUDA events on the
+        launching stream.  Returns the per-replay seconds (sorted)."""
         stream = torch.cuda.Stream(device=dev)
         with torch.cuda.stream(stream):
             for w in range(max(warmup, 3)):
@@ -226,26 +247,32 @@ def run_gpu(args):
             if dist is not None:
                 dist.barrier()
             torch.cuda.synchronize()
-            e0 = torch.cuda.Event(enable_timing=True)
-            e1 = torch.cuda.Event(enable_timing=True)
-            e0.record(stream)
-            g.replay()
-            e1.record(stream)
-            stream.synchronize()
+            ts = []
+            for _ in range(replays):
+                e0 = torch.cuda.Event(enable_timing=True)
+                e1 = torch.cuda.Event(enable_timing=True)
+                e0.record(stream)
+                g.replay()
+                e1.record(stream)
+                stream.synchronize()
+                ts.append(e0.elapsed_time(e1) * 1e-3)
             torch.cuda.synchronize()
-        return e0.elapsed_time(e1) * 1e-3   # seconds for `steps` steps
+        return sorted(ts)
 
     # ---- headline: M = 1
     step1, outs1, xs1 = make_runner(1)
     bytes_step = sum(algorithmic_bytes(s, 1) for s in specs)
+    torch.cuda.nvtx.range_push("headline: fused decode step, M=1")
     with ClockSampler(local) as clk:
-        t_total = time_steps(step1, args.steps, args.warmup)
+        replays = time_steps(step1, args.steps, args.warmup)
         # keep the sampler busy for at least a few samples on very short runs
         t_end = time.time() + 0.3
         while time.time() < t_end:
             step1(0)
         torch.cuda.synchronize()
+    torch.cuda.nvtx.range_pop()
     clocks = clk.summary()
+    t_total = replays[len(replays) // 2]          # median replay of the K-step graph
     t_max = max_over_ranks(t_total, dist, dev)
     ms_per_step = t_max / args.steps * 1e3
     value = whole_job_gbs(world, bytes_step, t_max, args.steps)
@@ -255,6 +282,8 @@ def run_gpu(args):
     achieved = bytes_per_launch / avg_launch_s * 1e-9
 
     details = {"us_per_layer_M1": avg_launch_s * 1e6 / len(specs), "us_per_step_M1": avg_launch_s * 1e6, "weight_sets": R,
+               "replays": {"count": len(replays), "us_per_step_min": replays[0] / args.steps * 1e6,
+                           "us_per_step_median": t_total / args.steps * 1e6, "us_per_step_max": replays[-1] / args.steps * 1e6},
                "per_shape_M1": {}, "hbm_nominal_gbs": 8000.0,
                "frac_of_nominal": achieved / 8000.0}
 
@@ -307,19 +336,58 @@ def run_gpu(args):
             us = e0.elapsed_time(e1) * 1e3 / reps
             b = algorithmic_bytes(s, M)
             return {"us": us, "GBps": b / us * 1e-3, "frac_measured": b / us * 1e-3 / peaks["hbm_gbs"]}
+        def time_dense_fp16_gemv(i, reps=200):
+            """Context for the paper's "1.6x over FP16" (Section 5, latency paragraph): torch.matmul of an fp16 [1, K] row
+            with a dense fp16 [N, K] weight of the same shape, rotating over copies larger than L2."""
+            s = specs[i]
+            copies = max(2, int(np.ceil(2.2 * l2 / (2 * s.N * s.K))))
+            ws = [torch.randn(s.N, s.K, device=dev, dtype=torch.float16) for _ in range(copies)]
+            x = torch.randn(1, s.K, device=dev, dtype=torch.float16)
+            y = torch.empty(1, s.N, device=dev, dtype=torch.float16)
+            stream = torch.cuda.Stream(device=dev)
+            with torch.cuda.stream(stream):
+                for k in range(3):
+                    torch.matmul(x, ws[k % copies].t(), out=y)
+                stream.synchronize()
+                g = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(g, stream=stream):
+                    for k in range(reps):
+                        torch.matmul(x, ws[k % copies].t(), out=y)
+                g.replay()
+                stream.synchronize()
+                e0 = torch.cuda.Event(enable_timing=True)
+                e1 = torch.cuda.Event(enable_timing=True)
+                e0.record(stream)
+                g.replay()
+                e1.record(stream)
+                stream.synchronize()
+            us = e0.elapsed_time(e1) * 1e3 / reps
+            return {"us": us, "GBps": 2.0 * s.N * s.K / us * 1e-3}
         seen = set()
+        count = {}
+        for s in specs:
+            count[(s.N, s.K)] = count.get((s.N, s.K), 0) + 1
+        torch.cuda.nvtx.range_push("per-layer launches, M=1 and M=8")
         for i, s in enumerate(specs):
             if (s.N, s.K) in seen:
                 continue
             seen.add((s.N, s.K))
             for M in (1, 8):
                 details.setdefault(f"per_shape_M{M}", {})[f"{s.N}x{s.K}"] = time_shape(i, M)
+            d1 = details["per_shape_M1"][f"{s.N}x{s.K}"]
+            d1["dense_fp16_gemv"] = time_dense_fp16_gemv(i)
+            d1["speedup_over_dense_fp16"] = d1["dense_fp16_gemv"]["us"] / d1["us"]
+        torch.cuda.nvtx.range_pop()
+        # the same seven layers as seven launches (one per layer, each timed over rotating copies): per-layer us = total / R
+        set_us = sum(details["per_shape_M1"][f"{s.N}x{s.K}"]["us"] for s in specs)
+        details["per_layer_set_M1"] = {"us_per_set": set_us, "GBps": bytes_step / set_us * 1e-3,
+                                       "frac_measured": bytes_step / set_us * 1e-3 / peaks["hbm_gbs"]}
 
         # ---- the whole step (one fused launch) with more rows of x
         step_m = {}
         for M in (2, 4, 8):
             stepM, _, _ = make_runner(M)
-            tM = time_steps(stepM, 60, 5) / 60
+            tM = time_steps(stepM, 60, 5, replays=9)[4] / 60
             bM = sum(algorithmic_bytes(s, M) for s in specs)
             step_m[f"M{M}"] = {"us": tM * 1e6, "GBps": bM / tM * 1e-9, "frac_measured": bM / tM * 1e-9 / peaks["hbm_gbs"]}
         details["step_by_M"] = step_m
@@ -467,12 +535,15 @@ def run_gpu(args):
                     stream.synchronize()
                     ts.append(e0.elapsed_time(e1) * 1e-3)
             t = float(np.median(ts))
-            finite = bool(torch.isfinite(h[nb & 1].float()).all())
+            finite = bool(torch.isfinite(h[nb & 1].float()).all()) and bool(torch.isfinite(gu[0].float()).all())
             nbytes = nb * sum(algorithmic_bytes(s5, 1) for s5 in sp)
             return {"tokens_per_s": 1.0 / t, "us_per_token": t * 1e6, "GBps": nbytes / t * 1e-9,
                     "frac_measured": nbytes / t * 1e-9 / peaks["hbm_gbs"], "launches": len(launches), "finite": finite}
+        torch.cuda.nvtx.range_push("config 5 chain sweep")
         details["config5_chain"] = {f"Kc{Kc}_{dn}": time_chain(Kc, dn)
-                                    for (Kc, dn) in ((4096, "uniform"), (256, "uniform"), (65536, "uniform"), (4096, "zipf"))}
+                                    for Kc in (256, 4096, 65536) for dn in ("uniform", "zipf")}
+        torch.cuda.nvtx.range_pop()
+        assert all(v["finite"] for v in details["config5_chain"].values()), "a chain of the sweep left fp16 range"
         # ---- codebook construction: the blocks of a 4096 x 4096 sign matrix (v = 16), 8192 centroids
         def time_kmeans(n=4096 * 4096 // 16, v=16, Kc=8192, max_iter=8):
             words = torch.from_numpy(wl.make_sign_words(n, v, cfg["seed"] + 31).view(np.int32)).to(dev)
@@ -566,18 +637,21 @@ def run_gpu(args):
 
     if rank == 0:
         peak = peaks["hbm_gbs"]
+        traffic, traffic_note = recorded_traffic()
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
                 "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
                 "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
                 "config": {"workload": "config 2: LLaMA-2-7B decode layer set (7 projections, v=16, Kc=8192), M=1",
                            "cold_l2": f"inputs larger than L2: {R} weight sets x {step_idx_bytes / 1e6:.1f} MB of indices",
-                           "timing": "one CUDA graph of all steps, CUDA events on the launching stream",
+                           "timing": "one CUDA graph of all steps replayed 25 times, CUDA events on the launching stream around every replay, median replay",
                            "multi_gpu": "replicas only"},
                 "clocks": clocks, "e2e": e2e, "gpu_launches": launches,
                 "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
-                             "frac": achieved / peak, "traffic": TRAFFIC_BYTES_PER_LAUNCH, "peak_source": f"of {peaks['source']}",
+                             "frac": achieved / peak, "traffic": traffic, "traffic_note": traffic_note,
+                             "peak_source": f"of {peaks['source']}",
                              "kernel": "gemv_imma_kernel (7 layers per launch)", "bytes_per_launch": bytes_per_launch,
-                             "avg_launch_us": avg_launch_s * 1e6},
+                             "avg_launch_us": avg_launch_s * 1e6,
+                             "per_layer_launches": details.get("per_layer_set_M1")},
                 "cpu_baseline": cpu, "details": details}
         print(json.dumps(line))
     if dist is not None:

@@ -20,7 +20,18 @@
  *   - Returns a btc_status; never aborts, traps or prints.  Argument errors are
  *     detected on the host before anything is launched.
  *   - idx values must be < Kc; this is the caller's contract (kernels do not
- *     check it).  btc_validate_indices checks it on the device.
+ *     check it).  btc_validate_indices checks it on the device.  With the
+ *     environment variable BTC_DEBUG_CHECK_INDICES=1 every btc_linear_* call first
+ *     enqueues that check on the same stream; a violation raises the device-side
+ *     status word (btc_device_status then reports BTC_ERR_INDEX), nothing traps.
+ *   - Programmatic dependent launch: the decode kernels let the next kernel on the
+ *     stream start early and themselves start before their predecessor has
+ *     finished.  They read x only after the predecessor has completed, but they
+ *     prefetch idx, C_packed, alpha and mu right away.  So idx, C_packed, alpha and
+ *     mu must be complete in memory before the call is enqueued: they must not be
+ *     written by a preceding kernel that itself triggers its dependents early (the
+ *     library's own kernels that write them -- btc_codebook_pack,
+ *     btc_codebook_kmeans -- do not).  x and y carry no such restriction.
  *   - Ranges: 1 <= v <= 32, K % v == 0, 1 <= Kc <= 65536 (Kc need not be a power
  *     of two), N >= 1, M >= 1.
  *   - Alignment: x, idx, y and C_packed 16-byte aligned; alpha / mu 2-byte.
@@ -49,7 +60,8 @@ typedef enum {
     BTC_ERR_UNSUPPORTED = 4, /* dtype / option not implemented by this entry point      */
     BTC_ERR_WORKSPACE = 5,   /* workspace missing or smaller than ..._workspace_bytes() */
     BTC_ERR_CUDA = 6,        /* a CUDA runtime / driver call failed                     */
-    BTC_ERR_TIMEOUT = 7      /* a bounded device-side wait ran out (status word)        */
+    BTC_ERR_TIMEOUT = 7,     /* a bounded device-side wait ran out (status word)        */
+    BTC_ERR_INDEX = 8        /* debug check: an index >= Kc was seen (status word)      */
 } btc_status;
 
 typedef enum { BTC_F16 = 0, BTC_BF16 = 1, BTC_F32 = 2 } btc_dtype;

@@ -46,6 +46,10 @@ static int run_linear(Path path, const void *x, int x_dt, const uint16_t *idx, c
         if (!aligned(ws, 256)) return BTC_ERR_ALIGN;
     }
     cudaStream_t s = (cudaStream_t)stream;
+    if (debug_check_indices_enabled()) {
+        rc = launch_index_check(idx, (size_t)N * (K / v), Kc, s);
+        if (rc != BTC_OK) return rc;
+    }
 
     LinearArgs a;
     a.x = x; a.idx = idx; a.Cp = Cp;
@@ -69,18 +73,12 @@ static int run_linear(Path path, const void *x, int x_dt, const uint16_t *idx, c
 
     rc = BTC_ERR_UNSUPPORTED;
     if (path == PATH_GEMV || M <= 8) {
-        // M <= 2: the integer-MMA kernel (3 digit columns per row of x fit one MMA); above that the fp16 bit-trick
-        // kernel is the faster one (its cost does not grow with M up to 8)
-        if (M <= 2) {
-            rc = launch_gemv_imma(&a, 1, s);
-            if (rc == BTC_ERR_UNSUPPORTED) rc = launch_gemv_decode(a, s);
-        } else {
-            // (a very long K with few row tiles: the tensor-core launch with K split over the SMs, when the workspace has
-            // room for its partial sums)
-            if (gemm_tcgen05_small_m_pays(M, N, K, v)) rc = launch_gemm_tcgen05(a, s, true);
-            if (rc == BTC_ERR_UNSUPPORTED) rc = launch_gemv_decode(a, s);
-            if (rc == BTC_ERR_UNSUPPORTED) rc = launch_gemv_imma(&a, 1, s);
-        }
+        // the decode kernel (integer form up to two rows of x, fp16 form above); for M = 5..8 with few row tiles and a
+        // very long K the tensor-core launch with K split over the SMs, when the workspace has room for its partial
+        // sums; the older fp16 kernel and the any-shape kernel take what the first does not cover
+        if (M > 2 && gemm_tcgen05_small_m_pays(M, N, K, v)) rc = launch_gemm_tcgen05(a, s, true);
+        if (rc == BTC_ERR_UNSUPPORTED) rc = launch_gemv_imma(&a, 1, s);
+        if (rc == BTC_ERR_UNSUPPORTED) rc = launch_gemv_decode(a, s);
     }
     else rc = launch_gemm_tcgen05(a, s);
     if (rc == BTC_ERR_UNSUPPORTED) {
@@ -107,6 +105,7 @@ extern "C" const char *btc_status_string(int st)
     case BTC_ERR_WORKSPACE: return "workspace missing or too small";
     case BTC_ERR_CUDA: return "CUDA call failed (see btc_last_cuda_error)";
     case BTC_ERR_TIMEOUT: return "a bounded device-side wait ran out";
+    case BTC_ERR_INDEX: return "an index >= Kc was seen (debug check, BTC_DEBUG_CHECK_INDICES=1)";
     default: return "unknown status";
     }
 }
@@ -163,6 +162,10 @@ extern "C" int btc_linear_gemv_batch(const btc_linear_problem *problems, int cou
             if (rc != BTC_OK) return rc;
             if (p.mu && !aligned(p.mu, 2)) return BTC_ERR_ALIGN;
             if (p.M > 8) return BTC_ERR_SHAPE;
+            if (debug_check_indices_enabled()) {
+                rc = launch_index_check(p.idx, (size_t)p.N * (p.K / p.v), p.Kc, s);
+                if (rc != BTC_OK) return rc;
+            }
             LinearArgs &a = group[n];
             a.x = p.x; a.idx = p.idx; a.Cp = p.C_packed;
             a.alpha = reinterpret_cast<const __half *>(p.alpha);

@@ -50,6 +50,12 @@ int imma_status_read(int *out);
 int imma_status_reset();
 int imma_selftest_wait(cudaStream_t s);
 
+// pack.cu: debug check of the index range (BTC_DEBUG_CHECK_INDICES=1) and its status word.
+bool debug_check_indices_enabled();
+int launch_index_check(const uint16_t *idx, size_t count, int Kc, cudaStream_t s);
+int index_status_read(int *out);
+int index_status_reset();
+
 // transform.cu: x' = x * D * (P1 (x) P2) into xt (same dtype/shape as x).
 int launch_transform(const void *x, int x_dt, const btc_transform &T, void *xt, int M, int K,
                      cudaStream_t s);

@@ -756,6 +756,8 @@ extern "C" BTC_API int btc_device_status_reset(void)
     const int zero = 0;
     cudaError_t e = cudaMemcpyToSymbol(btc::g_gemm_status, &zero, sizeof(int));
     if (e != cudaSuccess) return btc::cuda_fail(e);
+    const int rc = btc::index_status_reset();
+    if (rc != BTC_OK) return rc;
     return btc::imma_status_reset();
 }
 
@@ -773,7 +775,10 @@ extern "C" BTC_API int btc_device_status(int *status_host)
     int v2 = 0;
     const int rc = btc::imma_status_read(&v2);
     if (rc != BTC_OK) return rc;
-    *status_host = v ? v : v2;
+    int v3 = 0;
+    const int rc3 = btc::index_status_read(&v3);
+    if (rc3 != BTC_OK) return rc3;
+    *status_host = v ? v : (v2 ? v2 : v3);
     return BTC_OK;
 }
 

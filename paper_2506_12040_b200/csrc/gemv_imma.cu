@@ -1,55 +1,58 @@
 // Decode path for small M (1..8): streams the index matrices of up to IM_MAXP independent layers
 // once and evaluates every block dot
 //     <x_j, C[idx]> = 2 * sum_{bit=1} x  -  sum x            (identity for +-1 codewords)
-// (block-dot sum of the paper's appendix "Binary codebook LUT-GEMM") with exact integer accumulation
-// inside every K-slice.
+// (block-dot sum of the paper's appendix "Binary codebook LUT-GEMM") on the warp-level MMA, in one of
+// two forms.
 //
-// Why integers.  One output needs K sign applications.  At the HBM rate an SM receives 180 weights per
-// clock (v = 16), while its plain ALUs issue 64 integer lane-operations per clock and the warp-level
-// fp16 MMA retires one m16n8k16 per 2.2 clocks; measured, the fp16 bit trick tops out at 76 weights
-// per clock per SM, the int8 form below at 121.  So the sum over set bits is taken by
-// mma.sync.m16n8k32 (u8 x s8 -> s32):
+// Integer form (M <= 2).  One output needs K sign applications.  At the HBM rate an SM receives 180
+// weights per clock (v = 16), while its plain ALUs issue 64 integer lane-operations per clock; of the
+// warp-level MMAs that run natively here, mma.sync.m16n8k32 (u8 x s8 -> s32) takes the most weights per
+// expansion instruction:
 //   A (16 rows x 32 k, u8) = masked codeword bits: the codeword table stores weight t at bit (t >> 2)
 //       of byte (t & 3), so `word & (0x01010101 << c)` IS the four bytes {0 or 2^c} of weights
 //       4c .. 4c+3: one LOP3 expands four weights.
 //   B (32 k x 8 cols, s8)  = the activations as three balanced base-256 digits of a block-fixed-point
-//       integer: X = rint(x * 2^s), |X| <= 2^(22 - cmax), with s chosen per K-slice (256 or 512
-//       activations of one row of x) from its largest magnitude, pre-shifted by (cmax - c) so that
-//       every product is bit * X * 2^cmax; digit d of row m sits in column 3 m + d.
+//       integer: X = rint(x * 2^s), |X| <= 2^(22 - cmax), with s chosen per K-slice (512 activations
+//       of one row of x at v = 16) from its largest magnitude, pre-shifted by (cmax - c) so that every
+//       product is bit * X * 2^cmax; digit d of row m sits in column 4 m + d, so that both rows of x
+//       see the same lanes and the same order of fp32 operations.
 //   D (16 x 8, s32)        = exact partial sums.
 // The three digit sums of a (slice, output) are recombined in fp32 (each is below 2^24, so the
 // conversions are exact), scaled by 2^-s and added over the slices; then alpha (and mu) are applied.
 // Roundings: the quantisation of x (2^-20 of the slice's largest magnitude for v = 16) and a handful
 // of fp32 operations per output.
 //
-// Work split: persistent CTAs.  A "row group" is 32 rows (16 when M > 2) of one layer; a CTA owns a
-// contiguous, cost-weighted range of row groups over all layers of the launch.  Layers wider than
-// 256 blocks are cut into K-parts of 256 blocks; a CTA walks up to IM_RC of its row groups part by
-// part, so the activation fragments change only once per part, and the epilogue adds the parts.
-//   warps 0..15  compute: warp w owns K-slice w % KS of the part and tile w / KS of the row group
-//                (KS = 8 slices of 32 blocks, 2 tiles when M <= 2; 16 slices of 16 blocks, 1 tile
-//                otherwise); lane (g = lane / 4, t = lane % 4) supplies two rows of the tile and
-//                BPL consecutive blocks; its activations stay in registers as MMA B fragments.
-//   warp 16      producer: TMA boxes (64 blocks x rows, 128-byte swizzle) of the index matrix into
-//                a shared ring, bulk copy of the codeword table.
-//   warps 17,18  epilogue: add the K-slices' partial results in a fixed order (with M <= 2 they arrive as
-//                integer digit sums and are recombined here; with more rows of x each compute warp
-//                recombines its own), add the K-parts, apply alpha (and mu, both staged in shared
-//                memory once per chunk of row groups), store y.
+// fp16 form (3 <= M <= 8): see the comment at its branch in the kernel.  Masked codeword bits act as
+// fp16 numbers on mma.sync.m16n8k16 against the activations themselves (eight rows of x are the eight
+// columns of B), fp32 accumulation; twice the expansion instructions per weight, but no digits and a
+// cost that does not grow with M.
+//
+// Work split.  A tile is 16 output rows of one layer; a CTA owns a contiguous, cost-weighted range of
+// tiles of ONE layer (no CTA works on two layers: each switch would cost a table load).  Layers wider
+// than one K-part (256 blocks; 128 in the fp16 form) are walked part by part over chunks of RC tiles, so
+// the activation fragments change only once per part.
+//   warps 0..7   compute: warp w owns K-slice w of the part (32 blocks; 16 in the fp16 form); lane
+//                (g = lane / 4, t = lane % 4) supplies two rows of the tile and BPL consecutive blocks;
+//                its activations stay in registers as MMA B fragments.  A tile's codewords are looked
+//                up while the previous tile's MMAs are in flight.  The slice's share of every (row, m)
+//                is parked in shared memory as one float; after the last part of a chunk the eight
+//                warps meet once, add the slices in a fixed order, apply alpha (and mu) and store y.
+//   warp 8       producer: TMA boxes (64 blocks x 16 rows, 128-byte swizzle) of the index matrix into
+//                a shared ring of (tile, part) stages; bulk copy of the codeword table.
+// Two CTAs fit an SM (shared memory and registers are sized for it), so while the CTAs of one launch
+// compute, those of the next launch on the stream (programmatic dependent launch) already pull their
+// indices and table into shared memory; only the activations are read after the dependency wait.
 // Every mbarrier wait is bounded; when one runs out the CTA raises a status word and drains.
 #include <cuda.h>
 #include "btc_internal.cuh"
 
 namespace btc {
 
-constexpr int IM_CWARPS = 16;                   // compute warps
-constexpr int IM_EWARPS = 2;                    // epilogue warps (four would cap the kernel at 80 registers: spills)
-constexpr int IM_THREADS = (IM_CWARPS + 1 + IM_EWARPS) * 32;
-constexpr int IM_STAGES = 8;                     // most index stages a launch may use (fewer when shared memory is short)
+constexpr int IM_CWARPS = 8;                    // compute warps = K-slices of a part
+constexpr int IM_THREADS = (IM_CWARPS + 1) * 32;
+constexpr int IM_STAGES = 12;                   // most index stages a launch may use (fewer when shared memory is short)
 constexpr int IM_BOX_COLS = 64;                 // blocks per TMA box row: 128 bytes, the swizzle span
-constexpr int IM_STAGE_BYTES = 16 * 1024;       // one iteration's indices: 4 boxes of 32 rows x 128 bytes
-constexpr int IM_PW = 256;                      // blocks per K-part (16 per compute warp)
-constexpr int IM_RC = 16;                       // row groups a CTA walks part by part at a time
+constexpr int IM_BOX_BYTES = 16 * 128;          // one box: 16 rows x 128 bytes
 
 __device__ int g_imma_status = 0;
 
@@ -63,23 +66,22 @@ struct ImProblem {
     void *y;
     int M, N, K, v, Kc, Kb;
     int x_dt, y_dt;
-    int parts;                // ceil(Kb / IM_PW)
-    int groups;               // row groups: ceil(N / (16 * TRK))
+    int parts;                // ceil(Kb / part width)
+    int groups;               // tiles: ceil(N / 16)
     int ncls;                 // v / 4
-    int cost;                 // cost of one row group (blocks, plus the per-part fragment rebuild; see launch_gemv_imma)
+    int cost, fixed;          // cost of one tile and of a CTA's set-up for this layer (see launch_gemv_imma)
     int per, rem;             // groups / cta_count and groups % cta_count
-    int cta_begin, cta_count; // the CTAs that work on this layer (no CTA works on two layers: each switch would cost a
-                              // table load and a fragment rebuild, and the slowest CTA sets the launch's time)
+    int cta_begin, cta_count; // the CTAs that work on this layer
 };
 
 struct ImBatch {
-    CUtensorMap map[IM_MAXP]; // idx of each layer as a 2-D tensor {K/v, N} of 16-bit words, box {64, rows}, 128-byte swizzle
+    CUtensorMap map[IM_MAXP]; // idx of each layer as a 2-D tensor {K/v, N} of 16-bit words, box {64, 16}, 128-byte swizzle
     ImProblem p[IM_MAXP];
     int count;
     int tab_smem_bytes;       // bytes reserved for the codeword table (0: gather from global memory)
     int tab_head;             // entries of every table that are staged there; the rest is gathered from global memory
-                              // (L1/L2): a table of 65536 codewords does not fit, and with frequency-ordered codebooks
-                              // the head serves most lookups
+                              // (L1/L2): a table of 65536 20-bit codewords does not fit, and with frequency-ordered
+                              // codebooks the head serves most lookups
     int stages;               // index stages in the ring (2 .. IM_STAGES)
 };
 
@@ -103,21 +105,28 @@ __device__ __forceinline__ bool im_mbar_try(uint32_t bar, uint32_t parity) {
         : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
     return ok != 0;
 }
-// Bounded wait: false (and the CTA-wide abort flag latched) once ~1 s has passed.  A waiting warp backs off with
-// nanosleep so that it does not take issue slots from the warps it is waiting for.
+// Bounded wait, called by all 32 lanes of a warp together; the answer is the same in every lane (a vote), so the
+// full-mask shuffles, MMAs and __syncwarp that follow never see a split warp.  False once ~1 s has passed or the
+// CTA-wide abort flag is up.  A waiting warp backs off with nanosleep so that it does not take issue slots from the
+// warps it is waiting for.
 __device__ __forceinline__ bool im_mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag,
                                              long long limit_clk = 2000000000LL) {
-    if (im_mbar_try(bar, parity)) return true;
-    const long long t0 = clock64();
-    int spins = 0;
-    while (!im_mbar_try(bar, parity)) {
-        __nanosleep(spins < 4 ? 20 : 100);
-        if ((++spins & 255) == 0) {
-            if (*abort_flag) return false;
-            if (clock64() - t0 > limit_clk) {
-                *abort_flag = 1;
-                atomicExch(&g_imma_status, (int)BTC_ERR_TIMEOUT);
-                return false;
+    bool ok = im_mbar_try(bar, parity);
+    if (!__all_sync(0xffffffffu, ok)) {
+        const long long t0 = clock64();
+        int spins = 0;
+        for (;;) {
+            ok = im_mbar_try(bar, parity);
+            if (__all_sync(0xffffffffu, ok)) break;
+            __nanosleep(spins < 4 ? 20 : 100);
+            if ((++spins & 255) == 0) {
+                bool give_up = (*abort_flag != 0);
+                if (!give_up && clock64() - t0 > limit_clk) {
+                    *abort_flag = 1;
+                    atomicExch(&g_imma_status, (int)BTC_ERR_TIMEOUT);
+                    give_up = true;
+                }
+                if (__any_sync(0xffffffffu, give_up)) return false;
             }
         }
     }
@@ -132,71 +141,145 @@ __device__ __forceinline__ void im_tma_2d(uint32_t dst, const CUtensorMap *map, 
         "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
         ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(bar) : "memory");
 }
-__device__ __forceinline__ void im_mma_u8s8(int (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
-                                            uint32_t b0, uint32_t b1) {
+__device__ __forceinline__ void im_mma_u8s8(int (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint64_t b) {
     asm volatile(
-        "mma.sync.aligned.m16n8k32.row.col.s32.u8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
+        "{\n\t.reg .b32 b0, b1;\n\t"
+        "mov.b64 {b0, b1}, %8;\n\t"
+        "mma.sync.aligned.m16n8k32.row.col.s32.u8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {b0,b1}, {%0,%1,%2,%3};\n\t}"
         : "+r"(c[0]), "+r"(c[1]), "+r"(c[2]), "+r"(c[3])
-        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "l"(b));
+}
+__device__ __forceinline__ void im_mma_f16(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint64_t b) {
+    asm volatile(
+        "{\n\t.reg .b32 b0, b1;\n\t"
+        "mov.b64 {b0, b1}, %8;\n\t"
+        "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {b0,b1}, {%0,%1,%2,%3};\n\t}"
+        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "l"(b));
+}
+// Two 16-bit indices packed in one word -> the shared addresses base + 4 * index of both.
+__device__ __forceinline__ void im_pair_addr(uint32_t pair, uint32_t base, uint32_t &lo, uint32_t &hi) {
+    asm("{\n\t.reg .u16 l, h;\n\t"
+        "mov.b32 {l, h}, %2;\n\t"
+        "mad.wide.u16 %0, l, 4, %3;\n\t"
+        "mad.wide.u16 %1, h, 4, %3;\n\t}"
+        : "=r"(lo), "=r"(hi) : "r"(pair), "r"(base));
+}
+__device__ __forceinline__ uint32_t im_lds32(uint32_t addr) {
+    uint32_t v;
+    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(addr));
+    return v;
 }
 __device__ __forceinline__ void im_named_bar(int id, int threads) {
     asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
 }
 
-// Two packed fp16 (dt = BTC_F16) or bf16 numbers -> two floats.
-__device__ __forceinline__ void im_unpack2(uint32_t w, int dt, float &lo, float &hi)
+// Eight consecutive activations of a row of x starting at element k0 (a multiple of 8) as floats.
+__device__ __forceinline__ void im_load8(const void *xrow, int dt, int k0, float (&f)[8])
 {
-    if (dt == BTC_F16) {
-        const float2 f = __half22float2(*reinterpret_cast<const __half2 *>(&w));
-        lo = f.x; hi = f.y;
+    if (dt == BTC_F32) {
+        const float4 a = __ldg(reinterpret_cast<const float4 *>(reinterpret_cast<const float *>(xrow) + k0));
+        const float4 b = __ldg(reinterpret_cast<const float4 *>(reinterpret_cast<const float *>(xrow) + k0) + 1);
+        f[0] = a.x; f[1] = a.y; f[2] = a.z; f[3] = a.w; f[4] = b.x; f[5] = b.y; f[6] = b.z; f[7] = b.w;
     } else {
-        lo = __uint_as_float(w << 16);
-        hi = __uint_as_float(w & 0xffff0000u);
+        const uint4 q = __ldg(reinterpret_cast<const uint4 *>(reinterpret_cast<const uint16_t *>(xrow) + k0));
+        const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            if (dt == BTC_F16) {
+                const float2 p = __half22float2(*reinterpret_cast<const __half2 *>(&w[i]));
+                f[2 * i] = p.x; f[2 * i + 1] = p.y;
+            } else {
+                f[2 * i] = __uint_as_float(w[i] << 16);
+                f[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
+            }
+        }
     }
+}
+
+// Eight fp16 (dt = BTC_F16) or bf16 numbers held in a uint4 -> floats.
+__device__ __forceinline__ void im_cvt8(const uint4 &q, int dt, float *f)
+{
+    const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        if (dt == BTC_F16) {
+            const float2 p = __half22float2(*reinterpret_cast<const __half2 *>(&w[i]));
+            f[2 * i] = p.x; f[2 * i + 1] = p.y;
+        } else {
+            f[2 * i] = __uint_as_float(w[i] << 16);
+            f[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
+        }
+    }
+}
+
+// Block-fixed-point scale of one K-slice of a row of x from the largest magnitude any lane saw (reduced over the warp
+// here): X = rint(x * sc) has |X| <= 2^pbits, inv = 1 / sc, both powers of two.  A slice of zeros gives sc = inv = 0;
+// a slice holding an inf or a nan gives inv = nan, so every output of that row of x becomes a nan, as the exact product
+// would.
+__device__ __forceinline__ void im_slice_scale(float amax, int pbits, float &sc, float &inv)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+    // amax = f * 2^e with f in [1, 2) (a float widened from fp16 / bf16 is normal or zero; an fp32 subnormal counts
+    // as tiny): |x| < 2^(e+1)
+    const int ex = max((int)((__float_as_uint(amax) >> 23) & 0xffu) - 127 + 1, -100);
+    const bool nz = amax > 0.f && amax < 3.0e38f;
+    sc = nz ? __uint_as_float((uint32_t)(127 + pbits - ex) << 23) : 0.0f;
+    inv = nz ? __uint_as_float((uint32_t)(127 - pbits + ex) << 23) : (amax == 0.f ? 0.0f : __uint_as_float(0x7fc00000u));
 }
 
 // Shared-memory layout (dynamic), offsets computed identically on host and device.
 struct ImSmem {
-    uint32_t bars;        // mbarriers: full[S], empty[S], part_full[2], part_empty[2], tab_full, tab_free
-    uint32_t misc;        // abort flag, per-part scale slots
-    uint32_t rowsc;       // alpha and mu of the rows of the current chunk, float [2][IM_RC * 32]
+    uint32_t bars;        // mbarriers: full[S], empty[S], tab_full
+    uint32_t misc;        // abort flag; per compute warp and row m of x: its share of sum_k x
     uint32_t planes;      // per compute warp: digit planes of its K-slice of one row of x
     uint32_t tab;         // codeword table
     uint32_t ring;        // index stages
-    uint32_t part;        // partial sums, two buffers: digit sums int [16 warps][16 rows][8 cols] (M <= 2), else partial dot
-                          // products float [tile][16 rows][m][K-slice]
-    uint32_t acc;         // dot products summed over K-parts, float [IM_RC][rows][cols / 2]
+    uint32_t part;        // partial dot products, float [tile of the chunk][16 rows][MAXM][8 slices]
     uint32_t total;
 };
-constexpr int IM_NBARS = 2 * IM_STAGES + 6;
-constexpr int IM_SLOTS = 4;                      // scale slots: K-parts whose partial sums may still be in flight
-struct ImScale { float inv; float sx; };         // per (slot, compute warp, row m of x): 1/scale (a power of two), and
-                                                 // the warp's share of sum_k x over the slice
-constexpr int IM_MISC_BYTES = 16 + IM_SLOTS * IM_CWARPS * 8 * (int)sizeof(ImScale) + IM_CWARPS * 4;
-constexpr int IM_PLANE_WORDS = 3 * (IM_PW + 64) * 5;   // all K-slices: 3 digits x (256 blocks + skew) x (v / 4 <= 5) words
+constexpr int IM_NBARS = 2 * IM_STAGES + 1;
+constexpr int IM_MISC_BYTES = 16 + IM_CWARPS * 8 * 4;
 
-__host__ __device__ inline ImSmem im_smem_layout(int tab_bytes, int cols, int rows, int stages)
+// NM = 1: the integer form (M <= 2, one MMA per A fragment).  NM = 0: the fp16 form (M <= 8).
+template <int NM> struct ImShape {
+    static constexpr int PW = (NM == 1) ? 256 : 128;           // blocks per K-part
+    static constexpr int SLICE = PW / IM_CWARPS;               // blocks per compute warp
+    static constexpr int BPL = SLICE / 4;                      // blocks per lane
+    static constexpr int MAXM = (NM == 1) ? 2 : 8;
+    static constexpr int RC = 12;                              // tiles a CTA walks part by part at a time
+    static constexpr int PROW = RC * 16 + 4;                   // NM = 0: floats per (slice, m) row of the partial sums
+    static constexpr int STAGE_BYTES = PW / IM_BOX_COLS * IM_BOX_BYTES;
+};
+
+__host__ __device__ inline ImSmem im_smem_layout(int tab_bytes, int nm, int stages)
 {
+    const int slice = (nm == 1 ? 256 : 128) / IM_CWARPS;
+    const int maxm = nm == 1 ? 2 : 8;
+    const int rc = 12;
+    const int stage_bytes = (nm == 1 ? 256 : 128) / IM_BOX_COLS * IM_BOX_BYTES;
     ImSmem L;
     uint32_t o = 0;
     L.bars = o; o += IM_NBARS * 8;
     o = (o + 15u) & ~15u;
     L.misc = o; o += IM_MISC_BYTES;
     o = (o + 15u) & ~15u;
-    L.rowsc = o; o += 2u * IM_RC * 32u * 4u;
-    L.planes = o; o += IM_PLANE_WORDS * 4;
+    L.planes = o;
+    if (nm != 0) o += (uint32_t)IM_CWARPS * 3u * (uint32_t)(slice + 4) * 5u * 4u;   // 3 digits x (blocks + skew) x (v / 4 <= 5) words
+    o = (o + 15u) & ~15u;
+    L.part = o;
+    o += (nm == 0) ? (uint32_t)IM_CWARPS * (uint32_t)maxm * (uint32_t)(rc * 16 + 4) * 4u
+                   : (uint32_t)rc * 16u * (uint32_t)maxm * IM_CWARPS * 4u;
     o = (o + 127u) & ~127u;
     L.tab = o; o += (uint32_t)tab_bytes;
     o = (o + 1023u) & ~1023u;                     // swizzled TMA boxes want 1024-byte alignment
-    L.ring = o; o += (uint32_t)stages * IM_STAGE_BYTES;
-    // cols == 8 (M <= 2): a 16 x 8 tile of digit sums per compute warp; else one float per (warp, row, m)
-    L.part = o; o += 2u * IM_CWARPS * 16u * (uint32_t)(cols == 8 ? 8 : (cols == 16 ? 5 : 8)) * 4u;
-    L.acc = o; o += (uint32_t)IM_RC * (uint32_t)rows * (uint32_t)(cols / 2) * 4u;
+    L.ring = o; o += (uint32_t)stages * (uint32_t)stage_bytes;
     L.total = o;
     return L;
 }
 
-// Row groups [lo, hi) of layer P that fall to CTA b: the layer's cta_count CTAs split its row groups evenly (the first
+// Tiles [lo, hi) of layer P that fall to CTA b: the layer's cta_count CTAs split its tiles evenly (the first
 // `rem` of them take one more); per and rem come from the host, so no division runs here.
 __device__ __forceinline__ void im_group_range(const ImProblem &P, int b, int &lo, int &hi)
 {
@@ -211,50 +294,31 @@ __device__ __forceinline__ void im_group_range(const ImProblem &P, int b, int &l
 // shared memory, the rest from global memory; 3: whole tables in shared memory as 16-bit halves (v <= 16; a table of
 // 65536 codewords then takes 128 KB), widened by `h | (h << 12)` after the gather.
 template <int NCLS, int NM, int TAB_MODE>
-__global__ void __launch_bounds__(IM_THREADS, 1)
+__global__ void __launch_bounds__(IM_THREADS, 2)
 gemv_imma_kernel(const __grid_constant__ ImBatch batch)
 {
     extern __shared__ __align__(128) unsigned char smem[];
-    constexpr int TRK = (NM == 1) ? 2 : 1;               // 16-row tiles per row group
-    constexpr int ROWS = TRK * 16;
-    constexpr int COLS = 8 * NM;
-    constexpr int KS = 16 / TRK;                         // K-slices of a part; warp w: slice w % KS, tile w / KS
-    constexpr int SLICE = IM_PW / KS;                    // blocks per slice
-    constexpr int BPL = SLICE / 4;                       // blocks per lane
-    constexpr int MAXM = (NM == 1) ? 2 : (NM == 2 ? 5 : 8);
-    const ImSmem L = im_smem_layout(batch.tab_smem_bytes, COLS, ROWS, batch.stages);
+    using S = ImShape<NM>;
+    constexpr int PW = S::PW, SLICE = S::SLICE, BPL = S::BPL, MAXM = S::MAXM, RC = S::RC;
+    constexpr int STAGE_BYTES = S::STAGE_BYTES;
+    const ImSmem L = im_smem_layout(batch.tab_smem_bytes, NM, batch.stages);
     const int NST = batch.stages;
     uint64_t *bars = reinterpret_cast<uint64_t *>(smem + L.bars);
     volatile int *s_abort = reinterpret_cast<volatile int *>(smem + L.misc);
-    ImScale *s_scale = reinterpret_cast<ImScale *>(smem + L.misc + 16);           // [IM_SLOTS][16 warps][8]
-    float *s_xmax = reinterpret_cast<float *>(smem + L.misc + 16 + IM_SLOTS * IM_CWARPS * 8 * sizeof(ImScale));   // [16 warps]
+    float *s_sx = reinterpret_cast<float *>(smem + L.misc + 16);                  // [8 warps][8]
     uint32_t *s_planes = reinterpret_cast<uint32_t *>(smem + L.planes);
     uint32_t *s_tab = reinterpret_cast<uint32_t *>(smem + L.tab);
     unsigned char *s_ring = smem + L.ring;
-    // Who recombines the three digit sums of a (K-slice, row, m): with M <= 2 the compute warps set the pace, so they
-    // hand over their raw 16 x 8 integer tiles and the epilogue warps recombine; with more rows of x the epilogue
-    // would fall behind, so each compute warp recombines its own sums and hands over one float per (row, m).
-    constexpr bool FPART = (NM > 1);
-    constexpr int TILE_INTS = 16 * COLS;                 // one compute warp's integer tile
     float *s_part = reinterpret_cast<float *>(smem + L.part);
-    int *s_parti = reinterpret_cast<int *>(smem + L.part);
-    float *s_acc = reinterpret_cast<float *>(smem + L.acc);
-    float *s_alpha = reinterpret_cast<float *>(smem + L.rowsc), *s_mu = s_alpha + IM_RC * 32;
-    constexpr int ACC_M = COLS / 2;                      // floats per row of s_acc (>= MAXM)
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     auto bar_full = [&](int s) { return im_smem_u32(bars + s); };
     auto bar_empty = [&](int s) { return im_smem_u32(bars + IM_STAGES + s); };
-    auto bar_pfull = [&](int b) { return im_smem_u32(bars + 2 * IM_STAGES + b); };
-    auto bar_pempty = [&](int b) { return im_smem_u32(bars + 2 * IM_STAGES + 2 + b); };
-    const uint32_t bar_tabfull = im_smem_u32(bars + 2 * IM_STAGES + 4);
-    const uint32_t bar_tabfree = im_smem_u32(bars + 2 * IM_STAGES + 5);
+    const uint32_t bar_tabfull = im_smem_u32(bars + 2 * IM_STAGES);
 
     if (tid == 0) {
         for (int s = 0; s < NST; ++s) { im_mbar_init(bar_full(s), 1); im_mbar_init(bar_empty(s), IM_CWARPS); }
-        for (int b = 0; b < 2; ++b) { im_mbar_init(bar_pfull(b), IM_CWARPS); im_mbar_init(bar_pempty(b), IM_EWARPS); }
         im_mbar_init(bar_tabfull, 1);
-        im_mbar_init(bar_tabfree, IM_CWARPS);
         *s_abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -263,340 +327,518 @@ gemv_imma_kernel(const __grid_constant__ ImBatch batch)
     constexpr bool tab_smem = TAB_MODE != 0;             // (part of) the codeword table is staged in shared memory
     const uint32_t tab_head = (uint32_t)batch.tab_head;
 
-    // All three roles walk the same sequence: layers pi (those with row groups for this CTA, counted
-    // by ps), chunks [c0, c1) of at most IM_RC row groups, K-parts j (counted by pc), row groups r; li
-    // counts iterations.
-    if (warp == IM_CWARPS) {
-        // ============================================================ producer
-        int li = 0, ps = 0;
-        int s = 0;                                             // ring stage li % NST; rph = (li / NST) & 1
-        uint32_t rph = 0;
-        bool ok = true;
-        for (int pi = 0; pi < batch.count && ok; ++pi) {
-            const ImProblem &P = batch.p[pi];
-            int glo, ghi;
-            im_group_range(P, (int)blockIdx.x, glo, ghi);
-            if (glo >= ghi) continue;
-            if (tab_smem) {
-                if (ps > 0 && !im_mbar_wait(bar_tabfree, (ps - 1) & 1, s_abort)) break;
-                if (lane == 0) {
-                    const uint32_t bytes = TAB_MODE == 3 ? (uint32_t)((P.Kc + 7) / 8 * 8 * 2)
-                                                         : (uint32_t)(min((P.Kc + 3) / 4 * 4, batch.tab_head) * 4);
-                    im_mbar_expect_tx(bar_tabfull, bytes);
-                    im_bulk_g2s(im_smem_u32(s_tab), TAB_MODE == 3 ? static_cast<const void *>(P.tab16) : static_cast<const void *>(P.tab),
-                                bytes, bar_tabfull);
-                }
+    // the one layer this CTA works on, and its tiles
+    int pi = 0, glo = 0, ghi = 0;
+    for (; pi < batch.count; ++pi) {
+        im_group_range(batch.p[pi], (int)blockIdx.x, glo, ghi);
+        if (glo < ghi) break;
+    }
+    if (pi < batch.count) {
+        const ImProblem &P = batch.p[pi];
+        // Both roles walk the same sequence: chunks [c0, c1) of at most RC tiles, K-parts j, tiles r.
+        if (warp == IM_CWARPS) {
+            // ============================================================ producer
+            if (tab_smem && lane == 0) {
+                const uint32_t bytes = TAB_MODE == 3 ? (uint32_t)((P.Kc + 7) / 8 * 8 * 2)
+                                                     : (uint32_t)(min((P.Kc + 3) / 4 * 4, batch.tab_head) * 4);
+                im_mbar_expect_tx(bar_tabfull, bytes);
+                im_bulk_g2s(im_smem_u32(s_tab), TAB_MODE == 3 ? static_cast<const void *>(P.tab16) : static_cast<const void *>(P.tab),
+                            bytes, bar_tabfull);
             }
-            ++ps;
-            for (int c0 = glo; c0 < ghi && ok; c0 += IM_RC) {
-                const int c1 = min(c0 + IM_RC, ghi);
+            int li = 0, s = 0;                                     // ring stage li % NST; rph = (li / NST) & 1
+            uint32_t rph = 0;
+            bool ok = true;
+            for (int c0 = glo; c0 < ghi && ok; c0 += RC) {
+                const int c1 = min(c0 + RC, ghi);
                 for (int j = 0; j < P.parts && ok; ++j) {
-                    const int pw = min(IM_PW, P.Kb - j * IM_PW);          // blocks of this part
+                    // every stage is filled whole (boxes of 64 blocks x 16 rows): rows past N and blocks past K/v arrive
+                    // as zeros, so a consumer never meets an index left behind by an earlier stage
+                    constexpr int nbox = PW / IM_BOX_COLS;
                     for (int r = c0; r < c1; ++r, ++li) {
                         if (li >= NST && !im_mbar_wait(bar_empty(s), rph ^ 1u, s_abort)) { ok = false; break; }
-                        // boxes of 64 blocks x ROWS rows; rows past N and blocks past K/v arrive as zeros
-                        const int nbox = (pw + IM_BOX_COLS - 1) / IM_BOX_COLS;
-                        constexpr uint32_t BOX_BYTES = ROWS * 128;
-                        if (lane == 0) im_mbar_expect_tx(bar_full(s), (uint32_t)nbox * BOX_BYTES);
+                        if (lane == 0) im_mbar_expect_tx(bar_full(s), (uint32_t)nbox * IM_BOX_BYTES);
                         __syncwarp();
                         if (lane < nbox)
-                            im_tma_2d(im_smem_u32(s_ring + (size_t)s * IM_STAGE_BYTES + (size_t)lane * BOX_BYTES), &batch.map[pi],
-                                      j * IM_PW + lane * IM_BOX_COLS, r * ROWS, bar_full(s));
+                            im_tma_2d(im_smem_u32(s_ring + (size_t)s * STAGE_BYTES + (size_t)lane * IM_BOX_BYTES), &batch.map[pi],
+                                      j * PW + lane * IM_BOX_COLS, r * 16, bar_full(s));
                         if (++s == NST) { s = 0; rph ^= 1u; }
                     }
                 }
             }
-        }
-    } else if (warp > IM_CWARPS) {
-        // ============================================================ epilogue (two warps)
-        // 64 threads = ROWS rows x SPLIT groups of compute warps; the groups of a row sit in adjacent lanes.
-        constexpr int SPLIT = (IM_EWARPS * 32) / ROWS;         // 2 or 4
-        constexpr int WPG = KS / SPLIT;                        // compute warps (K-slices) per group: 4
-        const int et = (warp - IM_CWARPS - 1) * 32 + lane;
-        const int R = et / SPLIT, grp = et % SPLIT;
-        asm volatile("griddepcontrol.wait;" ::: "memory");
-        int li = 0, pc = 0;
-        bool ok = true;
-        for (int pi = 0; pi < batch.count && ok; ++pi) {
-            const ImProblem &P = batch.p[pi];
-            int glo, ghi;
-            im_group_range(P, (int)blockIdx.x, glo, ghi);
-            if (glo >= ghi) continue;
-            const float unshift2 = 2.0f / (float)(1 << (P.ncls - 1));
-            for (int c0 = glo; c0 < ghi && ok; c0 += IM_RC) {
-                const int c1 = min(c0 + IM_RC, ghi);
-                float sxtot[MAXM];                               // sum_k x[m, k] over the parts seen so far
-#pragma unroll
-                for (int m = 0; m < MAXM; ++m) sxtot[m] = 0.f;
-                // alpha / mu of this thread's row in every row group of the chunk go to shared memory once per chunk (each
-                // thread reads back only what it wrote, so no barrier is needed): the loads, a trip to DRAM, overlap the
-                // compute warps' fragment build instead of sitting in every iteration's chain
-                if (grp == 0) {
-                    unsigned short ab[IM_RC], mb[IM_RC];
-#pragma unroll
-                    for (int i = 0; i < IM_RC; ++i) {                // all loads in flight together
-                        const int n = (c0 + i) * ROWS + R;
-                        ab[i] = 0; mb[i] = 0;
-                        if (i < c1 - c0 && n < P.N) {
-                            ab[i] = __ldg(reinterpret_cast<const unsigned short *>(P.alpha) + n);
-                            if (P.mu) mb[i] = __ldg(reinterpret_cast<const unsigned short *>(P.mu) + n);
-                        }
-                    }
-#pragma unroll
-                    for (int i = 0; i < IM_RC; ++i) {
-                        s_alpha[i * ROWS + R] = __half2float(__ushort_as_half(ab[i]));
-                        s_mu[i * ROWS + R] = __half2float(__ushort_as_half(mb[i]));
-                    }
-                }
-                for (int j = 0; j < P.parts && ok; ++j, ++pc) {
-                    const bool last = (j == P.parts - 1);
-                    const ImScale *sc = s_scale + (size_t)(pc % IM_SLOTS) * IM_CWARPS * 8;
-                    float sxp[MAXM];                             // sum_k x[m, k] over this part (fixed order of warps)
-#pragma unroll
-                    for (int m = 0; m < MAXM; ++m) sxp[m] = 0.f;
-                    for (int r = c0; r < c1; ++r, ++li) {
-                        const int buf = li & 1;
-                        const int n = r * ROWS + R;
-                        const bool live = (n < P.N) && (grp == 0);
-                        if (!im_mbar_wait(bar_pfull(buf), (li >> 1) & 1, s_abort)) { ok = false; break; }
-                        const float al = s_alpha[(r - c0) * ROWS + R], mu = s_mu[(r - c0) * ROWS + R];
-                        if (r == c0) {
-#pragma unroll
-                            for (int m = 0; m < MAXM; ++m)
-                                if (m < P.M)
-                                    for (int w = 0; w < IM_CWARPS; ++w) sxp[m] += sc[w * 8 + m].sx;
-#pragma unroll
-                            for (int m = 0; m < MAXM; ++m) sxtot[m] += sxp[m];
-                        }
-                        float *accrow = s_acc + ((size_t)(P.parts > 1 ? (r - c0) : 0) * ROWS + R) * ACC_M;
-                        float dots[MAXM];
-                        if constexpr (FPART) {
-                            // row R lies in tile R / 16; its K-slices' partial dot products sit side by side
-                            const float *base = s_part + ((((size_t)buf * TRK + (R >> 4)) * 16 + (R & 15)) * MAXM) * KS + grp * WPG;
-#pragma unroll
-                            for (int m = 0; m < MAXM; ++m) {
-                                dots[m] = 0.f;
-                                if (m < P.M) {
-                                    const float4 q = *reinterpret_cast<const float4 *>(base + m * KS);
-                                    dots[m] = ((q.x + q.y) + q.z) + q.w;
-                                }
-                            }
-                        } else {
-                            // row R lies in tile R / 16, written by the compute warps (R / 16) * KS + slice
-                            const int *base = s_parti + ((size_t)buf * IM_CWARPS + (R >> 4) * KS + grp * WPG) * TILE_INTS + (size_t)(R & 15) * COLS;
-#pragma unroll
-                            for (int m = 0; m < MAXM; ++m) dots[m] = 0.f;
-#pragma unroll
-                            for (int w = 0; w < WPG; ++w) {
-                                int pv[COLS];
-#pragma unroll
-                                for (int c4 = 0; c4 < COLS / 4; ++c4) {
-                                    if (c4 * 4 < 3 * P.M) {                 // columns 3 m + d, m < M
-                                        const int4 q = *reinterpret_cast<const int4 *>(base + (size_t)w * TILE_INTS + c4 * 4);
-                                        pv[c4 * 4] = q.x; pv[c4 * 4 + 1] = q.y; pv[c4 * 4 + 2] = q.z; pv[c4 * 4 + 3] = q.w;
-                                    } else {
-                                        pv[c4 * 4] = pv[c4 * 4 + 1] = pv[c4 * 4 + 2] = pv[c4 * 4 + 3] = 0;
-                                    }
-                                }
-#pragma unroll
-                                for (int m = 0; m < MAXM; ++m) {
-                                    if (m < P.M) {
-                                        // each digit sum is below 2^24 in magnitude, so the conversions are exact
-                                        const float T = ((float)pv[3 * m + 2] * 256.0f + (float)pv[3 * m + 1]) * 256.0f + (float)pv[3 * m];
-                                        dots[m] += T * sc[(grp * WPG + w) * 8 + m].inv;
-                                    }
-                                }
-                            }
-                        }
-                        __syncwarp();
-                        if (lane == 0) im_mbar_arrive(bar_pempty(buf));
-#pragma unroll
-                        for (int m = 0; m < MAXM; ++m) {
-                            if (m < P.M) {
-#pragma unroll
-                                for (int o = 1; o < SPLIT; o <<= 1) dots[m] += __shfl_xor_sync(0xffffffffu, dots[m], o);
-                                float dot = dots[m] * unshift2 - sxp[m];        // 2 * sum_{bit=1} x - sum x over this part
-                                if (grp == 0) {
-                                    if (j > 0) dot += accrow[m];
-                                    if (!last) accrow[m] = dot;
-                                }
-                                if (last && live) {
-                                    const float yv = al * dot + mu * sxtot[m];
-                                    store_from_float(P.y, P.y_dt, (size_t)m * P.N + n, yv);
-                                }
-                            }
-                        }
-                    }
-                }
-            }
-        }
-    } else {
-        // ============================================================ compute warps
-        const int g = lane >> 2, t = lane & 3;
-        constexpr float MAGIC = 12582912.0f;                   // 1.5 * 2^23: float -> int by addition
-        constexpr int MAGIC_BITS = 0x4B400000;
-        const int ks = warp % KS, rh = warp / KS;             // K-slice and tile of this warp
-        // MMA row g (and g + 8) carries tile row sg (and sg + 8): neighbouring g differ in bit 2 of the row, so the
-        // eight lanes of a shared-memory phase read distinct swizzled chunks
-        const int sg = ((g & 1) << 2) | (g >> 1);
-        // digit planes of a slice: block b, class c of digit d at word d * PSW + (b + b / BPL) * NCLS + c; the skew
-        // puts the lanes of a fragment read (t: blocks BPL apart, d: planes) on different banks
-        constexpr int PSW = (SLICE + 4) * NCLS;
-        uint32_t *planes = s_planes + ks * (3 * PSW);
-        asm volatile("griddepcontrol.wait;" ::: "memory");
-        int li = 0, ps = 0, pc = 0;
-        int s = 0;                                             // ring stage li % NST; rph = (li / NST) & 1
-        uint32_t rph = 0;
-        bool ok = true;
-        for (int pi = 0; pi < batch.count && ok; ++pi) {
-            const ImProblem &P = batch.p[pi];
-            int glo, ghi;
-            im_group_range(P, (int)blockIdx.x, glo, ghi);
-            if (glo >= ghi) continue;
+        } else {
+            // ============================================================ compute warps
+            if constexpr (NM == 0) {
+            // ---- fp16 form (M <= 8).  An fp16 bit pattern with one bit p <= 14 set is the number 2^(p-24), so the
+            // codeword word of the "fp16 layout" (weight t at bit (t & 1) * 16 + P0 + (t >> 1), P0 = 12 - v/2) masked
+            // with one bit per half IS a pair of multiplicands {0 or 2^(P0+i-24)} for the weights 2i, 2i+1: one LOP3
+            // per two weights, no conversion.  mma.sync.m16n8k16 (fp16 x fp16 -> fp32):
+            //   A (16 rows x 16 k) = masked codeword bits: lane (g, t) supplies, for rows g and g + 8, four weights
+            //       (class c = weights 4c .. 4c+3) of a block it owns; the four lanes of a quad own four blocks;
+            //   B (16 k x 8 cols)  = the activations of row m = column, as fp16, scaled per K-slice by 2^(E-i) so that
+            //       every product is bit * x * 2^(E+P0-24) exactly (E from the slice's largest magnitude: no overflow);
+            //   D (16 x 8, fp32)   = sums over set bits for 16 outputs x 8 rows of x, fp32 accumulation.
+            // The sum of the slice's activations (for the identity's "- sum x" and the mean term) comes from the same
+            // MMAs with all mask bits as A.  The cost does not depend on M.
+            const int g = lane >> 2, t = lane & 3;
+            const int ks = warp;
+            const int sg = ((g & 1) << 2) | (g >> 1);
             const int M = P.M, K = P.K, Kb = P.Kb, v = P.v;
-            const int cmax = P.ncls - 1;
-            const int PBITS = 22 - cmax;                       // |X| <= 2^PBITS
-            const int ngroups = SLICE * v / 8;                 // groups of 8 activations in a slice (<= 80)
+            const int P0 = 12 - v / 2;
+            constexpr int PROW = S::PROW;
+            uint32_t pm[2 * NCLS];                                 // mask of pair i: bit P0 + i of both halves
+#pragma unroll
+            for (int i = 0; i < 2 * NCLS; ++i) pm[i] = (2 * i < v) ? (0x00010001u << (P0 + i)) : 0u;
+            const uint32_t *gtab = P.tab;
+            const int xsz = (P.x_dt == BTC_F32) ? 4 : 2;
             bool tab_ready = !tab_smem;
-            const uint32_t *gtab = P.tab;                      // (s_tab is named directly below so that its loads are shared-memory loads)
+            bool ok = true;
+            int s = 0;
+            uint32_t rph = 0;
+            const int boff = (ks * SLICE + BPL * t) * 2;
+            const uint32_t idx_off = (uint32_t)(boff >> 7) * IM_BOX_BYTES + (uint32_t)sg * 128
+                                     + ((((boff >> 4) & 7) ^ (sg & 7)) << 4) + (boff & 15);
+            const int ct = tid;
+            for (int c0 = glo; c0 < ghi; c0 += RC) {
+                const int c1 = min(c0 + RC, ghi);
+                const int nrows = (c1 - c0) * 16;
+                const int nout = nrows * M;
+                constexpr int OPT = (RC * 16 * MAXM + IM_CWARPS * 32 - 1) / (IM_CWARPS * 32);
+                unsigned short areg[OPT], mreg[OPT];
+#pragma unroll
+                for (int q = 0; q < OPT; ++q) {
+                    const int o = ct + q * (IM_CWARPS * 32);
+                    areg[q] = 0; mreg[q] = 0;
+                    if (o < nout) {
+                        const int n = c0 * 16 + (o % nrows);
+                        if (n < P.N) {
+                            areg[q] = __ldg(reinterpret_cast<const unsigned short *>(P.alpha) + n);
+                            if (P.mu) mreg[q] = __ldg(reinterpret_cast<const unsigned short *>(P.mu) + n);
+                        }
+                    }
+                }
+                if (c0 == glo) asm volatile("griddepcontrol.wait;" ::: "memory");
+                float sx0 = 0.f, sx1 = 0.f;                        // lanes g = 0: this slice's sum_k x[m, k], m = 2t, 2t+1
 
-            for (int c0 = glo; c0 < ghi && ok; c0 += IM_RC) {
-                const int c1 = min(c0 + IM_RC, ghi);
-                for (int j = 0; j < P.parts && ok; ++j, ++pc) {
-                    const int pw = min(IM_PW, Kb - j * IM_PW);
-                    const int jb0 = j * IM_PW + ks * SLICE;         // first block of this warp's slice
-                    const bool wvalid = ks * SLICE + BPL * t < pw;  // this lane's blocks exist (pw % 8 == 0)
-                    const int kend = (j * IM_PW + pw) * v;          // end of the part in x
-                    // byte offset of this lane's index chunk inside a stage (128-byte swizzle: 16-byte chunk c of row q
-                    // sits at chunk c ^ (q & 7)); rows sg and sg + 8 of tile rh
-                    const int boff = (ks * SLICE + BPL * t) * 2;
-                    const int irow = rh * 16 + sg;
-                    const uint32_t idx_off = (uint32_t)(boff >> 7) * (ROWS * 128) + (uint32_t)irow * 128
-                                             + ((((boff >> 4) & 7) ^ (irow & 7)) << 4) + (boff & 15);
-                    ImScale *scale_out = s_scale + ((size_t)(pc % IM_SLOTS) * IM_CWARPS + warp) * 8;
-
-                    // ---- B fragments for this part.  The warp's slice of each row of x (16 blocks) is
-                    //      quantised with its own scale: X = rint(x * 2^(PBITS - e)), 2^e > max |x| of the slice.
-                    uint32_t breg[BPL][NCLS][NM];
+                for (int j = 0; j < P.parts; ++j) {
+                    const int pw = min(PW, Kb - j * PW);
+                    const bool wvalid = ks * SLICE + BPL * t < pw;
+                    // ---- B fragments: lane (g = m, t) reads the activations of row m for its own BPL blocks
+                    uint64_t breg[BPL][NCLS];
+                    const bool has = wvalid && g < M;
+                    const unsigned char *xrow = reinterpret_cast<const unsigned char *>(P.x) + (size_t)g * K * xsz;
+                    // 16-bit activations: all of this lane's loads are issued before anything uses them; with v = 16 a
+                    // lane's four blocks are 128 contiguous bytes, read 16 bytes (two classes) at a time
+                    uint2 raw[BPL][NCLS];
+                    const bool x16 = P.x_dt != BTC_F32;
+                    if (NCLS == 4 && v == 16) {
+#pragma unroll
+                        for (int e = 0; e < BPL; ++e)
+#pragma unroll
+                            for (int c = 0; c < NCLS; c += 2) {
+                                uint4 q = make_uint4(0u, 0u, 0u, 0u);
+                                if (x16 && has)
+                                    q = __ldg(reinterpret_cast<const uint4 *>(
+                                        xrow + ((size_t)(j * PW + ks * SLICE + BPL * t + e) * 16 + 4 * c) * 2));
+                                raw[e][c] = make_uint2(q.x, q.y);
+                                raw[e][c + 1] = make_uint2(q.z, q.w);
+                            }
+                    } else {
+#pragma unroll
+                        for (int e = 0; e < BPL; ++e)
+#pragma unroll
+                            for (int c = 0; c < NCLS; ++c) {
+                                raw[e][c] = make_uint2(0u, 0u);
+                                if (x16 && has && 4 * c < v)
+                                    raw[e][c] = __ldg(reinterpret_cast<const uint2 *>(
+                                        xrow + ((size_t)(j * PW + ks * SLICE + BPL * t + e) * v + 4 * c) * 2));
+                            }
+                    }
+                    // the four activations of class c of this lane's block e, as floats (fp32 activations are read from
+                    // memory twice: once for the largest magnitude, once to scale; the second read is served by L1)
+                    auto x4 = [&](int e, int c, float (&f)[4]) {
+                        f[0] = f[1] = f[2] = f[3] = 0.f;
+                        if (x16) {
+                            const uint2 q = raw[e][c];
+                            if (P.x_dt == BTC_F16) {
+                                const float2 a = __half22float2(*reinterpret_cast<const __half2 *>(&q.x));
+                                const float2 b = __half22float2(*reinterpret_cast<const __half2 *>(&q.y));
+                                f[0] = a.x; f[1] = a.y; f[2] = b.x; f[3] = b.y;
+                            } else {
+                                f[0] = __uint_as_float(q.x << 16); f[1] = __uint_as_float(q.x & 0xffff0000u);
+                                f[2] = __uint_as_float(q.y << 16); f[3] = __uint_as_float(q.y & 0xffff0000u);
+                            }
+                        } else if (has && 4 * c < v) {
+                            const size_t k0 = (size_t)(j * PW + ks * SLICE + BPL * t + e) * v + 4 * c;
+                            const float4 q = __ldg(reinterpret_cast<const float4 *>(xrow + k0 * 4));
+                            f[0] = q.x; f[1] = q.y; f[2] = q.z; f[3] = q.w;
+                        }
+                    };
+                    float amax = 0.f;
 #pragma unroll
                     for (int e = 0; e < BPL; ++e)
 #pragma unroll
-                        for (int c = 0; c < NCLS; ++c)
+                        for (int c = 0; c < NCLS; ++c) {
+                            float f[4];
+                            x4(e, c, f);
+                            amax = fmaxf(fmaxf(amax, fmaxf(fabsf(f[0]), fabsf(f[1]))), fmaxf(fabsf(f[2]), fabsf(f[3])));
+                        }
+                    // largest magnitude of (row m, slice): over the four lanes of the quad
+                    amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 1));
+                    amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 2));
+                    // amax = f * 2^e, f in [1, 2): x * 2^(14 - e) stays below 2^15
+                    int E = 14 - ((int)((__float_as_uint(amax) >> 23) & 0xffu) - 127);
+                    E = min(max(E, -90), 100);
 #pragma unroll
-                            for (int nm = 0; nm < NM; ++nm) breg[e][c][nm] = 0u;
-                    // The TRK warps of a slice share its planes: each quantises every TRK-th group of 8 activations.
-                    constexpr int NU = (SLICE * 20 / 8 + 32 * TRK - 1) / (32 * TRK);   // groups per lane (v <= 20)
-                    auto slice_sync = [&]() {
-                        if (TRK == 1) __syncwarp();
-                        else im_named_bar(1 + ks, TRK * 32);
-                    };
-                    for (int m = 0; m < M; ++m) {
-                        const uint16_t *xrow = reinterpret_cast<const uint16_t *>(P.x) + (size_t)m * K;
-                        uint4 q4[NU];
-                        float amax = 0.f;
+                    for (int e = 0; e < BPL; ++e) {
 #pragma unroll
-                        for (int u = 0; u < NU; ++u) {
-                            const int gi = lane + 32 * (rh + TRK * u);
-                            const int k0 = jb0 * v + 8 * gi;
-                            q4[u] = make_uint4(0u, 0u, 0u, 0u);
-                            if (gi < ngroups && k0 < kend) q4[u] = __ldg(reinterpret_cast<const uint4 *>(xrow + k0));
-                            const uint32_t wds[4] = {q4[u].x, q4[u].y, q4[u].z, q4[u].w};
+                        for (int c = 0; c < NCLS; ++c) {
+                            float f[4];
+                            x4(e, c, f);
+                            const float s0 = __uint_as_float((uint32_t)(127 + E - 2 * c) << 23);        // 2^(E - i), i = 2c
+                            const float s1 = __uint_as_float((uint32_t)(127 + E - 2 * c - 1) << 23);    // i = 2c + 1
+                            const __half2 h0 = __floats2half2_rn(f[0] * s0, f[1] * s0);
+                            const __half2 h1 = __floats2half2_rn(f[2] * s1, f[3] * s1);
+                            breg[e][c] = (uint64_t)(*reinterpret_cast<const uint32_t *>(&h0))
+                                         | ((uint64_t)(*reinterpret_cast<const uint32_t *>(&h1)) << 32);
+                        }
+                    }
+                    // scale of the two output columns this lane holds (m = 2t, 2t+1): 2^(24 - E_m - P0)
+                    const int Elo = __shfl_sync(0xffffffffu, E, 8 * t), Ehi = __shfl_sync(0xffffffffu, E, 8 * t + 4);
+                    const float us_lo = __uint_as_float((uint32_t)(127 + 24 - Elo - P0) << 23);
+                    const float us_hi = __uint_as_float((uint32_t)(127 + 24 - Ehi - P0) << 23);
+                    {   // sum of the slice's activations: the same MMAs with every mask bit as A
+                        float sa[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-                            for (int jj = 0; jj < 4; ++jj) {
-                                float lo, hi;
-                                im_unpack2(wds[jj], P.x_dt, lo, hi);
-                                amax = fmaxf(amax, fmaxf(fabsf(lo), fabsf(hi)));
+                        for (int e = 0; e < BPL; ++e)
+#pragma unroll
+                            for (int c = 0; c < NCLS; ++c)
+                                im_mma_f16(sa, pm[2 * c], pm[2 * c], pm[2 * c + 1], pm[2 * c + 1], breg[e][c]);
+                        sx0 += sa[0] * us_lo;
+                        sx1 += sa[1] * us_hi;
+                    }
+                    if (!tab_ready) {
+                        ok &= im_mbar_wait(bar_tabfull, 0, s_abort);
+                        tab_ready = true;
+                    }
+                    uint32_t w0[BPL], w1[BPL];
+                    auto fetch = [&]() {
+                        ok &= im_mbar_wait(bar_full(s), rph, s_abort);
+                        const unsigned char *pa = s_ring + (size_t)s * STAGE_BYTES + idx_off;
+                        uint2 qa = *reinterpret_cast<const uint2 *>(pa), qb = *reinterpret_cast<const uint2 *>(pa + 8 * 128);
+                        if (!ok) { qa = make_uint2(0u, 0u); qb = qa; }
+                        // the index loads must have RETURNED before the stage is handed back: the arrive below does not
+                        // wait for loads in flight, and the producer's next copy into this stage may land within a few
+                        // hundred clocks when it comes from L2 (seen as stale half boxes before this line was here)
+                        asm volatile("" :: "r"(qa.x), "r"(qa.y), "r"(qb.x), "r"(qb.y) : "memory");
+                        __syncwarp();
+                        if (lane == 0) im_mbar_arrive(bar_empty(s));
+                        if (++s == NST) { s = 0; rph ^= 1u; }
+                        const uint32_t ia[2] = {qa.x, qa.y}, ib[2] = {qb.x, qb.y};
+                        if constexpr (TAB_MODE == 1) {
+                            const uint32_t tb = im_smem_u32(s_tab);
+#pragma unroll
+                            for (int i = 0; i < 2; ++i) {
+                                uint32_t a0, a1, b0, b1;
+                                im_pair_addr(ia[i], tb, a0, a1);
+                                im_pair_addr(ib[i], tb, b0, b1);
+                                w0[2 * i] = im_lds32(a0); w0[2 * i + 1] = im_lds32(a1);
+                                w1[2 * i] = im_lds32(b0); w1[2 * i + 1] = im_lds32(b1);
+                            }
+                        } else {
+#pragma unroll
+                            for (int e = 0; e < BPL; ++e) {
+                                const uint32_t i0 = (e & 1) ? (ia[e >> 1] >> 16) : (ia[e >> 1] & 0xffffu);
+                                const uint32_t i1 = (e & 1) ? (ib[e >> 1] >> 16) : (ib[e >> 1] & 0xffffu);
+                                if (TAB_MODE == 0) { w0[e] = __ldg(gtab + i0); w1[e] = __ldg(gtab + i1); }
+                                else {
+                                    w0[e] = i0 < tab_head ? s_tab[i0] : __ldg(gtab + i0);
+                                    w1[e] = i1 < tab_head ? s_tab[i1] : __ldg(gtab + i1);
+                                }
                             }
                         }
+                    };
+                    fetch();
+                    for (int r = c0; r < c1; ++r) {
+                        float acc[2][4];
 #pragma unroll
-                        for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
-                        if (TRK > 1) {
-                            if (lane == 0) s_xmax[warp] = amax;
-                            slice_sync();
-                            amax = fmaxf(s_xmax[ks], s_xmax[ks + KS]);
+                        for (int ch = 0; ch < 2; ++ch)
+#pragma unroll
+                            for (int i = 0; i < 4; ++i) acc[ch][i] = 0.f;
+                        if (ks * SLICE < pw) {
+#pragma unroll
+                            for (int e = 0; e < BPL; ++e)
+#pragma unroll
+                                for (int c = 0; c < NCLS; ++c)
+                                    im_mma_f16(acc[(e * NCLS + c) & 1], w0[e] & pm[2 * c], w1[e] & pm[2 * c], w0[e] & pm[2 * c + 1],
+                                               w1[e] & pm[2 * c + 1], breg[e][c]);
                         }
-                        // amax = f * 2^e with f in [1, 2) (a float from fp16 / bf16 is normal or zero): |x| < 2^(e+1)
-                        const int ex = max((int)((__float_as_uint(amax) >> 23) & 0xffu) - 127 + 1, -100);   // (clamped: bf16 can be tinier)
-                        const float sc = (amax > 0.f) ? __uint_as_float((uint32_t)(127 + PBITS - ex) << 23) : 1.0f;
-                        const float inv = (amax > 0.f) ? __uint_as_float((uint32_t)(127 - PBITS + ex) << 23) : 1.0f;
+                        if (r + 1 < c1) fetch();
+                        // rows sg, sg + 8 x columns m = 2t, 2t+1: one float per (slice, m, row); later parts add up
+                        if (2 * t < M) {
+                            const int rl = (r - c0) * 16 + sg;
+                            float *q0 = s_part + (size_t)(ks * MAXM + 2 * t) * PROW + rl, *q1 = q0 + PROW;
+                            const float v00 = (acc[0][0] + acc[1][0]) * us_lo, v01 = (acc[0][1] + acc[1][1]) * us_hi;
+                            const float v10 = (acc[0][2] + acc[1][2]) * us_lo, v11 = (acc[0][3] + acc[1][3]) * us_hi;
+                            if (j == 0) { q0[0] = v00; q1[0] = v01; q0[8] = v10; q1[8] = v11; }
+                            else { q0[0] += v00; q1[0] += v01; q0[8] += v10; q1[8] += v11; }
+                        }
+                    }
+                }
+                if (g == 0) { s_sx[ks * 8 + 2 * t] = sx0; s_sx[ks * 8 + 2 * t + 1] = sx1; }
+                im_named_bar(1, IM_CWARPS * 32);
+                if (ok && !*s_abort) {
+#pragma unroll
+                    for (int q = 0; q < OPT; ++q) {
+                        const int o = ct + q * (IM_CWARPS * 32);
+                        if (o < nout) {
+                            const int m = o / nrows, rl = o - m * nrows;
+                            const int n = c0 * 16 + rl;
+                            float dot1 = 0.f, sx = 0.f;
+#pragma unroll
+                            for (int w = 0; w < IM_CWARPS; ++w) {
+                                dot1 += s_part[(size_t)(w * MAXM + m) * PROW + rl];
+                                sx += s_sx[w * 8 + m];
+                            }
+                            if (n < P.N) {
+                                const float al = __half2float(__ushort_as_half(areg[q])), mu = __half2float(__ushort_as_half(mreg[q]));
+                                store_from_float(P.y, P.y_dt, (size_t)m * P.N + n, al * (2.0f * dot1 - sx) + mu * sx);
+                            }
+                        }
+                    }
+                }
+                if (c1 < ghi) im_named_bar(1, IM_CWARPS * 32);
+            }
+            } else {
+            const int g = lane >> 2, t = lane & 3;
+            constexpr float MAGIC = 12582912.0f;                   // 1.5 * 2^23: float -> int by addition
+            constexpr int MAGIC_BITS = 0x4B400000;
+            const int ks = warp;                                   // K-slice of this warp
+            // MMA row g (and g + 8) carries tile row sg (and sg + 8): neighbouring g differ in bit 2 of the row, so the
+            // eight lanes of a shared-memory phase read distinct swizzled chunks
+            const int sg = ((g & 1) << 2) | (g >> 1);
+            // digit planes of a slice: block b, class c of digit d at word d * PSW + (b + b / BPL) * NCLS + c; the skew
+            // puts the lanes of a fragment read (t: blocks BPL apart, d: planes) on different banks
+            constexpr int PSW = (SLICE + 4) * NCLS;
+            uint32_t *planes = s_planes + ks * (3 * (SLICE + 4) * 5);
+            const int M = P.M, K = P.K, Kb = P.Kb, v = P.v;
+            const int cmax = P.ncls - 1;
+            const int PBITS = 22 - cmax;                           // |X| <= 2^PBITS
+            const int ngroups = SLICE * v / 8;                     // groups of 8 activations in a slice (<= 80)
+            const float unshift2 = 2.0f / (float)(1 << cmax);
+            const uint32_t *gtab = P.tab;
+            const int xsz = (P.x_dt == BTC_F32) ? 4 : 2;
+            bool tab_ready = !tab_smem;
+            bool ok = true;
+            int li = 0, s = 0;
+            uint32_t rph = 0;
+            // byte offset of this lane's index chunk inside a stage (128-byte swizzle: 16-byte chunk c of row q sits
+            // at chunk c ^ (q & 7)); rows sg and sg + 8
+            const int boff = (ks * SLICE + BPL * t) * 2;
+            const uint32_t idx_off = (uint32_t)(boff >> 7) * IM_BOX_BYTES + (uint32_t)sg * 128
+                                     + ((((boff >> 4) & 7) ^ (sg & 7)) << 4) + (boff & 15);
+            const int ct = tid;                                    // 0 .. 255: position among the compute threads
+
+            for (int c0 = glo; c0 < ghi; c0 += RC) {
+                const int c1 = min(c0 + RC, ghi);
+                const int nrows = (c1 - c0) * 16;
+                const int nout = nrows * M;                        // outputs of this chunk: (m, tile row) pairs
+                // alpha / mu of the outputs this thread will finish (static data: the loads are issued ahead of the
+                // dependency wait and of the chunk's work, and land while it runs)
+                constexpr int OPT = (RC * 16 * MAXM + IM_CWARPS * 32 - 1) / (IM_CWARPS * 32);   // outputs per thread
+                unsigned short areg[OPT], mreg[OPT];
+#pragma unroll
+                for (int q = 0; q < OPT; ++q) {
+                    const int o = ct + q * (IM_CWARPS * 32);
+                    areg[q] = 0; mreg[q] = 0;
+                    if (o < nout) {
+                        const int n = c0 * 16 + (o % nrows);
+                        if (n < P.N) {
+                            areg[q] = __ldg(reinterpret_cast<const unsigned short *>(P.alpha) + n);
+                            if (P.mu) mreg[q] = __ldg(reinterpret_cast<const unsigned short *>(P.mu) + n);
+                        }
+                    }
+                }
+                if (c0 == glo) asm volatile("griddepcontrol.wait;" ::: "memory");
+                float sxw[MAXM];                                   // this warp's share of sum_k x[m, k] (lane 0)
+#pragma unroll
+                for (int m = 0; m < MAXM; ++m) sxw[m] = 0.f;
+
+                for (int j = 0; j < P.parts; ++j) {
+                    const int pw = min(PW, Kb - j * PW);
+                    const int jb0 = j * PW + ks * SLICE;            // first block of this warp's slice
+                    const bool wvalid = ks * SLICE + BPL * t < pw;  // this lane's blocks exist (pw % 8 == 0)
+                    const int kend = (j * PW + pw) * v;             // end of the part in x
+
+                    // ---- B fragments for this part.  The warp's slice of each row of x is quantised with its own
+                    //      scale: X = rint(x * 2^(PBITS - e)), 2^e > max |x| of the slice.
+                    // (kept as 64-bit values: the two registers of an MMA's B operand then always sit in an aligned pair)
+                    constexpr int NPAIR = (NCLS + 1) / 2;
+                    uint64_t breg[BPL][NPAIR][NM];
+                    float invs[MAXM];
+#pragma unroll
+                    for (int e = 0; e < BPL; ++e)
+#pragma unroll
+                        for (int c = 0; c < NPAIR; ++c)
+#pragma unroll
+                            for (int nm = 0; nm < NM; ++nm) breg[e][c][nm] = 0ull;
+#pragma unroll
+                    for (int m = 0; m < MAXM; ++m) invs[m] = 0.f;
+                    constexpr int NU = (SLICE * 20 / 8 + 31) / 32;  // groups of 8 activations per lane (v <= 20)
+                    const bool fast16 = (NM == 1 && NCLS == 4 && v == 16);   // lane = block of the slice: no index arithmetic
+                    // 16-bit activations of the fast path: row m + 1 is fetched while row m is quantised
+                    const bool pf16 = fast16 && P.x_dt != BTC_F32;
+                    const bool pin = ks * SLICE + lane < pw;
+                    const size_t pk0 = (size_t)(jb0 + lane) * 16;
+                    uint4 cur0 = make_uint4(0u, 0u, 0u, 0u), cur1 = cur0;
+                    if (pf16 && pin) {
+                        const uint4 *src = reinterpret_cast<const uint4 *>(reinterpret_cast<const uint16_t *>(P.x) + pk0);
+                        cur0 = __ldg(src);
+                        cur1 = __ldg(src + 1);
+                    }
+#pragma unroll 1
+                    for (int m = 0; m < M; ++m) {
+                        const unsigned char *xrow = reinterpret_cast<const unsigned char *>(P.x) + (size_t)m * K * xsz;
+                        float inv;
                         int xs = 0;
+                        uint4 nxt0 = make_uint4(0u, 0u, 0u, 0u), nxt1 = nxt0;
+                        if (pf16 && pin && m + 1 < M) {
+                            const uint4 *src = reinterpret_cast<const uint4 *>(reinterpret_cast<const uint16_t *>(P.x) + (size_t)(m + 1) * K + pk0);
+                            nxt0 = __ldg(src);
+                            nxt1 = __ldg(src + 1);
+                        }
+                        if (fast16) {
+                            float xf[16];
+                            const bool in = ks * SLICE + lane < pw;
 #pragma unroll
-                        for (int u = 0; u < NU; ++u) {
-                            const int gi = lane + 32 * (rh + TRK * u);
-                            if (gi < ngroups) {
-                                const uint32_t wds[4] = {q4[u].x, q4[u].y, q4[u].z, q4[u].w};
-                                int blk = (8 * gi) / v;                  // block of the group's first activation in the slice
-                                int cpos = 8 * gi - blk * v;             // and its position in that block
+                            for (int i = 0; i < 16; ++i) xf[i] = 0.f;
+                            if (pf16) {
+                                im_cvt8(cur0, P.x_dt, &xf[0]);
+                                im_cvt8(cur1, P.x_dt, &xf[8]);
+                            } else if (in) {
+                                im_load8(xrow, P.x_dt, (jb0 + lane) * 16, *reinterpret_cast<float (*)[8]>(&xf[0]));
+                                im_load8(xrow, P.x_dt, (jb0 + lane) * 16 + 8, *reinterpret_cast<float (*)[8]>(&xf[8]));
+                            }
+                            float amax = 0.f;
 #pragma unroll
-                                for (int h = 0; h < 2; ++h) {
-                                    const int c = cpos >> 2;
-                                    const int wi = (blk + blk / BPL) * NCLS + c;
-                                    cpos += 4;
-                                    if (cpos >= v) { cpos -= v; ++blk; }
-                                    const uint32_t sh = 1u << (cmax - c);
-                                    const uint32_t off = 0x8080u - (uint32_t)MAGIC_BITS * sh;    // arithmetic modulo 2^32
-                                    float f0, f1, f2, f3;
-                                    im_unpack2(wds[2 * h], P.x_dt, f0, f1);
-                                    im_unpack2(wds[2 * h + 1], P.x_dt, f2, f3);
-                                    const uint32_t b0 = (uint32_t)__float_as_int(f0 * sc + MAGIC), b1 = (uint32_t)__float_as_int(f1 * sc + MAGIC);
-                                    const uint32_t b2 = (uint32_t)__float_as_int(f2 * sc + MAGIC), b3 = (uint32_t)__float_as_int(f3 * sc + MAGIC);
-                                    xs += (int)(b0 + b1 + b2 + b3 - 4u * (uint32_t)MAGIC_BITS);
-                                    // Y = X * 2^(cmax - c) + 0x8080: byte d of Y is balanced digit d of X * 2^(cmax-c), + 0x80 for d < 2
-                                    const uint32_t y0 = b0 * sh + off, y1 = b1 * sh + off, y2 = b2 * sh + off, y3 = b3 * sh + off;
+                            for (int i = 0; i < 16; ++i) amax = fmaxf(amax, fabsf(xf[i]));
+                            float sc;
+                            im_slice_scale(amax, PBITS, sc, inv);
+                            uint32_t bq[16];
 #pragma unroll
-                                    for (int d = 0; d < 3; ++d) {
-                                        const uint32_t sel = (uint32_t)d | ((uint32_t)(4 + d) << 4);
-                                        const uint32_t lo2 = __byte_perm(y0, y1, sel), hi2 = __byte_perm(y2, y3, sel);
-                                        planes[d * PSW + wi] = __byte_perm(lo2, hi2, 0x5410) ^ (d < 2 ? 0x80808080u : 0u);
+                            for (int i = 0; i < 16; ++i) {
+                                bq[i] = (uint32_t)__float_as_int(xf[i] * sc + MAGIC);
+                                xs += (int)(bq[i] - (uint32_t)MAGIC_BITS);
+                            }
+                            uint32_t dg[3][4];                       // digit d of the four activations of class c, one byte each
+#pragma unroll
+                            for (int c = 0; c < 4; ++c) {
+                                const uint32_t sh = 1u << (3 - c);
+                                const uint32_t off = 0x8080u - (uint32_t)MAGIC_BITS * sh;        // arithmetic modulo 2^32
+                                // Y = X * 2^(cmax - c) + 0x8080: byte d of Y is balanced digit d of X * 2^(cmax-c), + 0x80 for d < 2
+                                const uint32_t y0 = bq[4 * c] * sh + off, y1 = bq[4 * c + 1] * sh + off;
+                                const uint32_t y2 = bq[4 * c + 2] * sh + off, y3 = bq[4 * c + 3] * sh + off;
+                                const uint32_t t0 = __byte_perm(y0, y1, 0x5140), t1 = __byte_perm(y2, y3, 0x5140);
+                                const uint32_t t2 = __byte_perm(y0, y1, 0x0062), t3 = __byte_perm(y2, y3, 0x0062);
+                                dg[0][c] = __byte_perm(t0, t1, 0x5410) ^ 0x80808080u;
+                                dg[1][c] = __byte_perm(t0, t1, 0x7632) ^ 0x80808080u;
+                                dg[2][c] = __byte_perm(t2, t3, 0x5410);
+                            }
+#pragma unroll
+                            for (int d = 0; d < 3; ++d)
+                                *reinterpret_cast<uint4 *>(planes + d * PSW + (lane + (lane >> 3)) * 4) =
+                                    make_uint4(dg[d][0], dg[d][1], dg[d][2], dg[d][3]);
+                        } else {
+                            float xf[NU][8];
+                            float amax = 0.f;
+#pragma unroll
+                            for (int u = 0; u < NU; ++u) {
+                                const int gi = lane + 32 * u;
+                                const int k0 = jb0 * v + 8 * gi;
+#pragma unroll
+                                for (int i = 0; i < 8; ++i) xf[u][i] = 0.f;
+                                if (gi < ngroups && k0 < kend) im_load8(xrow, P.x_dt, k0, xf[u]);
+#pragma unroll
+                                for (int i = 0; i < 8; ++i) amax = fmaxf(amax, fabsf(xf[u][i]));
+                            }
+                            float sc;
+                            im_slice_scale(amax, PBITS, sc, inv);
+#pragma unroll
+                            for (int u = 0; u < NU; ++u) {
+                                const int gi = lane + 32 * u;
+                                if (gi < ngroups) {
+                                    int blk = (8 * gi) / v;                  // block of the group's first activation in the slice
+                                    int cpos = 8 * gi - blk * v;             // and its position in that block
+#pragma unroll
+                                    for (int h = 0; h < 2; ++h) {
+                                        const int c = cpos >> 2;
+                                        const int wi = (blk + blk / BPL) * NCLS + c;
+                                        cpos += 4;
+                                        if (cpos >= v) { cpos -= v; ++blk; }
+                                        const uint32_t sh = 1u << (cmax - c);
+                                        const uint32_t off = 0x8080u - (uint32_t)MAGIC_BITS * sh;    // arithmetic modulo 2^32
+                                        const uint32_t b0 = (uint32_t)__float_as_int(xf[u][4 * h] * sc + MAGIC);
+                                        const uint32_t b1 = (uint32_t)__float_as_int(xf[u][4 * h + 1] * sc + MAGIC);
+                                        const uint32_t b2 = (uint32_t)__float_as_int(xf[u][4 * h + 2] * sc + MAGIC);
+                                        const uint32_t b3 = (uint32_t)__float_as_int(xf[u][4 * h + 3] * sc + MAGIC);
+                                        xs += (int)(b0 + b1 + b2 + b3 - 4u * (uint32_t)MAGIC_BITS);
+                                        // Y = X * 2^(cmax - c) + 0x8080: byte d of Y is balanced digit d of X * 2^(cmax-c), + 0x80 for d < 2
+                                        const uint32_t y0 = b0 * sh + off, y1 = b1 * sh + off, y2 = b2 * sh + off, y3 = b3 * sh + off;
+#pragma unroll
+                                        for (int d = 0; d < 3; ++d) {
+                                            const uint32_t sel = (uint32_t)d | ((uint32_t)(4 + d) << 4);
+                                            const uint32_t lo2 = __byte_perm(y0, y1, sel), hi2 = __byte_perm(y2, y3, sel);
+                                            planes[d * PSW + wi] = __byte_perm(lo2, hi2, 0x5410) ^ (d < 2 ? 0x80808080u : 0u);
+                                        }
                                     }
                                 }
                             }
                         }
 #pragma unroll
                         for (int o = 16; o > 0; o >>= 1) xs += __shfl_xor_sync(0xffffffffu, xs, o);
-                        if (lane == 0) {
-                            ImScale o2;
-                            o2.inv = inv;
-                            o2.sx = (float)xs * inv;                     // this warp's share of sum_k x over the slice
-                            scale_out[m] = o2;
-                        }
-                        slice_sync();
+#pragma unroll
+                        for (int mm = 0; mm < MAXM; ++mm)
+                            if (mm == m) { invs[mm] = inv; sxw[mm] += (float)xs * inv; }
+                        __syncwarp();
 #pragma unroll
                         for (int nm = 0; nm < NM; ++nm) {
                             const int col = g + 8 * nm;
-                            const int mc = col / 3, d = col - 3 * mc;
-                            if (mc == m && wvalid) {
+                            const int mc = col >> 2, d = col & 3;     // column 4 m + d
+                            if (mc == m && d < 3 && wvalid) {
                                 const uint32_t *src = planes + d * PSW + (BPL * t + t) * NCLS;
 #pragma unroll
                                 for (int e = 0; e < BPL; ++e) {
                                     if (NCLS == 4) {
                                         const uint4 q = *reinterpret_cast<const uint4 *>(src + e * 4);
-                                        breg[e][0][nm] = q.x; breg[e][1][nm] = q.y; breg[e][2][nm] = q.z; breg[e][NCLS - 1][nm] = q.w;
+                                        breg[e][0][nm] = (uint64_t)q.x | ((uint64_t)q.y << 32);
+                                        breg[e][NPAIR - 1][nm] = (uint64_t)q.z | ((uint64_t)q.w << 32);
                                     } else {
 #pragma unroll
-                                        for (int c = 0; c < NCLS; ++c) breg[e][c][nm] = src[e * NCLS + c];
+                                        for (int c = 0; c < NCLS / 2; ++c)
+                                            breg[e][c][nm] = (uint64_t)src[e * NCLS + 2 * c] | ((uint64_t)src[e * NCLS + 2 * c + 1] << 32);
+                                        // the odd class of two neighbouring blocks shares one MMA: block e even holds the pair
+                                        if ((NCLS & 1) && !(e & 1))
+                                            breg[e][NPAIR - 1][nm] = (uint64_t)src[e * NCLS + NCLS - 1] | ((uint64_t)src[(e + 1) * NCLS + NCLS - 1] << 32);
                                     }
                                 }
                             }
                         }
-                        slice_sync();
+                        __syncwarp();
+                        cur0 = nxt0; cur1 = nxt1;
                     }
                     if (!tab_ready) {
-                        if (!im_mbar_wait(bar_tabfull, ps & 1, s_abort)) { ok = false; break; }
+                        ok &= im_mbar_wait(bar_tabfull, 0, s_abort);
                         tab_ready = true;
                     }
 
-                    // ---- the row groups of the chunk, for this part
-                    // Loads this lane's indices of the next row group from the ring (tile rows sg and sg + 8 of tile rh;
-                    // 128-byte swizzle: 16-byte chunk c of row q sits at chunk c ^ (q & 7)) and frees the stage.
-                    uint32_t ia[BPL / 2], ib[BPL / 2];
-                    auto load_indices = [&]() -> bool {
-                        if (!im_mbar_wait(bar_full(s), rph, s_abort)) return false;
-                        const unsigned char *stage = s_ring + (size_t)s * IM_STAGE_BYTES;
-#pragma unroll
-                        for (int i = 0; i < BPL / 2; ++i) { ia[i] = 0u; ib[i] = 0u; }
-                        if (wvalid) {
-                            const unsigned char *pa = stage + idx_off;
+                    // ---- the tiles of the chunk, for this part.  A tile's codewords are fetched (index stage -> registers ->
+                    //      table lookups) while the previous tile's MMAs are still in flight.
+                    uint32_t w0[BPL], w1[BPL];                      // codewords of rows sg and sg + 8, this lane's blocks
+                    auto fetch = [&]() {
+                        uint32_t ia[BPL / 2], ib[BPL / 2];
+                        ok &= im_mbar_wait(bar_full(s), rph, s_abort);
+                        {
+                            // (every stage is filled whole: blocks past the part and rows past N arrive as zeros)
+                            const unsigned char *pa = s_ring + (size_t)s * STAGE_BYTES + idx_off;
                             const unsigned char *pb = pa + 8 * 128;                 // row + 8: same row & 7
                             if (BPL == 8) {
                                 const uint4 qa = *reinterpret_cast<const uint4 *>(pa), qb = *reinterpret_cast<const uint4 *>(pb);
@@ -608,120 +850,146 @@ gemv_imma_kernel(const __grid_constant__ ImBatch batch)
                                 ib[0] = qb.x; ib[1] = qb.y;
                             }
                         }
+                        if (!ok) {                                  // a wait gave up: the stage may hold anything
+#pragma unroll
+                            for (int i = 0; i < BPL / 2; ++i) { ia[i] = 0u; ib[i] = 0u; }
+                        }
+                        // the index loads must have returned before the stage is handed back (see the fp16 form)
+#pragma unroll
+                        for (int i = 0; i < BPL / 2; ++i) asm volatile("" :: "r"(ia[i]), "r"(ib[i]) : "memory");
                         __syncwarp();
                         if (lane == 0) im_mbar_arrive(bar_empty(s));
                         if (++s == NST) { s = 0; rph ^= 1u; }
-                        return true;
-                    };
-                    if (!load_indices()) { ok = false; break; }
-                    for (int r = c0; r < c1; ++r, ++li) {
-                        constexpr int CH = 2;        // accumulation chains: an MMA need not wait for the previous one
-                        int accs[CH][NM][4];
-                        int (&acc)[NM][4] = accs[0];
+                        if constexpr (TAB_MODE == 1) {
+                            // whole table in shared memory as 32-bit words: each pair of packed indices becomes two
+                            // shared addresses by one widening multiply-add per index (base + 4 * idx)
+                            const uint32_t tb = im_smem_u32(s_tab);
 #pragma unroll
-                        for (int nm = 0; nm < NM; ++nm)
+                            for (int i = 0; i < BPL / 2; ++i) {
+                                uint32_t a0, a1, b0, b1;
+                                im_pair_addr(ia[i], tb, a0, a1);
+                                im_pair_addr(ib[i], tb, b0, b1);
+                                w0[2 * i] = im_lds32(a0); w0[2 * i + 1] = im_lds32(a1);
+                                w1[2 * i] = im_lds32(b0); w1[2 * i + 1] = im_lds32(b1);
+                            }
+                        } else {
 #pragma unroll
-                            for (int i = 0; i < 4; ++i)
-#pragma unroll
-                                for (int ch = 0; ch < CH; ++ch) accs[ch][nm][i] = 0;
-                        if (ks * SLICE < pw) {                      // warp-uniform: the slice is not empty
-#pragma unroll
-                            for (int e4 = 0; e4 < BPL; e4 += 4) {
-                                uint32_t w0[4], w1[4];
-#pragma unroll
-                                for (int e = 0; e < 4; ++e) {
-                                    const uint32_t pa = ia[(e4 + e) >> 1], pb = ib[(e4 + e) >> 1];
-                                    const uint32_t i0 = (e & 1) ? (pa >> 16) : (pa & 0xffffu);
-                                    const uint32_t i1 = (e & 1) ? (pb >> 16) : (pb & 0xffffu);
-                                    if (TAB_MODE == 1) { w0[e] = s_tab[i0]; w1[e] = s_tab[i1]; }
-                                    else if (TAB_MODE == 3) {
-                                        const uint32_t h0 = reinterpret_cast<const uint16_t *>(s_tab)[i0];
-                                        const uint32_t h1 = reinterpret_cast<const uint16_t *>(s_tab)[i1];
-                                        w0[e] = h0 | (h0 << 12); w1[e] = h1 | (h1 << 12);
-                                    }
-                                    else if (TAB_MODE == 0) { w0[e] = __ldg(gtab + i0); w1[e] = __ldg(gtab + i1); }
-                                    else {
-                                        w0[e] = i0 < tab_head ? s_tab[i0] : __ldg(gtab + i0);
-                                        w1[e] = i1 < tab_head ? s_tab[i1] : __ldg(gtab + i1);
-                                    }
+                            for (int e = 0; e < BPL; ++e) {
+                                const uint32_t pa = ia[e >> 1], pb = ib[e >> 1];
+                                const uint32_t i0 = (e & 1) ? (pa >> 16) : (pa & 0xffffu);
+                                const uint32_t i1 = (e & 1) ? (pb >> 16) : (pb & 0xffffu);
+                                if (TAB_MODE == 3) {
+                                    const uint32_t h0 = reinterpret_cast<const uint16_t *>(s_tab)[i0];
+                                    const uint32_t h1 = reinterpret_cast<const uint16_t *>(s_tab)[i1];
+                                    w0[e] = h0 | (h0 << 12); w1[e] = h1 | (h1 << 12);
                                 }
-#pragma unroll
-                                for (int e = 0; e < 4; ++e) {
-#pragma unroll
-                                    for (int cp = 0; cp < NCLS / 2; ++cp) {
-                                        const uint32_t ma = 0x01010101u << (2 * cp), mb = 0x01010101u << (2 * cp + 1);
-#pragma unroll
-                                        for (int nm = 0; nm < NM; ++nm)
-                                            im_mma_u8s8(accs[((e & 1) * 2 + (cp & 1)) % CH][nm], w0[e] & ma, w1[e] & ma, w0[e] & mb, w1[e] & mb,
-                                                        breg[e4 + e][2 * cp][nm], breg[e4 + e][2 * cp + 1][nm]);
-                                    }
-                                }
-                                if (NCLS & 1) {
-                                    const uint32_t ml = 0x01010101u << (NCLS - 1);
-#pragma unroll
-                                    for (int ep = 0; ep < 2; ++ep)
-#pragma unroll
-                                        for (int nm = 0; nm < NM; ++nm)
-                                            im_mma_u8s8(acc[nm], w0[2 * ep] & ml, w1[2 * ep] & ml, w0[2 * ep + 1] & ml,
-                                                        w1[2 * ep + 1] & ml, breg[e4 + 2 * ep][NCLS - 1][nm], breg[e4 + 2 * ep + 1][NCLS - 1][nm]);
+                                else if (TAB_MODE == 0) { w0[e] = __ldg(gtab + i0); w1[e] = __ldg(gtab + i1); }
+                                else {
+                                    w0[e] = i0 < tab_head ? s_tab[i0] : __ldg(gtab + i0);
+                                    w1[e] = i1 < tab_head ? s_tab[i1] : __ldg(gtab + i1);
                                 }
                             }
                         }
-                        // the next row group's indices are fetched while this one's MMAs drain (their codewords are in
-                        // registers by now), so the barrier round trip is off the critical path
-                        if (r + 1 < c1 && !load_indices()) { ok = false; break; }
-                        // likewise the wait for the partial-sum buffer: its round trip overlaps the MMAs' drain
-                        const int buf = li & 1;
-                        if (li >= 2 && !im_mbar_wait(bar_pempty(buf), ((li >> 1) & 1) ^ 1, s_abort)) { ok = false; break; }
+                    };
+                    fetch();
+                    for (int r = c0; r < c1; ++r, ++li) {
+                        constexpr int CH = 2;        // accumulation chains: an MMA need not wait for the previous one
+                        int accs[CH][NM][4];
+#pragma unroll
+                        for (int ch = 0; ch < CH; ++ch)
+#pragma unroll
+                            for (int nm = 0; nm < NM; ++nm)
+#pragma unroll
+                                for (int i = 0; i < 4; ++i) accs[ch][nm][i] = 0;
+                        int (&acc)[NM][4] = accs[0];
+                        if (ks * SLICE < pw) {                      // warp-uniform: the slice is not empty
+#pragma unroll
+                            for (int e = 0; e < BPL; ++e) {
+#pragma unroll
+                                for (int cp = 0; cp < NCLS / 2; ++cp) {
+                                    const uint32_t ma = 0x01010101u << (2 * cp), mb = 0x01010101u << (2 * cp + 1);
+#pragma unroll
+                                    for (int nm = 0; nm < NM; ++nm)
+                                        im_mma_u8s8(accs[((e & 1) * 2 + (cp & 1)) % CH][nm], w0[e] & ma, w1[e] & ma, w0[e] & mb, w1[e] & mb,
+                                                    breg[e][cp][nm]);
+                                }
+                            }
+                            if (NCLS & 1) {
+                                const uint32_t ml = 0x01010101u << (NCLS - 1);
+#pragma unroll
+                                for (int ep = 0; ep < BPL / 2; ++ep)
+#pragma unroll
+                                    for (int nm = 0; nm < NM; ++nm)
+                                        im_mma_u8s8(accs[ep % CH][nm], w0[2 * ep] & ml, w1[2 * ep] & ml, w0[2 * ep + 1] & ml,
+                                                    w1[2 * ep + 1] & ml, breg[2 * ep][NPAIR - 1][nm]);
+                            }
+                        }
+                        if (r + 1 < c1) fetch();
 #pragma unroll
                         for (int nm = 0; nm < NM; ++nm)
 #pragma unroll
                             for (int i = 0; i < 4; ++i)
 #pragma unroll
                                 for (int ch = 1; ch < CH; ++ch) acc[nm][i] += accs[ch][nm][i];
-                        if constexpr (FPART) {
-                            // The three digit sums of (row, m) sit in columns 3 m .. 3 m + 2, spread over the lanes of a quad:
-                            // they are brought together by shuffles, recombined (each is below 2^24 in magnitude, so the
-                            // conversions are exact), scaled by the slice's 2^-s and stored as one float per (row, m).
-                            float *mine = s_part + (((size_t)buf * TRK + rh) * 16) * MAXM * KS + ks;
-#pragma unroll
-                            for (int m = 0; m < MAXM; ++m) {
-                                if (m < M) {                                // warp-uniform
-                                    int dlo[3], dhi[3];
-#pragma unroll
-                                    for (int d = 0; d < 3; ++d) {
-                                        const int col = 3 * m + d;          // a constant once unrolled
-                                        const int src = (lane & ~3) | ((col & 7) >> 1);
-                                        dlo[d] = __shfl_sync(0xffffffffu, acc[col >> 3][col & 1], src);
-                                        dhi[d] = __shfl_sync(0xffffffffu, acc[col >> 3][2 + (col & 1)], src);
-                                    }
-                                    if (t == (m & 3)) {
-                                        const float inv = scale_out[m].inv;
-                                        const float Tlo = ((float)dlo[2] * 256.0f + (float)dlo[1]) * 256.0f + (float)dlo[0];
-                                        const float Thi = ((float)dhi[2] * 256.0f + (float)dhi[1]) * 256.0f + (float)dhi[0];
-                                        mine[(sg * MAXM + m) * KS] = Tlo * inv;
-                                        mine[((sg + 8) * MAXM + m) * KS] = Thi * inv;
-                                    }
-                                }
-                            }
-                        } else {
-                            int *mine = s_parti + ((size_t)buf * IM_CWARPS + warp) * TILE_INTS;
-                            if (2 * t < 3 * M) {                        // columns 3 m + d, m < M: the others are never read
-                                *reinterpret_cast<int2 *>(mine + sg * COLS + 2 * t) = make_int2(acc[0][0], acc[0][1]);
-                                *reinterpret_cast<int2 *>(mine + (sg + 8) * COLS + 2 * t) = make_int2(acc[0][2], acc[0][3]);
+                        // The three digit sums of a (row, m) are recombined (each is below 2^24 in magnitude, so the
+                        // conversions are exact), scaled by the slice's 2^-s and parked as one float per (row, m, slice);
+                        // later parts add to what the same thread left there.
+                        float *mine = s_part + ((size_t)(r - c0) * 16 * MAXM) * IM_CWARPS + ks;
+                        {
+                            // columns 4 m + d: lane t = 2 m holds digits 0 and 1, lane 2 m + 1 holds digit 2 (and an empty column)
+                            const float wa = (t & 1) ? 65536.0f : 1.0f, wb = (t & 1) ? 0.0f : 256.0f;
+                            float plo = fmaf((float)acc[0][1], wb, (float)acc[0][0] * wa);
+                            float phi = fmaf((float)acc[0][3], wb, (float)acc[0][2] * wa);
+                            plo += __shfl_xor_sync(0xffffffffu, plo, 1);
+                            phi += __shfl_xor_sync(0xffffffffu, phi, 1);
+                            const int m = t >> 1;
+                            if (!(t & 1) && m < M) {
+                                const float iv = m ? invs[MAXM > 1 ? 1 : 0] : invs[0];
+                                float *qlo = mine + (sg * MAXM + m) * IM_CWARPS, *qhi = mine + ((sg + 8) * MAXM + m) * IM_CWARPS;
+                                if (j == 0) { *qlo = plo * iv; *qhi = phi * iv; }
+                                else { *qlo += plo * iv; *qhi += phi * iv; }
                             }
                         }
-                        __syncwarp();
-                        if (lane == 0) im_mbar_arrive(bar_pfull(buf));
                     }
                 }
+                if (lane == 0) {
+#pragma unroll
+                    for (int m = 0; m < MAXM; ++m) s_sx[ks * 8 + m] = sxw[m];
+                }
+                // ---- the eight slices meet: add them in a fixed order, apply alpha (and mu), store
+                im_named_bar(1, IM_CWARPS * 32);
+                if (ok && !*s_abort) {
+#pragma unroll
+                    for (int q = 0; q < OPT; ++q) {
+                        const int o = ct + q * (IM_CWARPS * 32);
+                        if (o < nout) {
+                            const int m = o / nrows, rl = o - m * nrows;
+                            const int n = c0 * 16 + rl;
+                            const float4 p0 = *reinterpret_cast<const float4 *>(s_part + ((size_t)rl * MAXM + m) * IM_CWARPS);
+                            const float4 p1 = *reinterpret_cast<const float4 *>(s_part + ((size_t)rl * MAXM + m) * IM_CWARPS + 4);
+                            const float dot1 = ((((((p0.x + p0.y) + p0.z) + p0.w) + p1.x) + p1.y) + p1.z) + p1.w;
+                            float sx = 0.f;
+#pragma unroll
+                            for (int w = 0; w < IM_CWARPS; ++w) sx += s_sx[w * 8 + m];
+                            if (n < P.N) {
+                                const float al = __half2float(__ushort_as_half(areg[q])), mu = __half2float(__ushort_as_half(mreg[q]));
+                                const float dot = dot1 * unshift2 - sx;         // 2 * sum_{bit=1} x - sum x
+                                store_from_float(P.y, P.y_dt, (size_t)m * P.N + n, al * dot + mu * sx);
+                            }
+                        }
+                    }
+                }
+                if (c1 < ghi) im_named_bar(1, IM_CWARPS * 32);      // the next chunk overwrites what was just read
             }
-            ++ps;
-            if (tab_smem && ok) {
-                __syncwarp();
-                if (lane == 0) im_mbar_arrive(bar_tabfree);
             }
         }
+    } else {
+        // (a CTA without work: the launch never creates one, but the dependency contract holds anyway)
+    }
+    // A CTA that gave up on a wait may still have copies in flight into its shared memory: let them land before it goes.
+    if (*s_abort) {
+        const long long t0 = clock64();
+        while (clock64() - t0 < 400000LL) __nanosleep(1000);
     }
     __syncthreads();
 }
@@ -744,20 +1012,20 @@ static im_encode_fn im_get_encode()
     return fn;
 }
 
-// Tensor map of an index matrix {K/v, N} (16-bit words), box {64, rows}, 128-byte swizzle.  Encoding goes through the
+// Tensor map of an index matrix {K/v, N} (16-bit words), box {64, 16}, 128-byte swizzle.  Encoding goes through the
 // driver and costs about a microsecond; a decode step re-uses the same matrices call after call, so the last few
 // maps are kept per host thread, keyed by everything the encoding depends on.
-static bool im_tensor_map(im_encode_fn enc, const uint16_t *idx, int Kb, int N, int rows, CUtensorMap *out)
+static bool im_tensor_map(im_encode_fn enc, const uint16_t *idx, int Kb, int N, CUtensorMap *out)
 {
-    struct Entry { const uint16_t *idx; int Kb, N, rows; CUtensorMap map; };
+    struct Entry { const uint16_t *idx; int Kb, N; CUtensorMap map; };
     constexpr int SLOTS = 64;
     thread_local Entry cache[SLOTS];
     thread_local int used = 0, next = 0;
     for (int i = 0; i < used; ++i)
-        if (cache[i].idx == idx && cache[i].Kb == Kb && cache[i].N == N && cache[i].rows == rows) { *out = cache[i].map; return true; }
+        if (cache[i].idx == idx && cache[i].Kb == Kb && cache[i].N == N) { *out = cache[i].map; return true; }
     const cuuint64_t dims[2] = {(cuuint64_t)Kb, (cuuint64_t)N};
     const cuuint64_t strides[1] = {(cuuint64_t)Kb * 2};
-    const cuuint32_t box[2] = {(cuuint32_t)IM_BOX_COLS, (cuuint32_t)rows};
+    const cuuint32_t box[2] = {(cuuint32_t)IM_BOX_COLS, 16u};
     const cuuint32_t estr[2] = {1, 1};
     CUtensorMap m;
     if (enc(&m, CU_TENSOR_MAP_DATA_TYPE_UINT16, 2, const_cast<uint16_t *>(idx), dims, strides, box, estr,
@@ -765,7 +1033,7 @@ static bool im_tensor_map(im_encode_fn enc, const uint16_t *idx, int Kb, int N, 
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
         return false;
     Entry &e = cache[next];
-    e.idx = idx; e.Kb = Kb; e.N = N; e.rows = rows; e.map = m;
+    e.idx = idx; e.Kb = Kb; e.N = N; e.map = m;
     next = (next + 1) % SLOTS;
     if (used < SLOTS) ++used;
     *out = m;
@@ -783,15 +1051,17 @@ static int im_sm_count()
     return n;
 }
 
-// Gives every layer a whole number of CTAs so that the largest load of any CTA -- ceil(groups / CTAs) row groups times
-// the layer's cost per row group; row groups are not divisible -- is as small as the budget allows, and returns the
-// grid size.  Smallest feasible load by bisection; a load T needs ceil(groups / floor(T / cost)) CTAs of a layer.
+// Gives every layer a whole number of CTAs so that the largest load of any CTA -- ceil(tiles / CTAs) tiles times
+// the layer's cost per tile, plus the layer's set-up cost; tiles are not divisible -- is as small as the budget
+// allows, and returns the grid size.  Smallest feasible load by bisection; a load T needs
+// ceil(tiles / floor((T - fixed) / cost)) CTAs of a layer.
 static int im_assign_ctas(ImBatch &b, int budget)
 {
+    auto tiles_per_cta = [&](int i, long long T) { return (T - b.p[i].fixed) / b.p[i].cost; };
     auto ctas_needed = [&](long long T) {
         long long sum = 0;
         for (int i = 0; i < b.count; ++i) {
-            const long long per = T / b.p[i].cost;                    // row groups one CTA may take
+            const long long per = tiles_per_cta(i, T);                // tiles one CTA may take
             if (per < 1) return (long long)1 << 40;
             sum += (b.p[i].groups + per - 1) / per;
         }
@@ -799,7 +1069,7 @@ static int im_assign_ctas(ImBatch &b, int budget)
     };
     long long lo = 1, hi = 0;
     for (int i = 0; i < b.count; ++i) {
-        const long long all = (long long)b.p[i].groups * b.p[i].cost;
+        const long long all = (long long)b.p[i].groups * b.p[i].cost + b.p[i].fixed;
         if (all > hi) hi = all;                                       // one CTA per layer always fits (budget >= count)
     }
     while (lo < hi) {
@@ -808,7 +1078,7 @@ static int im_assign_ctas(ImBatch &b, int budget)
     }
     int sum = 0;
     for (int i = 0; i < b.count; ++i) {
-        const long long per = lo / b.p[i].cost;
+        const long long per = tiles_per_cta(i, lo);
         b.p[i].cta_count = (int)((b.p[i].groups + per - 1) / per);
         sum += b.p[i].cta_count;
     }
@@ -816,8 +1086,8 @@ static int im_assign_ctas(ImBatch &b, int budget)
         int best = -1;
         for (int i = 0; i < b.count; ++i)
             if (b.p[i].cta_count < b.p[i].groups &&
-                (best < 0 || (double)b.p[i].groups * b.p[i].cost / b.p[i].cta_count >
-                                 (double)b.p[best].groups * b.p[best].cost / b.p[best].cta_count)) best = i;
+                (best < 0 || (double)b.p[i].groups * b.p[i].cost / b.p[i].cta_count + b.p[i].fixed >
+                                 (double)b.p[best].groups * b.p[best].cost / b.p[best].cta_count + b.p[best].fixed)) best = i;
         if (best < 0) break;
         ++b.p[best].cta_count; ++sum;
     }
@@ -834,14 +1104,15 @@ static int im_assign_ctas(ImBatch &b, int budget)
 template <int NCLS, int NM, int TS>
 static int im_launch(ImBatch &b, int groups_total, cudaStream_t s)
 {
-    constexpr int TRK = (NM == 1) ? 2 : 1;
-    const ImSmem L = im_smem_layout(b.tab_smem_bytes, 8 * NM, TRK * 16, b.stages);
+    const ImSmem L = im_smem_layout(b.tab_smem_bytes, NM, b.stages);
     auto kern = gemv_imma_kernel<NCLS, NM, TS>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)L.total);
     if (e != cudaSuccess) return cuda_fail(e);
     cudaLaunchConfig_t cfg = {};
-    const int sms = im_sm_count();
-    const int grid = im_assign_ctas(b, groups_total < sms ? groups_total : sms);
+    // CTAs that can be resident at once: two per SM when the shared memory asked for allows it
+    const int per_sm = (2u * (L.total + 1024u) <= 228u * 1024u) ? 2 : 1;
+    const int slots = im_sm_count() * per_sm;
+    const int grid = im_assign_ctas(b, groups_total < slots ? groups_total : slots);
     cfg.gridDim = dim3((unsigned)grid);
     cfg.blockDim = dim3(IM_THREADS);
     cfg.dynamicSmemBytes = L.total;
@@ -859,8 +1130,8 @@ template <int NCLS, int TS>
 static int im_launch_nm(ImBatch &b, int nm, int groups_total, cudaStream_t s)
 {
     if (nm == 1) return im_launch<NCLS, 1, TS>(b, groups_total, s);
-    if (nm == 2) return im_launch<NCLS, 2, TS>(b, groups_total, s);
-    return im_launch<NCLS, 3, TS>(b, groups_total, s);
+    if (TS == 3) return BTC_ERR_UNSUPPORTED;                // (the 16-bit table exists for the byte-lane words only)
+    return im_launch<NCLS, 0, TS == 3 ? 1 : TS>(b, groups_total, s);
 }
 
 int launch_gemv_imma(const LinearArgs *problems, int count, cudaStream_t s)
@@ -875,55 +1146,66 @@ int launch_gemv_imma(const LinearArgs *problems, int count, cudaStream_t s)
         const LinearArgs &a = problems[i];
         // covered: M <= 8, v a multiple of 4 up to 20, K/v a multiple of 8 (16-byte rows for the bulk copies)
         if (a.M < 1 || a.M > 8 || a.v % 4 != 0 || a.v > 20 || a.Kb % 8 != 0 || a.K > (1 << 20)) return BTC_ERR_UNSUPPORTED;
+        if (a.x_dt == BTC_F32 && a.K % 8 != 0) return BTC_ERR_UNSUPPORTED;
         if (a.M > m_max) m_max = a.M;
     }
-    const int nm = m_max <= 2 ? 1 : (m_max <= 5 ? 2 : 3);
-    const int rows = (nm == 1) ? 32 : 16;
+    const int nm = m_max <= 2 ? 1 : 0;                      // integer form up to two rows of x, fp16 form above
+    const int pw = nm == 1 ? 256 : 128;
+    // the ring is no longer than the longest walk of any CTA needs; the split below assumes the full ring
     int groups_total = 0;
     for (int i = 0; i < count; ++i) {
         const LinearArgs &a = problems[i];
         ImProblem &p = b.p[i];
         p.x = a.x; p.idx = a.idx; p.alpha = a.alpha; p.mu = a.mu; p.y = a.y;
         const int Kc4 = (a.Kc + 3) / 4 * 4;
-        p.tab = a.Cp + 2 * Kc4;                      // byte-lane words follow the two other forms
+        p.tab = a.Cp + (nm == 0 ? 1 : 2) * Kc4;      // fp16-layout words (fp16 form) or byte-lane words (integer form)
         p.tab16 = reinterpret_cast<const uint16_t *>(a.Cp + 3 * (size_t)Kc4);
         p.M = a.M; p.N = a.N; p.K = a.K; p.v = a.v; p.Kc = a.Kc; p.Kb = a.Kb;
         p.x_dt = a.x_dt; p.y_dt = a.y_dt;
-        p.parts = (a.Kb + IM_PW - 1) / IM_PW;
-        p.groups = (a.N + rows - 1) / rows;
+        p.parts = (a.Kb + pw - 1) / pw;
+        p.groups = (a.N + 15) / 16;
         p.ncls = a.v / 4;
-        if (!im_tensor_map(enc, a.idx, a.Kb, a.N, rows, &b.map[i]))
+        if (!im_tensor_map(enc, a.idx, a.Kb, a.N, &b.map[i]))
             return BTC_ERR_UNSUPPORTED;                     // shape the tensor map cannot describe: other kernels take it
-        // measured: an iteration (one row group x one part of up to 256 blocks) costs about the same whatever the
-        // part's width, and rebuilding the activation fragments for a part costs ~1.5 iterations, shared by the
-        // (few) row groups a CTA walks with it; a single-part layer rebuilds only once per CTA
-        p.cost = p.parts > 1 ? p.parts * (IM_PW + 110) : a.Kb + 40;
+        // a (tile, part) costs about the same whatever the part's width; rebuilding the activation fragments for a
+        // part costs about as much as one and a half of them and is shared by the tiles a CTA walks with that part
+        p.cost = p.parts * 16;                               // per tile, in sixteenths of a (tile, part)
+        p.fixed = p.parts * 24 * (nm == 0 ? 1 : a.M);        // per CTA (the fp16 form builds all rows of x at once)
         groups_total += p.groups;
         if (p.ncls > ncls_max) ncls_max = p.ncls;
         if (Kc4 * 4 > tab_max) tab_max = Kc4 * 4;
         if ((a.Kc + 7) / 8 * 16 > tab16_max) tab16_max = (a.Kc + 7) / 8 * 16;
         if (a.v > v_max) v_max = a.v;
     }
-    // the whole table in shared memory when it fits beside at least four index stages; else, for v <= 16, as 16-bit
-    // halves beside at least two; else as much of its head as fits
+    // Two CTAs per SM is the aim: 113 KB each.  The table goes to shared memory as 32-bit words when that leaves room
+    // for at least six index stages, else (v <= 16) as 16-bit halves, else as much of its head as fits one CTA per SM.
+    const uint32_t half_sm = 113u * 1024u, whole_sm = 227u * 1024u;
     int mode = 1;
     b.tab_smem_bytes = tab_max;
     b.tab_head = tab_max / 4;
-    if (im_smem_layout(tab_max, 8 * nm, rows, 4).total > 227u * 1024u) {
-        if (v_max <= 16 && im_smem_layout(tab16_max, 8 * nm, rows, 2).total <= 227u * 1024u) {
+    uint32_t budget = half_sm;
+    if (im_smem_layout(tab_max, nm, 6).total > half_sm) {
+        if (nm == 1 && v_max <= 16 && im_smem_layout(tab16_max, nm, 4).total <= half_sm) {
             mode = 3;
             b.tab_smem_bytes = tab16_max;
+        } else if (nm == 1 && v_max <= 16 && im_smem_layout(tab16_max, nm, 2).total <= whole_sm) {
+            mode = 3;
+            b.tab_smem_bytes = tab16_max;
+            budget = whole_sm;
+        } else if (im_smem_layout(tab_max, nm, 4).total <= whole_sm) {
+            budget = whole_sm;
         } else {
             mode = 2;
+            budget = whole_sm;
             int head_bytes = tab_max;
-            while (head_bytes > 0 && im_smem_layout(head_bytes, 8 * nm, rows, 4).total > 227u * 1024u) head_bytes -= 4096;
+            while (head_bytes > 0 && im_smem_layout(head_bytes, nm, 4).total > whole_sm) head_bytes -= 4096;
             if (head_bytes <= 0) { mode = 0; head_bytes = 0; }
             b.tab_smem_bytes = head_bytes;
             b.tab_head = head_bytes / 4;
         }
     }
     b.stages = IM_STAGES;
-    while (b.stages > 2 && im_smem_layout(b.tab_smem_bytes, 8 * nm, rows, b.stages).total > 227u * 1024u) --b.stages;
+    while (b.stages > 2 && im_smem_layout(b.tab_smem_bytes, nm, b.stages).total > budget) --b.stages;
     if (ncls_max <= 4) {
         if (mode == 1) return im_launch_nm<4, 1>(b, nm, groups_total, s);
         if (mode == 3) return im_launch_nm<4, 3>(b, nm, groups_total, s);

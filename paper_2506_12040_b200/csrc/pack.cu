@@ -1,4 +1,5 @@
 // Codebook packing, sign-matrix decode and index validation kernels (offline / checking helpers).
+#include <cstdlib>
 #include "btc_internal.cuh"
 
 namespace btc {
@@ -77,6 +78,55 @@ __global__ void validate_indices_kernel(const uint16_t *__restrict__ idx, size_t
     for (; i < count; i += stride) local += (idx[i] >= Kc) ? 1 : 0;
     for (int o = 16; o > 0; o >>= 1) local += __shfl_xor_sync(0xffffffffu, local, o);
     if ((threadIdx.x & 31) == 0 && local) atomicAdd(bad, local);
+}
+
+// Debug aid (switched on by the environment variable BTC_DEBUG_CHECK_INDICES=1): raises a status word when an index is
+// >= Kc.  No trap, no assert: the layer kernels still run (their result is then undefined), the context stays usable and
+// btc_device_status reports BTC_ERR_INDEX.
+__device__ int g_index_status = 0;
+
+__global__ void flag_bad_indices_kernel(const uint16_t *__restrict__ idx, size_t count, int Kc)
+{
+    size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const size_t stride = (size_t)gridDim.x * blockDim.x;
+    bool bad = false;
+    for (; i < count; i += stride) bad |= idx[i] >= Kc;
+    if (__any_sync(0xffffffffu, bad) && (threadIdx.x & 31) == 0) atomicExch(&g_index_status, (int)BTC_ERR_INDEX);
+}
+
+bool debug_check_indices_enabled()
+{
+    static int on = -1;
+    if (on < 0) {
+        const char *e = getenv("BTC_DEBUG_CHECK_INDICES");
+        on = (e && e[0] && e[0] != '0') ? 1 : 0;
+    }
+    return on == 1;
+}
+
+int launch_index_check(const uint16_t *idx, size_t count, int Kc, cudaStream_t s)
+{
+    if (Kc >= 65536 || count == 0) return BTC_OK;             // every 16-bit value is a valid index
+    size_t grid = (count + 255) / 256;
+    if (grid > 148 * 8) grid = 148 * 8;
+    flag_bad_indices_kernel<<<(unsigned)grid, 256, 0, s>>>(idx, count, Kc);
+    return cuda_check_launch();
+}
+
+int index_status_read(int *out)
+{
+    int v = 0;
+    cudaError_t e = cudaMemcpyFromSymbol(&v, g_index_status, sizeof(int));
+    if (e != cudaSuccess) return cuda_fail(e);
+    *out = v;
+    return BTC_OK;
+}
+
+int index_status_reset()
+{
+    const int zero = 0;
+    cudaError_t e = cudaMemcpyToSymbol(g_index_status, &zero, sizeof(int));
+    return e == cudaSuccess ? BTC_OK : cuda_fail(e);
 }
 
 }  // namespace btc

@@ -425,3 +425,35 @@ def test_bounded_wait_gives_up_and_context_stays_usable():
     y, _ = run_layer(L, "gemv")
     rel, fwd = errors(y, oracle_y(L), L)
     assert rel <= TOL_GEMV and fwd <= TOL_GEMV and btc.device_status() == 0
+
+
+def test_debug_index_check_raises_status_word_only():
+    """BTC_DEBUG_CHECK_INDICES=1 (read when the library first needs it, hence a fresh process): every linear call first
+    runs a range check of idx on the same stream; an index >= Kc raises the status word (BTC_ERR_INDEX = 8), nothing
+    traps, and after a reset the library works as before.  The planted index (Kc + 4 of a 4096-entry table that sits in
+    shared memory in front of the index stages) keeps the layer kernel's own lookup inside its shared memory."""
+    import os
+    import subprocess
+    import sys
+    code = r'''
+import numpy as np, torch, sys
+sys.path.insert(0, "tests")
+import paper_2506_12040_b200 as btc, workloads as wl
+from util import to_device
+L = wl.make_layer(wl.LayerSpec("t", 64, 256, 16, 4096), 1, seed=1)
+d = to_device(L)
+assert btc.device_status() == 0
+btc.linear_gemv(d["x"], d["idx"], d["Cp"], d["alpha"], 16, 4096); torch.cuda.synchronize()
+assert btc.device_status() == 0
+bad = d["idx"].clone(); bad[3, 2] = 4100
+btc.linear_gemv(d["x"], bad, d["Cp"], d["alpha"], 16, 4096); torch.cuda.synchronize()
+assert btc.device_status() == 8, btc.device_status()
+btc.device_status_reset()
+y = btc.linear_gemv(d["x"], d["idx"], d["Cp"], d["alpha"], 16, 4096); torch.cuda.synchronize()
+assert btc.device_status() == 0 and bool(torch.isfinite(y).all())
+print("index check ok")
+'''
+    env = dict(os.environ, BTC_DEBUG_CHECK_INDICES="1")
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    r = subprocess.run([sys.executable, "-c", code], cwd=root, env=env, capture_output=True, text=True, timeout=600)
+    assert r.returncode == 0 and "index check ok" in r.stdout, r.stdout + r.stderr
