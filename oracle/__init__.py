@@ -140,6 +140,38 @@ def pack_codebook(C_pm1) -> np.ndarray:
     return out
 
 
+def index_bits(Kc: int) -> int:
+    """ceil(log2 Kc), at least 1: the index width of the paper's storage accounting (Section 4.3)."""
+    b = 1
+    while (1 << b) < Kc:
+        b += 1
+    return b
+
+
+def packed_row_bytes(Kb: int, bits: int, align: int = 16) -> int:
+    """Bytes from one packed row to the next: ceil(Kb*bits/8) rounded up to `align`."""
+    n = (Kb * bits + 7) // 8
+    return (n + align - 1) // align * align
+
+
+def pack_indices(idx, bits: int, pitch: Optional[int] = None) -> np.ndarray:
+    """uint16 [N, Kb] -> uint8 [N, pitch]: each row the little-endian bit string of its indices, `bits` bits each."""
+    idx = np.ascontiguousarray(idx, dtype=np.uint16)
+    N, Kb = idx.shape
+    pitch = packed_row_bytes(Kb, bits) if pitch is None else pitch
+    out = np.empty((N, pitch), dtype=np.uint8)
+    _check(_load().btc_oracle_pack_indices(_p(idx), N, Kb, bits, ctypes.c_size_t(pitch), _p(out)))
+    return out
+
+
+def unpack_indices(packed, Kb: int, bits: int) -> np.ndarray:
+    packed = np.ascontiguousarray(packed, dtype=np.uint8)
+    N, pitch = packed.shape
+    idx = np.empty((N, Kb), dtype=np.uint16)
+    _check(_load().btc_oracle_unpack_indices(_p(packed), N, Kb, bits, ctypes.c_size_t(pitch), _p(idx)))
+    return idx
+
+
 def sqdist_pm1(b, c) -> float:
     b = np.ascontiguousarray(b, dtype=np.int8)
     c = np.ascontiguousarray(c, dtype=np.int8)

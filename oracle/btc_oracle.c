@@ -202,6 +202,44 @@ double btc_oracle_storage_bits(int N, int K, int v, int Kc)
 }
 
 /*
+ * Dense index packing (Section 4.3 counts ceil(log2 c) bits per index: "v*c + ceil(log2 c) * mn/v").
+ * Row n of the packed matrix is the little-endian bit string of its K/v indices, `bits` bits each:
+ * bit q of index j is bit j*bits + q of the row, and bit p of the row is bit p % 8 of byte p / 8.
+ * Rows start every `pitch` bytes (pitch >= ceil(Kb*bits/8)); bytes between the end of the bit string and
+ * the pitch are zero.  Written bit by bit on purpose.
+ */
+int btc_oracle_pack_indices(const uint16_t *idx, int N, int Kb, int bits, size_t pitch, uint8_t *out)
+{
+    if (bits < 1 || bits > 16 || pitch * 8 < (size_t)Kb * bits) return 2;
+    memset(out, 0, pitch * (size_t)N);
+    for (int n = 0; n < N; ++n)
+        for (int j = 0; j < Kb; ++j) {
+            const unsigned val = idx[(size_t)n * Kb + j];
+            if (bits < 16 && (val >> bits)) return 3;
+            for (int q = 0; q < bits; ++q) {
+                const size_t p = (size_t)j * bits + q;
+                if ((val >> q) & 1u) out[(size_t)n * pitch + p / 8] |= (uint8_t)(1u << (p % 8));
+            }
+        }
+    return 0;
+}
+
+int btc_oracle_unpack_indices(const uint8_t *in, int N, int Kb, int bits, size_t pitch, uint16_t *idx)
+{
+    if (bits < 1 || bits > 16 || pitch * 8 < (size_t)Kb * bits) return 2;
+    for (int n = 0; n < N; ++n)
+        for (int j = 0; j < Kb; ++j) {
+            unsigned val = 0;
+            for (int q = 0; q < bits; ++q) {
+                const size_t p = (size_t)j * bits + q;
+                if ((in[(size_t)n * pitch + p / 8] >> (p % 8)) & 1u) val |= 1u << q;
+            }
+            idx[(size_t)n * Kb + j] = (uint16_t)val;
+        }
+    return 0;
+}
+
+/*
  * Bits per weight.  mode 0 "nominal": log2(Kc)/v; mode 1 "container": ceil(log2 Kc)/v (the paper's
  * accounting); mode 2 "stored": 16/v (uint16 indices as this library keeps them).  Adds the row
  * scales (scale_bits_per_row / K) and, when with_codebook != 0, the codebook v*Kc/(N*K).

@@ -414,3 +414,51 @@ def test_kmeans_objective_never_increases_and_few_distinct_vectors_are_kept_exac
     C2, z2, iters, n_unique = km.optimize_codebook(few, c + 5, max_iter=10)
     assert C2.shape[0] == n_unique <= c and km.total_hamming(few, C2, z2) == 0
     assert len({tuple(r) for r in C2.tolist()}) == n_unique
+
+
+# ------------------------------------------------------------------ dense index packing (Section 4.3)
+
+def test_index_packing_hand_written_12_bit_example():
+    """Two 12-bit indices 0xABC, 0x123 -> bit string LSB first: bytes BC, 3A (low nibble A of the first index's top
+    bits, high nibble 3 of the second index's low bits), 12.  Worked by hand."""
+    idx = np.array([[0xABC, 0x123]], dtype=np.uint16)
+    packed = oracle.pack_indices(idx, 12, pitch=4)
+    assert packed.tolist() == [[0xBC, 0x3A, 0x12, 0x00]]
+    assert oracle.unpack_indices(packed, 2, 12).tolist() == [[0xABC, 0x123]]
+    # 13 bits: 0x1ABC, 0x0123 -> bits 0..12 = 0x1ABC, bits 13..25 = 0x0123: the 26-bit number 0x0123 << 13 | 0x1ABC
+    word = (0x0123 << 13) | 0x1ABC
+    packed13 = oracle.pack_indices(np.array([[0x1ABC, 0x0123]], dtype=np.uint16), 13, pitch=4)
+    assert packed13.tolist() == [[word & 0xFF, (word >> 8) & 0xFF, (word >> 16) & 0xFF, (word >> 24) & 0xFF]]
+
+
+@pytest.mark.parametrize("bits", [1, 5, 8, 12, 13, 15, 16])
+def test_index_packing_against_numpy_bit_strings_and_round_trip(bits):
+    """Independent construction: numpy unpackbits / packbits with little-endian bit order over the concatenated fields."""
+    rng = np.random.default_rng(bits)
+    N, Kb = 7, 37
+    idx = rng.integers(0, 1 << bits, size=(N, Kb), dtype=np.uint32).astype(np.uint16)
+    packed = oracle.pack_indices(idx, bits)
+    fields = ((idx[:, :, None].astype(np.uint32) >> np.arange(bits, dtype=np.uint32)) & 1).astype(np.uint8)   # [N, Kb, bits]
+    want = np.packbits(fields.reshape(N, Kb * bits), axis=1, bitorder="little")
+    nbytes = (Kb * bits + 7) // 8
+    assert packed.shape[1] == oracle.packed_row_bytes(Kb, bits) and packed.shape[1] % 16 == 0
+    assert np.array_equal(packed[:, :nbytes], want) and not packed[:, nbytes:].any()
+    assert np.array_equal(oracle.unpack_indices(packed, Kb, bits), idx)
+
+
+def test_index_packing_size_is_the_papers_storage_count():
+    """Section 4.3: the indices of an m x n layer take ceil(log2 c) * mn / v bits.  A packed 4096 x 4096 layer at v = 16
+    holds exactly that many bits (the row length is a multiple of 16 bytes here, so there is no padding), and the
+    index width follows the codebook sizes of Table 3a."""
+    for Kc, bits in ((4096, 12), (8192, 13), (7132, 13), (21619, 15), (65536, 16), (256, 8), (2, 1), (1, 1)):
+        assert oracle.index_bits(Kc) == bits
+    N = K = 4096
+    v = 16
+    for Kc in (4096, 8192):
+        b = oracle.index_bits(Kc)
+        assert oracle.packed_row_bytes(K // v, b) * N * 8 == oracle.storage_bits(N, K, v, Kc) - v * Kc
+    # rejects an index that does not fit the width, and a pitch shorter than the bit string
+    with pytest.raises(ValueError):
+        oracle.pack_indices(np.array([[4096]], dtype=np.uint16), 12)
+    with pytest.raises(ValueError):
+        oracle.pack_indices(np.zeros((1, 9), dtype=np.uint16), 12, pitch=13)
