@@ -392,6 +392,20 @@ def run_gpu(args):
             step_m[f"M{M}"] = {"us": tM * 1e6, "GBps": bM / tM * 1e-9, "frac_measured": bM / tM * 1e-9 / peaks["hbm_gbs"]}
         details["step_by_M"] = step_m
 
+        # ---- the same step over dense-packed 13-bit index rows (Section 4.3's index width: 0.8125 bit per weight stored)
+        packed_sets = [[btc.index_pack(sets[r][i]["idx"], s.Kc) for i, s in enumerate(specs)] for r in range(R)]
+        outs_p = [torch.empty((1, s.N), dtype=torch.float32, device=dev) for s in specs]
+        batches_p = [btc.GemvBatch([dict(x=xs1[i], idx=packed_sets[r][i], idx_bits=btc.index_bits(s.Kc), C_packed=sets[r][i]["Cp"],
+                                         alpha=sets[r][i]["alpha"], v=s.v, Kc=s.Kc, out=outs_p[i]) for i, s in enumerate(specs)])
+                     for r in range(R)]
+        tP = time_steps(lambda r: batches_p[r].run(), 60, 5, replays=9)[4] / 60
+        bP = sum(int(packed_sets[0][i].numel()) + 4 * s.Kc + 2 * s.N + 2 * s.K + 4 * s.N for i, s in enumerate(specs))
+        details["step_packed_indices_M1"] = {"us": tP * 1e6, "algorithmic_bytes": bP, "GBps": bP / tP * 1e-9,
+                                             "frac_measured": bP / tP * 1e-9 / peaks["hbm_gbs"],
+                                             "index_bits": btc.index_bits(specs[0].Kc),
+                                             "stored_bits_per_weight": btc.index_bits(specs[0].Kc) / specs[0].v}
+        del packed_sets, batches_p
+
         # ---- tensor-core path, config 4 shapes, with a cuBLAS fp16 GEMM of the same shape as context
         gem = {}
         c4 = wl.CONFIGS[4]

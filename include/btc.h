@@ -183,15 +183,37 @@ BTC_API int btc_linear_gemm(const void *x, int x_dtype, const uint16_t *idx, con
 #define BTC_BATCH_MAX 8
 typedef struct {
     const void *x;
-    const uint16_t *idx;
+    const void *idx;       /* uint16 [N, K/v]; or, with idx_bits set, the rows written by btc_index_pack */
     const uint32_t *C_packed;
     const void *alpha;
     const void *mu;        /* NULL = no mean term */
     void *y;
     int x_dtype, y_dtype;
     int M, N, K, v, Kc;
+    int idx_bits;          /* 0 or 16: uint16 containers; else btc_index_bits(Kc): dense-packed rows (see below) */
 } btc_linear_problem;
 BTC_API int btc_linear_gemv_batch(const btc_linear_problem *problems, int count, void *stream);
+
+/* ---- dense-packed indices ------------------------------------------------------------------
+ * The paper's storage count gives an index ceil(log2 c) bits ("v*c + ceil(log2 c) * mn/v", Section 4.3): 12 bits for
+ * 4096 centroids, 13 for 8192 (Table 3a pairs v = 16 with codebooks of that size), which is what makes v = 16 a
+ * sub-1-bit format; in uint16 containers the same layer occupies 16/v = 1 bit per weight.  btc_index_pack rewrites
+ * uint16 [N, Kb] indices as N rows of btc_index_packed_row_bytes(Kb, Kc) bytes (the bit string rounded up to 16
+ * bytes; padding is zero): row n is the little-endian bit string of its Kb indices, btc_index_bits(Kc) bits each --
+ * bit q of index j is bit j*bits + q of the row, bit p of the row is bit p % 8 of byte p / 8.  btc_index_unpack is
+ * the inverse.  idx values must be < 2^bits (higher bits are dropped).  Both are device-to-device, asynchronous on
+ * `stream`; `packed` 16-byte aligned.
+ * btc_linear_gemv_packed is btc_linear_gemv (no transform, no workspace) reading such rows; the same layers ride in
+ * btc_linear_gemv_batch with idx_bits set.  The decode kernel unpacks widths of 12 and 13 bits (v a multiple of 4 up
+ * to 16, codeword table in shared memory); other widths return BTC_ERR_UNSUPPORTED -- keep those layers in uint16
+ * containers.  All layers of one batch call must use the same index format. */
+BTC_API int btc_index_bits(int Kc);                            /* ceil(log2 Kc), at least 1; 0 for an invalid Kc */
+BTC_API size_t btc_index_packed_row_bytes(int Kb, int Kc);
+BTC_API int btc_index_pack(const uint16_t *idx, int N, int Kb, int Kc, void *packed, void *stream);
+BTC_API int btc_index_unpack(const void *packed, int N, int Kb, int Kc, uint16_t *idx, void *stream);
+BTC_API int btc_linear_gemv_packed(const void *x, int x_dtype, const void *idx_packed, const uint32_t *C_packed,
+                    const void *alpha, const void *mu, void *y, int y_dtype, int M, int N, int K, int v, int Kc,
+                    void *stream);
 
 /* ---- btc_linear_gemm for callers that cannot allocate device memory ---------------------------
  * (No counterpart in the paper: this is a packaging variant of btc_linear_gemm, same arithmetic.)

@@ -22,6 +22,7 @@ EXPORTS = (
     "btc_codebook_pack", "btc_codebook_pack_host", "btc_linear_workspace_bytes", "btc_linear_gemv",
     "btc_linear_gemm", "btc_linear_gemv_batch", "btc_linear_gemm_static_scratch", "btc_decode_pm1", "btc_validate_indices", "btc_bits_per_weight", "btc_device_status", "btc_device_status_reset", "btc_selftest_bounded_wait",
     "btc_codebook_kmeans_workspace_bytes", "btc_codebook_kmeans",
+    "btc_index_bits", "btc_index_packed_row_bytes", "btc_index_pack", "btc_index_unpack", "btc_linear_gemv_packed",
 )
 
 
@@ -34,7 +35,8 @@ class BtcLinearProblem(ctypes.Structure):
     _fields_ = [("x", ctypes.c_void_p), ("idx", ctypes.c_void_p), ("C_packed", ctypes.c_void_p),
                 ("alpha", ctypes.c_void_p), ("mu", ctypes.c_void_p), ("y", ctypes.c_void_p),
                 ("x_dtype", ctypes.c_int), ("y_dtype", ctypes.c_int),
-                ("M", ctypes.c_int), ("N", ctypes.c_int), ("K", ctypes.c_int), ("v", ctypes.c_int), ("Kc", ctypes.c_int)]
+                ("M", ctypes.c_int), ("N", ctypes.c_int), ("K", ctypes.c_int), ("v", ctypes.c_int), ("Kc", ctypes.c_int),
+                ("idx_bits", ctypes.c_int)]
 
 
 class BtcError(RuntimeError):
@@ -76,6 +78,12 @@ def _load() -> ctypes.CDLL:
     L.btc_codebook_kmeans_workspace_bytes.restype = sz
     L.btc_codebook_kmeans_workspace_bytes.argtypes = [ci, ci]
     L.btc_codebook_kmeans.argtypes = [vp, sz, ci, ci, ci, vp, vp, vp, vp, sz, vp]
+    L.btc_index_bits.argtypes = [ci]
+    L.btc_index_packed_row_bytes.restype = sz
+    L.btc_index_packed_row_bytes.argtypes = [ci, ci]
+    L.btc_index_pack.argtypes = [vp, ci, ci, ci, vp, vp]
+    L.btc_index_unpack.argtypes = [vp, ci, ci, ci, vp, vp]
+    L.btc_linear_gemv_packed.argtypes = [vp, ci, vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, vp]
     L.btc_bits_per_weight.restype = ctypes.c_double
     L.btc_bits_per_weight.argtypes = [ci] * 7
     return L
@@ -208,18 +216,26 @@ class GemvBatch:
             for t, n in ((x, "x"), (idx, "idx"), (Cp, "C_packed"), (alpha, "alpha")):
                 _dev(t, n)
             M, K = x.shape
-            N, Kb = idx.shape
             v, Kc = int(L["v"]), int(L["Kc"])
+            bits = int(L.get("idx_bits", 0))
+            if bits in (0, 16):
+                N, Kb = idx.shape
+                if idx.element_size() != 2:
+                    raise ValueError("idx must be 16-bit")
+            else:                       # dense-packed rows (uint8 [N, row bytes]) written by index_pack
+                N, Kb = idx.shape[0], K // v
+                if idx.dtype != torch.uint8 or idx.shape[1] != int(lib.btc_index_packed_row_bytes(Kb, Kc)):
+                    raise ValueError("idx is not the buffer index_pack wrote for this (K/v, Kc)")
             if Kb * v != K or alpha.numel() != N or Cp.numel() != packed_words(Kc, v):
                 raise ValueError("shape mismatch between x, idx, v, alpha and C_packed")
-            if x.dtype not in (torch.float16, torch.bfloat16) or alpha.dtype != torch.float16 or idx.element_size() != 2:
-                raise ValueError("x must be fp16/bf16, alpha fp16, idx 16-bit")
+            if x.dtype not in (torch.float16, torch.bfloat16) or alpha.dtype != torch.float16:
+                raise ValueError("x must be fp16/bf16, alpha fp16")
             mu = L.get("mu")
             out = L.get("out")
             if out is None:
                 out = torch.empty((M, N), dtype=torch.float32, device=x.device)
             arr[i] = BtcLinearProblem(x.data_ptr(), idx.data_ptr(), Cp.data_ptr(), alpha.data_ptr(), _ptr(mu),
-                                      out.data_ptr(), _DT[x.dtype], _DT[out.dtype], M, N, K, v, Kc)
+                                      out.data_ptr(), _DT[x.dtype], _DT[out.dtype], M, N, K, v, Kc, bits)
             self.layers.append((x, idx, Cp, alpha, mu, out))          # keeps the tensors alive
         self._arr = arr
         self.outs = [t[5] for t in self.layers]
@@ -257,6 +273,50 @@ def linear_gemm_static_scratch(x, idx, C_packed, alpha, v, Kc, mu=None, out=None
                                             M, N, K, v, Kc, _stream())
     if st:
         raise BtcError(st, "btc_linear_gemm_static_scratch")
+    return out
+
+
+def index_bits(Kc: int) -> int:
+    return int(lib.btc_index_bits(Kc))
+
+
+def index_pack(idx: torch.Tensor, Kc: int) -> torch.Tensor:
+    """16-bit indices [N, K/v] (device) -> dense-packed rows, uint8 [N, row bytes] (btc_index_pack)."""
+    _dev(idx, "idx")
+    if idx.dim() != 2 or idx.element_size() != 2:
+        raise ValueError("idx must be 16-bit integers [N, K/v]")
+    N, Kb = idx.shape
+    out = torch.empty((N, int(lib.btc_index_packed_row_bytes(Kb, Kc))), dtype=torch.uint8, device=idx.device)
+    st = lib.btc_index_pack(idx.data_ptr(), N, Kb, Kc, out.data_ptr(), _stream())
+    if st:
+        raise BtcError(st, "btc_index_pack")
+    return out
+
+
+def index_unpack(packed: torch.Tensor, Kb: int, Kc: int) -> torch.Tensor:
+    _dev(packed, "packed")
+    N = packed.shape[0]
+    out = torch.empty((N, Kb), dtype=torch.int16, device=packed.device)
+    st = lib.btc_index_unpack(packed.data_ptr(), N, Kb, Kc, out.data_ptr(), _stream())
+    if st:
+        raise BtcError(st, "btc_index_unpack")
+    return out
+
+
+def linear_gemv_packed(x, idx_packed, C_packed, alpha, v, Kc, mu=None, out=None, out_dtype=torch.float32):
+    """btc_linear_gemv_packed: the decode path (M <= 8) reading dense-packed index rows."""
+    for t, n in ((x, "x"), (idx_packed, "idx_packed"), (C_packed, "C_packed"), (alpha, "alpha")):
+        _dev(t, n)
+    M, K = x.shape
+    N = idx_packed.shape[0]
+    if idx_packed.dtype != torch.uint8 or idx_packed.shape[1] != int(lib.btc_index_packed_row_bytes(K // v, Kc)):
+        raise ValueError("idx_packed is not the buffer index_pack wrote for this (K/v, Kc)")
+    if out is None:
+        out = torch.empty((M, N), dtype=out_dtype, device=x.device)
+    st = lib.btc_linear_gemv_packed(x.data_ptr(), _DT[x.dtype], idx_packed.data_ptr(), C_packed.data_ptr(), alpha.data_ptr(),
+                                    _ptr(mu), out.data_ptr(), _DT[out.dtype], M, N, K, v, Kc, _stream())
+    if st:
+        raise BtcError(st, "btc_linear_gemv_packed")
     return out
 
 

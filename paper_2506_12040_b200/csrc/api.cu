@@ -158,16 +158,24 @@ extern "C" int btc_linear_gemv_batch(const btc_linear_problem *problems, int cou
         int n = 0;
         for (; n < IM_MAXP && i + n < count; ++n) {
             const btc_linear_problem &p = problems[i + n];
-            int rc = validate(p.x, p.x_dtype, p.idx, p.C_packed, p.alpha, p.y, p.y_dtype, p.M, p.N, p.K, p.v, p.Kc);
+            int rc = validate(p.x, p.x_dtype, static_cast<const uint16_t *>(p.idx), p.C_packed, p.alpha, p.y, p.y_dtype, p.M, p.N, p.K, p.v, p.Kc);
             if (rc != BTC_OK) return rc;
             if (p.mu && !aligned(p.mu, 2)) return BTC_ERR_ALIGN;
             if (p.M > 8) return BTC_ERR_SHAPE;
-            if (debug_check_indices_enabled()) {
-                rc = launch_index_check(p.idx, (size_t)p.N * (p.K / p.v), p.Kc, s);
+            if (debug_check_indices_enabled() && (p.idx_bits == 0 || p.idx_bits == 16)) {
+                rc = launch_index_check(static_cast<const uint16_t *>(p.idx), (size_t)p.N * (p.K / p.v), p.Kc, s);
                 if (rc != BTC_OK) return rc;
             }
             LinearArgs &a = group[n];
-            a.x = p.x; a.idx = p.idx; a.Cp = p.C_packed;
+            a = LinearArgs();
+            if (p.idx_bits != 0 && p.idx_bits != 16) {
+                // dense-packed rows: the width must be the codebook's index width
+                if (p.idx_bits != btc_index_bits(p.Kc)) return BTC_ERR_SHAPE;
+                a.idx_bits = p.idx_bits;
+                a.idx_packed = p.idx;
+                a.idx_pitch = btc_index_packed_row_bytes(p.K / p.v, p.Kc);
+            }
+            a.x = p.x; a.idx = static_cast<const uint16_t *>(p.idx); a.Cp = p.C_packed;
             a.alpha = reinterpret_cast<const __half *>(p.alpha);
             a.mu = reinterpret_cast<const __half *>(p.mu);
             a.y = p.y; a.workspace = nullptr; a.workspace_bytes = 0;
@@ -179,6 +187,7 @@ extern "C" int btc_linear_gemv_batch(const btc_linear_problem *problems, int cou
             // some layer of the run is outside the fused kernel: one launch per layer instead
             for (int k = 0; k < n; ++k) {
                 rc = launch_gemv_imma(&group[k], 1, s);
+                if (rc == BTC_ERR_UNSUPPORTED && group[k].idx_bits) return rc;     // only the decode kernel reads dense indices
                 if (rc == BTC_ERR_UNSUPPORTED) rc = launch_gemv_decode(group[k], s);
                 if (rc == BTC_ERR_UNSUPPORTED) rc = launch_linear_generic(group[k], s);
                 if (rc != BTC_OK) return rc;
@@ -202,4 +211,16 @@ extern "C" double btc_bits_per_weight(int N, int K, int v, int Kc, int scale_bit
     double r = ib / v + (double)scale_bits_per_row / K;
     if (with_codebook) r += (double)v * Kc / ((double)N * K);
     return r;
+}
+
+extern "C" int btc_linear_gemv_packed(const void *x, int x_dtype, const void *idx_packed, const uint32_t *C_packed,
+                                      const void *alpha, const void *mu, void *y, int y_dtype, int M, int N, int K,
+                                      int v, int Kc, void *stream)
+{
+    btc_linear_problem p;
+    p.x = x; p.idx = idx_packed; p.C_packed = C_packed; p.alpha = alpha; p.mu = mu; p.y = y;
+    p.x_dtype = x_dtype; p.y_dtype = y_dtype; p.M = M; p.N = N; p.K = K; p.v = v; p.Kc = Kc;
+    p.idx_bits = btc_index_bits(Kc);
+    if (p.idx_bits == 16) p.idx_bits = 0;                    // 16-bit fields ARE the uint16 container
+    return btc_linear_gemv_batch(&p, 1, stream);
 }

@@ -19,6 +19,10 @@ struct LinearArgs {
     size_t workspace_bytes;
     int x_dt, y_dt;
     int M, N, K, v, Kc, Kb;   // Kb = K / v
+    // dense-packed indices (idx_bits > 0): idx is unused, idx_packed holds rows of idx_pitch bytes, idx_bits bits per index
+    const void *idx_packed = nullptr;
+    size_t idx_pitch = 0;
+    int idx_bits = 0;
 };
 
 // Records a CUDA error for btc_last_cuda_error() and maps it to BTC_ERR_CUDA.

@@ -58,7 +58,7 @@ __device__ int g_imma_status = 0;
 
 struct ImProblem {
     const void *x;
-    const uint16_t *idx;
+    const void *idx;          // uint16 [N, K/v], or rows of dense ib-bit fields
     const uint32_t *tab;      // byte-lane codeword words [Kc]
     const uint16_t *tab16;    // the same squeezed into 16 bits (v <= 16)
     const __half *alpha;
@@ -170,6 +170,42 @@ __device__ __forceinline__ uint32_t im_lds32(uint32_t addr) {
     asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(addr));
     return v;
 }
+// NF consecutive IB-bit fields starting at field f0 of a packed row in shared memory (row: 4-byte aligned).  The words
+// that hold them are read aligned and shifted into place; one word past the last needed bit may be read (the stage
+// keeps 16 spare bytes for it).
+template <int IB, int NF>
+__device__ __forceinline__ void im_unpack_fields(const unsigned char *row, int f0, uint32_t (&f)[NF])
+{
+    constexpr int NW = (NF * IB + 31) / 32;                // words of the aligned bit string
+    const uint32_t bit0 = (uint32_t)f0 * IB;
+    const uint32_t *wp = reinterpret_cast<const uint32_t *>(row) + (bit0 >> 5);
+    const uint32_t sh = bit0 & 31u;
+    uint32_t w[NW + 1], a[NW + 1];
+#pragma unroll
+    for (int k = 0; k <= NW; ++k) w[k] = wp[k];
+#pragma unroll
+    for (int k = 0; k < NW; ++k) a[k] = __funnelshift_r(w[k], w[k + 1], sh);
+    a[NW] = 0u;
+#pragma unroll
+    for (int i = 0; i < NF; ++i) {
+        constexpr uint32_t mask = (1u << IB) - 1u;
+        const int lo = (i * IB) >> 5, s = (i * IB) & 31;
+        f[i] = __funnelshift_r(a[lo], a[lo + 1], s) & mask;
+    }
+}
+// Codeword of index i: from the shared table (32-bit words, or 16-bit halves widened by h | (h << 12)), its shared
+// head, or global memory, as TAB_MODE says.
+template <int TAB_MODE>
+__device__ __forceinline__ uint32_t im_codeword(uint32_t i, const uint32_t *s_tab, const uint32_t *gtab, uint32_t tab_head)
+{
+    if (TAB_MODE == 1) return s_tab[i];
+    if (TAB_MODE == 3) {
+        const uint32_t h = reinterpret_cast<const uint16_t *>(s_tab)[i];
+        return h | (h << 12);
+    }
+    if (TAB_MODE == 0) return __ldg(gtab + i);
+    return i < tab_head ? s_tab[i] : __ldg(gtab + i);
+}
 __device__ __forceinline__ void im_named_bar(int id, int threads) {
     asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
 }
@@ -250,15 +286,23 @@ template <int NM> struct ImShape {
     static constexpr int MAXM = (NM == 1) ? 2 : 8;
     static constexpr int RC = 12;                              // tiles a CTA walks part by part at a time
     static constexpr int PROW = RC * 16 + 4;                   // NM = 0: floats per (slice, m) row of the partial sums
-    static constexpr int STAGE_BYTES = PW / IM_BOX_COLS * IM_BOX_BYTES;
 };
 
-__host__ __device__ inline ImSmem im_smem_layout(int tab_bytes, int nm, int stages)
+// Bytes of one index stage: a (tile, part) of 16 rows.  ib = 0: 16-bit containers, boxes of 64 blocks x 16 rows with the
+// 128-byte swizzle.  ib > 0: dense ib-bit fields (Section 4.3's index width), one unswizzled box of 16 rows x
+// part_width * ib / 8 bytes, plus one spare 16 bytes because a lane's last aligned word may lie just past its row.
+__host__ __device__ constexpr int im_stage_bytes(int nm, int ib)
+{
+    return ib == 0 ? (nm == 1 ? 256 : 128) / IM_BOX_COLS * IM_BOX_BYTES
+                   : (16 * ((nm == 1 ? 256 : 128) * ib / 8) + 16 + 127) / 128 * 128;
+}
+
+__host__ __device__ inline ImSmem im_smem_layout(int tab_bytes, int nm, int stages, int ib = 0)
 {
     const int slice = (nm == 1 ? 256 : 128) / IM_CWARPS;
     const int maxm = nm == 1 ? 2 : 8;
     const int rc = 12;
-    const int stage_bytes = (nm == 1 ? 256 : 128) / IM_BOX_COLS * IM_BOX_BYTES;
+    const int stage_bytes = im_stage_bytes(nm, ib);
     ImSmem L;
     uint32_t o = 0;
     L.bars = o; o += IM_NBARS * 8;
@@ -293,15 +337,16 @@ __device__ __forceinline__ void im_group_range(const ImProblem &P, int b, int &l
 // TAB_MODE 0: tables gathered from global memory; 1: whole tables in shared memory; 2: the first tab_head entries in
 // shared memory, the rest from global memory; 3: whole tables in shared memory as 16-bit halves (v <= 16; a table of
 // 65536 codewords then takes 128 KB), widened by `h | (h << 12)` after the gather.
-template <int NCLS, int NM, int TAB_MODE>
+template <int NCLS, int NM, int TAB_MODE, int IB>
 __global__ void __launch_bounds__(IM_THREADS, 2)
 gemv_imma_kernel(const __grid_constant__ ImBatch batch)
 {
     extern __shared__ __align__(128) unsigned char smem[];
     using S = ImShape<NM>;
     constexpr int PW = S::PW, SLICE = S::SLICE, BPL = S::BPL, MAXM = S::MAXM, RC = S::RC;
-    constexpr int STAGE_BYTES = S::STAGE_BYTES;
-    const ImSmem L = im_smem_layout(batch.tab_smem_bytes, NM, batch.stages);
+    constexpr int STAGE_BYTES = im_stage_bytes(NM, IB);
+    constexpr int ROWB = PW * IB / 8;                     // bytes of one row of a packed stage (IB > 0)
+    const ImSmem L = im_smem_layout(batch.tab_smem_bytes, NM, batch.stages, IB);
     const int NST = batch.stages;
     uint64_t *bars = reinterpret_cast<uint64_t *>(smem + L.bars);
     volatile int *s_abort = reinterpret_cast<volatile int *>(smem + L.misc);
@@ -356,11 +401,19 @@ gemv_imma_kernel(const __grid_constant__ ImBatch batch)
                     constexpr int nbox = PW / IM_BOX_COLS;
                     for (int r = c0; r < c1; ++r, ++li) {
                         if (li >= NST && !im_mbar_wait(bar_empty(s), rph ^ 1u, s_abort)) { ok = false; break; }
-                        if (lane == 0) im_mbar_expect_tx(bar_full(s), (uint32_t)nbox * IM_BOX_BYTES);
-                        __syncwarp();
-                        if (lane < nbox)
-                            im_tma_2d(im_smem_u32(s_ring + (size_t)s * STAGE_BYTES + (size_t)lane * IM_BOX_BYTES), &batch.map[pi],
-                                      j * PW + lane * IM_BOX_COLS, r * 16, bar_full(s));
+                        if constexpr (IB == 0) {
+                            if (lane == 0) im_mbar_expect_tx(bar_full(s), (uint32_t)nbox * IM_BOX_BYTES);
+                            __syncwarp();
+                            if (lane < nbox)
+                                im_tma_2d(im_smem_u32(s_ring + (size_t)s * STAGE_BYTES + (size_t)lane * IM_BOX_BYTES), &batch.map[pi],
+                                          j * PW + lane * IM_BOX_COLS, r * 16, bar_full(s));
+                        } else {
+                            // dense fields: the part of 16 rows is one box of 32-bit words (coordinates in words)
+                            if (lane == 0) {
+                                im_mbar_expect_tx(bar_full(s), 16u * ROWB);
+                                im_tma_2d(im_smem_u32(s_ring + (size_t)s * STAGE_BYTES), &batch.map[pi], j * (ROWB / 4), r * 16, bar_full(s));
+                            }
+                        }
                         if (++s == NST) { s = 0; rph ^= 1u; }
                     }
                 }
@@ -523,6 +576,28 @@ gemv_imma_kernel(const __grid_constant__ ImBatch batch)
                     uint32_t w0[BPL], w1[BPL];
                     auto fetch = [&]() {
                         ok &= im_mbar_wait(bar_full(s), rph, s_abort);
+                        if constexpr (IB > 0) {
+                            uint32_t fa[BPL], fb[BPL];
+                            const unsigned char *st = s_ring + (size_t)s * STAGE_BYTES;
+                            im_unpack_fields<IB, BPL>(st + sg * ROWB, ks * SLICE + BPL * t, fa);
+                            im_unpack_fields<IB, BPL>(st + (sg + 8) * ROWB, ks * SLICE + BPL * t, fb);
+                            if (!ok) {
+#pragma unroll
+                                for (int e = 0; e < BPL; ++e) { fa[e] = 0u; fb[e] = 0u; }
+                            }
+                            // (the loads must have returned before the stage is handed back: see below)
+#pragma unroll
+                            for (int e = 0; e < BPL; ++e) asm volatile("" :: "r"(fa[e]), "r"(fb[e]) : "memory");
+                            __syncwarp();
+                            if (lane == 0) im_mbar_arrive(bar_empty(s));
+                            if (++s == NST) { s = 0; rph ^= 1u; }
+#pragma unroll
+                            for (int e = 0; e < BPL; ++e) {
+                                w0[e] = im_codeword<TAB_MODE>(fa[e], s_tab, gtab, tab_head);
+                                w1[e] = im_codeword<TAB_MODE>(fb[e], s_tab, gtab, tab_head);
+                            }
+                            return;
+                        }
                         const unsigned char *pa = s_ring + (size_t)s * STAGE_BYTES + idx_off;
                         uint2 qa = *reinterpret_cast<const uint2 *>(pa), qb = *reinterpret_cast<const uint2 *>(pa + 8 * 128);
                         if (!ok) { qa = make_uint2(0u, 0u); qb = qa; }
@@ -549,11 +624,8 @@ gemv_imma_kernel(const __grid_constant__ ImBatch batch)
                             for (int e = 0; e < BPL; ++e) {
                                 const uint32_t i0 = (e & 1) ? (ia[e >> 1] >> 16) : (ia[e >> 1] & 0xffffu);
                                 const uint32_t i1 = (e & 1) ? (ib[e >> 1] >> 16) : (ib[e >> 1] & 0xffffu);
-                                if (TAB_MODE == 0) { w0[e] = __ldg(gtab + i0); w1[e] = __ldg(gtab + i1); }
-                                else {
-                                    w0[e] = i0 < tab_head ? s_tab[i0] : __ldg(gtab + i0);
-                                    w1[e] = i1 < tab_head ? s_tab[i1] : __ldg(gtab + i1);
-                                }
+                                w0[e] = im_codeword<TAB_MODE>(i0, s_tab, gtab, tab_head);
+                                w1[e] = im_codeword<TAB_MODE>(i1, s_tab, gtab, tab_head);
                             }
                         }
                     };
@@ -836,19 +908,35 @@ gemv_imma_kernel(const __grid_constant__ ImBatch batch)
                     auto fetch = [&]() {
                         uint32_t ia[BPL / 2], ib[BPL / 2];
                         ok &= im_mbar_wait(bar_full(s), rph, s_abort);
+                        if constexpr (IB > 0) {
+                            uint32_t fa[BPL], fb[BPL];
+                            const unsigned char *st = s_ring + (size_t)s * STAGE_BYTES;
+                            im_unpack_fields<IB, BPL>(st + sg * ROWB, ks * SLICE + BPL * t, fa);
+                            im_unpack_fields<IB, BPL>(st + (sg + 8) * ROWB, ks * SLICE + BPL * t, fb);
+                            if (!ok) {
+#pragma unroll
+                                for (int e = 0; e < BPL; ++e) { fa[e] = 0u; fb[e] = 0u; }
+                            }
+                            // (the loads must have returned before the stage is handed back: see the fp16 form)
+#pragma unroll
+                            for (int e = 0; e < BPL; ++e) asm volatile("" :: "r"(fa[e]), "r"(fb[e]) : "memory");
+                            __syncwarp();
+                            if (lane == 0) im_mbar_arrive(bar_empty(s));
+                            if (++s == NST) { s = 0; rph ^= 1u; }
+#pragma unroll
+                            for (int e = 0; e < BPL; ++e) {
+                                w0[e] = im_codeword<TAB_MODE>(fa[e], s_tab, gtab, tab_head);
+                                w1[e] = im_codeword<TAB_MODE>(fb[e], s_tab, gtab, tab_head);
+                            }
+                            return;
+                        }
                         {
                             // (every stage is filled whole: blocks past the part and rows past N arrive as zeros)
                             const unsigned char *pa = s_ring + (size_t)s * STAGE_BYTES + idx_off;
                             const unsigned char *pb = pa + 8 * 128;                 // row + 8: same row & 7
-                            if (BPL == 8) {
-                                const uint4 qa = *reinterpret_cast<const uint4 *>(pa), qb = *reinterpret_cast<const uint4 *>(pb);
-                                ia[0] = qa.x; ia[1] = qa.y; ia[BPL / 2 - 2] = qa.z; ia[BPL / 2 - 1] = qa.w;
-                                ib[0] = qb.x; ib[1] = qb.y; ib[BPL / 2 - 2] = qb.z; ib[BPL / 2 - 1] = qb.w;
-                            } else {
-                                const uint2 qa = *reinterpret_cast<const uint2 *>(pa), qb = *reinterpret_cast<const uint2 *>(pb);
-                                ia[0] = qa.x; ia[1] = qa.y;
-                                ib[0] = qb.x; ib[1] = qb.y;
-                            }
+                            const uint4 qa = *reinterpret_cast<const uint4 *>(pa), qb = *reinterpret_cast<const uint4 *>(pb);
+                            ia[0] = qa.x; ia[1] = qa.y; ia[2] = qa.z; ia[3] = qa.w;
+                            ib[0] = qb.x; ib[1] = qb.y; ib[2] = qb.z; ib[3] = qb.w;
                         }
                         if (!ok) {                                  // a wait gave up: the stage may hold anything
 #pragma unroll
@@ -878,16 +966,8 @@ gemv_imma_kernel(const __grid_constant__ ImBatch batch)
                                 const uint32_t pa = ia[e >> 1], pb = ib[e >> 1];
                                 const uint32_t i0 = (e & 1) ? (pa >> 16) : (pa & 0xffffu);
                                 const uint32_t i1 = (e & 1) ? (pb >> 16) : (pb & 0xffffu);
-                                if (TAB_MODE == 3) {
-                                    const uint32_t h0 = reinterpret_cast<const uint16_t *>(s_tab)[i0];
-                                    const uint32_t h1 = reinterpret_cast<const uint16_t *>(s_tab)[i1];
-                                    w0[e] = h0 | (h0 << 12); w1[e] = h1 | (h1 << 12);
-                                }
-                                else if (TAB_MODE == 0) { w0[e] = __ldg(gtab + i0); w1[e] = __ldg(gtab + i1); }
-                                else {
-                                    w0[e] = i0 < tab_head ? s_tab[i0] : __ldg(gtab + i0);
-                                    w1[e] = i1 < tab_head ? s_tab[i1] : __ldg(gtab + i1);
-                                }
+                                w0[e] = im_codeword<TAB_MODE>(i0, s_tab, gtab, tab_head);
+                                w1[e] = im_codeword<TAB_MODE>(i1, s_tab, gtab, tab_head);
                             }
                         }
                     };
@@ -1015,25 +1095,36 @@ static im_encode_fn im_get_encode()
 // Tensor map of an index matrix {K/v, N} (16-bit words), box {64, 16}, 128-byte swizzle.  Encoding goes through the
 // driver and costs about a microsecond; a decode step re-uses the same matrices call after call, so the last few
 // maps are kept per host thread, keyed by everything the encoding depends on.
-static bool im_tensor_map(im_encode_fn enc, const uint16_t *idx, int Kb, int N, CUtensorMap *out)
+static bool im_tensor_map(im_encode_fn enc, const void *idx, int Kb, int N, int ib, size_t pitch, int box_words, CUtensorMap *out)
 {
-    struct Entry { const uint16_t *idx; int Kb, N; CUtensorMap map; };
+    struct Entry { const void *idx; int Kb, N, ib, box; CUtensorMap map; };
     constexpr int SLOTS = 64;
     thread_local Entry cache[SLOTS];
     thread_local int used = 0, next = 0;
     for (int i = 0; i < used; ++i)
-        if (cache[i].idx == idx && cache[i].Kb == Kb && cache[i].N == N) { *out = cache[i].map; return true; }
-    const cuuint64_t dims[2] = {(cuuint64_t)Kb, (cuuint64_t)N};
-    const cuuint64_t strides[1] = {(cuuint64_t)Kb * 2};
-    const cuuint32_t box[2] = {(cuuint32_t)IM_BOX_COLS, 16u};
+        if (cache[i].idx == idx && cache[i].Kb == Kb && cache[i].N == N && cache[i].ib == ib && cache[i].box == box_words) { *out = cache[i].map; return true; }
     const cuuint32_t estr[2] = {1, 1};
     CUtensorMap m;
-    if (enc(&m, CU_TENSOR_MAP_DATA_TYPE_UINT16, 2, const_cast<uint16_t *>(idx), dims, strides, box, estr,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
-        return false;
+    if (ib == 0) {
+        const cuuint64_t dims[2] = {(cuuint64_t)Kb, (cuuint64_t)N};
+        const cuuint64_t strides[1] = {(cuuint64_t)Kb * 2};
+        const cuuint32_t box[2] = {(cuuint32_t)IM_BOX_COLS, 16u};
+        if (enc(&m, CU_TENSOR_MAP_DATA_TYPE_UINT16, 2, const_cast<void *>(idx), dims, strides, box, estr,
+                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return false;
+    } else {
+        // dense ib-bit fields: rows of `pitch` bytes seen as 32-bit words; one box = a part of 16 rows, no swizzle
+        const cuuint64_t dims[2] = {(cuuint64_t)(pitch / 4), (cuuint64_t)N};
+        const cuuint64_t strides[1] = {(cuuint64_t)pitch};
+        const cuuint32_t box[2] = {(cuuint32_t)box_words, 16u};
+        if (enc(&m, CU_TENSOR_MAP_DATA_TYPE_UINT32, 2, const_cast<void *>(idx), dims, strides, box, estr,
+                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return false;
+    }
     Entry &e = cache[next];
-    e.idx = idx; e.Kb = Kb; e.N = N; e.map = m;
+    e.idx = idx; e.Kb = Kb; e.N = N; e.ib = ib; e.box = box_words; e.map = m;
     next = (next + 1) % SLOTS;
     if (used < SLOTS) ++used;
     *out = m;
@@ -1101,11 +1192,11 @@ static int im_assign_ctas(ImBatch &b, int budget)
     return begin;
 }
 
-template <int NCLS, int NM, int TS>
+template <int NCLS, int NM, int TS, int IB>
 static int im_launch(ImBatch &b, int groups_total, cudaStream_t s)
 {
-    const ImSmem L = im_smem_layout(b.tab_smem_bytes, NM, b.stages);
-    auto kern = gemv_imma_kernel<NCLS, NM, TS>;
+    const ImSmem L = im_smem_layout(b.tab_smem_bytes, NM, b.stages, IB);
+    auto kern = gemv_imma_kernel<NCLS, NM, TS, IB>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)L.total);
     if (e != cudaSuccess) return cuda_fail(e);
     cudaLaunchConfig_t cfg = {};
@@ -1127,11 +1218,25 @@ static int im_launch(ImBatch &b, int groups_total, cudaStream_t s)
 }
 
 template <int NCLS, int TS>
-static int im_launch_nm(ImBatch &b, int nm, int groups_total, cudaStream_t s)
+static int im_launch_nm(ImBatch &b, int nm, int ib, int groups_total, cudaStream_t s)
 {
-    if (nm == 1) return im_launch<NCLS, 1, TS>(b, groups_total, s);
+    if (ib != 0) {
+        // dense indices: built for the widths of the v = 16 codebooks of 4096 and 8192 centroids, whole table in
+        // shared memory
+        if constexpr (NCLS == 4 && (TS == 1 || TS == 3)) {
+            if (nm == 1) {
+                if (ib == 12) return im_launch<4, 1, TS, 12>(b, groups_total, s);
+                if (ib == 13) return im_launch<4, 1, TS, 13>(b, groups_total, s);
+            } else if (TS == 1) {
+                if (ib == 12) return im_launch<4, 0, 1, 12>(b, groups_total, s);
+                if (ib == 13) return im_launch<4, 0, 1, 13>(b, groups_total, s);
+            }
+        }
+        return BTC_ERR_UNSUPPORTED;
+    }
+    if (nm == 1) return im_launch<NCLS, 1, TS, 0>(b, groups_total, s);
     if (TS == 3) return BTC_ERR_UNSUPPORTED;                // (the 16-bit table exists for the byte-lane words only)
-    return im_launch<NCLS, 0, TS == 3 ? 1 : TS>(b, groups_total, s);
+    return im_launch<NCLS, 0, TS == 3 ? 1 : TS, 0>(b, groups_total, s);
 }
 
 int launch_gemv_imma(const LinearArgs *problems, int count, cudaStream_t s)
@@ -1148,7 +1253,9 @@ int launch_gemv_imma(const LinearArgs *problems, int count, cudaStream_t s)
         if (a.M < 1 || a.M > 8 || a.v % 4 != 0 || a.v > 20 || a.Kb % 8 != 0 || a.K > (1 << 20)) return BTC_ERR_UNSUPPORTED;
         if (a.x_dt == BTC_F32 && a.K % 8 != 0) return BTC_ERR_UNSUPPORTED;
         if (a.M > m_max) m_max = a.M;
+        if (a.idx_bits != problems[0].idx_bits) return BTC_ERR_UNSUPPORTED;      // one index format per launch
     }
+    const int ib = problems[0].idx_bits;
     const int nm = m_max <= 2 ? 1 : 0;                      // integer form up to two rows of x, fp16 form above
     const int pw = nm == 1 ? 256 : 128;
     // the ring is no longer than the longest walk of any CTA needs; the split below assumes the full ring
@@ -1156,7 +1263,7 @@ int launch_gemv_imma(const LinearArgs *problems, int count, cudaStream_t s)
     for (int i = 0; i < count; ++i) {
         const LinearArgs &a = problems[i];
         ImProblem &p = b.p[i];
-        p.x = a.x; p.idx = a.idx; p.alpha = a.alpha; p.mu = a.mu; p.y = a.y;
+        p.x = a.x; p.idx = a.idx_bits ? a.idx_packed : static_cast<const void *>(a.idx); p.alpha = a.alpha; p.mu = a.mu; p.y = a.y;
         const int Kc4 = (a.Kc + 3) / 4 * 4;
         p.tab = a.Cp + (nm == 0 ? 1 : 2) * Kc4;      // fp16-layout words (fp16 form) or byte-lane words (integer form)
         p.tab16 = reinterpret_cast<const uint16_t *>(a.Cp + 3 * (size_t)Kc4);
@@ -1165,7 +1272,7 @@ int launch_gemv_imma(const LinearArgs *problems, int count, cudaStream_t s)
         p.parts = (a.Kb + pw - 1) / pw;
         p.groups = (a.N + 15) / 16;
         p.ncls = a.v / 4;
-        if (!im_tensor_map(enc, a.idx, a.Kb, a.N, &b.map[i]))
+        if (!im_tensor_map(enc, p.idx, a.Kb, a.N, ib, a.idx_pitch, pw * ib / 32, &b.map[i]))
             return BTC_ERR_UNSUPPORTED;                     // shape the tensor map cannot describe: other kernels take it
         // a (tile, part) costs about the same whatever the part's width; rebuilding the activation fragments for a
         // part costs about as much as one and a half of them and is shared by the tiles a CTA walks with that part
@@ -1184,37 +1291,37 @@ int launch_gemv_imma(const LinearArgs *problems, int count, cudaStream_t s)
     b.tab_smem_bytes = tab_max;
     b.tab_head = tab_max / 4;
     uint32_t budget = half_sm;
-    if (im_smem_layout(tab_max, nm, 6).total > half_sm) {
-        if (nm == 1 && v_max <= 16 && im_smem_layout(tab16_max, nm, 4).total <= half_sm) {
+    if (im_smem_layout(tab_max, nm, 6, ib).total > half_sm) {
+        if (nm == 1 && v_max <= 16 && im_smem_layout(tab16_max, nm, 4, ib).total <= half_sm) {
             mode = 3;
             b.tab_smem_bytes = tab16_max;
-        } else if (nm == 1 && v_max <= 16 && im_smem_layout(tab16_max, nm, 2).total <= whole_sm) {
+        } else if (nm == 1 && v_max <= 16 && im_smem_layout(tab16_max, nm, 2, ib).total <= whole_sm) {
             mode = 3;
             b.tab_smem_bytes = tab16_max;
             budget = whole_sm;
-        } else if (im_smem_layout(tab_max, nm, 4).total <= whole_sm) {
+        } else if (im_smem_layout(tab_max, nm, 4, ib).total <= whole_sm) {
             budget = whole_sm;
         } else {
             mode = 2;
             budget = whole_sm;
             int head_bytes = tab_max;
-            while (head_bytes > 0 && im_smem_layout(head_bytes, nm, 4).total > whole_sm) head_bytes -= 4096;
+            while (head_bytes > 0 && im_smem_layout(head_bytes, nm, 4, ib).total > whole_sm) head_bytes -= 4096;
             if (head_bytes <= 0) { mode = 0; head_bytes = 0; }
             b.tab_smem_bytes = head_bytes;
             b.tab_head = head_bytes / 4;
         }
     }
     b.stages = IM_STAGES;
-    while (b.stages > 2 && im_smem_layout(b.tab_smem_bytes, nm, b.stages).total > budget) --b.stages;
+    while (b.stages > 2 && im_smem_layout(b.tab_smem_bytes, nm, b.stages, ib).total > budget) --b.stages;
     if (ncls_max <= 4) {
-        if (mode == 1) return im_launch_nm<4, 1>(b, nm, groups_total, s);
-        if (mode == 3) return im_launch_nm<4, 3>(b, nm, groups_total, s);
-        if (mode == 2) return im_launch_nm<4, 2>(b, nm, groups_total, s);
-        return im_launch_nm<4, 0>(b, nm, groups_total, s);
+        if (mode == 1) return im_launch_nm<4, 1>(b, nm, ib, groups_total, s);
+        if (mode == 3) return im_launch_nm<4, 3>(b, nm, ib, groups_total, s);
+        if (mode == 2) return im_launch_nm<4, 2>(b, nm, ib, groups_total, s);
+        return im_launch_nm<4, 0>(b, nm, ib, groups_total, s);
     }
-    if (mode == 1) return im_launch_nm<5, 1>(b, nm, groups_total, s);
-    if (mode == 2) return im_launch_nm<5, 2>(b, nm, groups_total, s);
-    return im_launch_nm<5, 0>(b, nm, groups_total, s);
+    if (mode == 1) return im_launch_nm<5, 1>(b, nm, ib, groups_total, s);
+    if (mode == 2) return im_launch_nm<5, 2>(b, nm, ib, groups_total, s);
+    return im_launch_nm<5, 0>(b, nm, ib, groups_total, s);
 }
 
 // Self-test of the bounded wait: one warp waits (with a ~1 ms limit) on a barrier that nothing ever arrives on, which

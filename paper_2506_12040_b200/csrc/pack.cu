@@ -80,6 +80,39 @@ __global__ void validate_indices_kernel(const uint16_t *__restrict__ idx, size_t
     if ((threadIdx.x & 31) == 0 && local) atomicAdd(bad, local);
 }
 
+// Dense index packing: row n of the output is the little-endian bit string of its Kb indices, `bits` bits each
+// (Section 4.3 counts ceil(log2 c) bits per index).  One thread per 32-bit word of a packed row: it collects the
+// fields that overlap its 32 bits.  Words past the bit string (row padding) are written as zeros.
+__global__ void index_pack_kernel(const uint16_t *__restrict__ idx, int N, int Kb, int bits, int pitch_words,
+                                  uint32_t *__restrict__ out)
+{
+    const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= (size_t)N * pitch_words) return;
+    const int n = (int)(i / pitch_words), w = (int)(i % pitch_words);
+    const long long b0 = 32ll * w, b1 = b0 + 32;              // this word's bit range of the row
+    uint32_t word = 0;
+    for (long long j = b0 / bits; j < Kb && j * bits < b1; ++j) {
+        const uint32_t val = idx[(size_t)n * Kb + j] & ((1u << bits) - 1u);
+        const long long sh = j * bits - b0;                   // position of the field's bit 0 in this word (may be < 0)
+        word |= sh >= 0 ? (val << sh) : (val >> (-sh));
+    }
+    out[i] = word;
+}
+
+__global__ void index_unpack_kernel(const uint32_t *__restrict__ in, int N, int Kb, int bits, int pitch_words,
+                                    uint16_t *__restrict__ idx)
+{
+    const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= (size_t)N * Kb) return;
+    const int n = (int)(i / Kb), j = (int)(i % Kb);
+    const long long bit = (long long)j * bits;
+    const uint32_t *row = in + (size_t)n * pitch_words;
+    const int w = (int)(bit >> 5), sh = (int)(bit & 31);
+    uint64_t two = row[w];
+    if (sh + bits > 32) two |= (uint64_t)row[w + 1] << 32;   // (only read when the field really crosses the word)
+    idx[i] = (uint16_t)((two >> sh) & ((1u << bits) - 1u));
+}
+
 // Debug aid (switched on by the environment variable BTC_DEBUG_CHECK_INDICES=1): raises a status word when an index is
 // >= Kc.  No trap, no assert: the layer kernels still run (their result is then undefined), the context stays usable and
 // btc_device_status reports BTC_ERR_INDEX.
@@ -185,5 +218,46 @@ extern "C" int btc_validate_indices(const uint16_t *idx, size_t count, int Kc, i
     size_t grid = (count + 255) / 256;
     if (grid > 148 * 16) grid = 148 * 16;
     validate_indices_kernel<<<(unsigned)grid, 256, 0, s>>>(idx, count, Kc, bad_count);
+    return cuda_check_launch();
+}
+
+extern "C" int btc_index_bits(int Kc)
+{
+    if (Kc < 1 || Kc > 65536) return 0;
+    int b = 1;
+    while ((1 << b) < Kc) ++b;
+    return b;
+}
+
+extern "C" size_t btc_index_packed_row_bytes(int Kb, int Kc)
+{
+    const int b = btc_index_bits(Kc);
+    if (b == 0 || Kb < 1) return 0;
+    return (((size_t)Kb * b + 7) / 8 + 15) / 16 * 16;
+}
+
+extern "C" int btc_index_pack(const uint16_t *idx, int N, int Kb, int Kc, void *packed, void *stream)
+{
+    if (!idx || !packed) return BTC_ERR_NULL;
+    const int bits = btc_index_bits(Kc);
+    if (bits == 0 || N < 1 || Kb < 1) return BTC_ERR_SHAPE;
+    if (reinterpret_cast<uintptr_t>(packed) % 16) return BTC_ERR_ALIGN;
+    const int pw = (int)(btc_index_packed_row_bytes(Kb, Kc) / 4);
+    const size_t total = (size_t)N * pw, grid = (total + 255) / 256;
+    if (grid > 0x7fffffffull) return BTC_ERR_SHAPE;
+    index_pack_kernel<<<(unsigned)grid, 256, 0, (cudaStream_t)stream>>>(idx, N, Kb, bits, pw, static_cast<uint32_t *>(packed));
+    return cuda_check_launch();
+}
+
+extern "C" int btc_index_unpack(const void *packed, int N, int Kb, int Kc, uint16_t *idx, void *stream)
+{
+    if (!idx || !packed) return BTC_ERR_NULL;
+    const int bits = btc_index_bits(Kc);
+    if (bits == 0 || N < 1 || Kb < 1) return BTC_ERR_SHAPE;
+    if (reinterpret_cast<uintptr_t>(packed) % 16) return BTC_ERR_ALIGN;
+    const int pw = (int)(btc_index_packed_row_bytes(Kb, Kc) / 4);
+    const size_t total = (size_t)N * Kb, grid = (total + 255) / 256;
+    if (grid > 0x7fffffffull) return BTC_ERR_SHAPE;
+    index_unpack_kernel<<<(unsigned)grid, 256, 0, (cudaStream_t)stream>>>(static_cast<const uint32_t *>(packed), N, Kb, bits, pw, idx);
     return cuda_check_launch();
 }

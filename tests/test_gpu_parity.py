@@ -457,3 +457,50 @@ print("index check ok")
     root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
     r = subprocess.run([sys.executable, "-c", code], cwd=root, env=env, capture_output=True, text=True, timeout=600)
     assert r.returncode == 0 and "index check ok" in r.stdout, r.stdout + r.stderr
+
+
+# ------------------------------------------------------------------ dense-packed indices (Section 4.3 index width)
+
+@pytest.mark.parametrize("Kc,N,Kb", [(2, 5, 16), (256, 33, 24), (4096, 300, 64), (8192, 129, 688), (7132, 17, 40), (21619, 64, 8),
+                                     (65536, 9, 16)])
+def test_index_pack_and_unpack_bit_exact(Kc, N, Kb):
+    """btc_index_pack / btc_index_unpack against the oracle's bit-by-bit packing: every byte, padding included."""
+    idx = wl.make_indices(N, Kb, Kc, "uniform", 77 + Kc, 1)
+    d = torch.from_numpy(idx.view(np.int16)).cuda()
+    packed = btc.index_pack(d, Kc)
+    bits = oracle.index_bits(Kc)
+    assert btc.index_bits(Kc) == bits and packed.shape[1] == oracle.packed_row_bytes(Kb, bits)
+    assert np.array_equal(packed.cpu().numpy(), oracle.pack_indices(idx, bits))
+    back = btc.index_unpack(packed, Kb, Kc)
+    assert np.array_equal(back.cpu().numpy().view(np.uint16), idx)
+
+
+@pytest.mark.parametrize("N,K,v,Kc,M,mu", [(300, 2048, 16, 4096, 1, False), (129, 4096, 16, 8192, 2, True), (1000, 11008, 16, 8192, 1, False),
+                                           (257, 1152, 16, 7132, 8, False), (77, 1152, 12, 4096, 4, True), (64, 512, 8, 4096, 1, False)])
+def test_linear_on_packed_indices_matches_oracle_and_unpacked(N, K, v, Kc, M, mu):
+    """The decode kernel reading 12- / 13-bit rows: every output against the oracle, and bit-identical to the same kernel
+    reading the uint16 containers (same lookups, same arithmetic)."""
+    L = wl.make_layer(_spec(N, K, v, Kc, with_mu=mu, outlier_frac=0.01), M, seed=N + K + M)
+    d = to_device(L)
+    packed = btc.index_pack(d["idx"], Kc)
+    y = btc.linear_gemv_packed(d["x"], packed, d["Cp"], d["alpha"], v, Kc, mu=d["mu"])
+    y16 = btc.GemvBatch([dict(x=d["x"], idx=d["idx"], C_packed=d["Cp"], alpha=d["alpha"], mu=d["mu"], v=v, Kc=Kc)]).run()[0]
+    torch.cuda.synchronize()
+    rel, fwd = errors(y, oracle_y(L), L)
+    assert rel <= TOL_GEMV and fwd <= TOL_GEMV, (rel, fwd)
+    assert torch.equal(y, y16)
+    assert btc.device_status() == 0
+
+
+def test_fused_decode_step_on_packed_indices_full_size():
+    """The seven full-size layers of config 2 as ONE launch over 13-bit index rows (M = 1): every output against the oracle."""
+    cfg = wl.CONFIGS[2]
+    Ls = [wl.make_layer(s, 1, cfg["seed"], i) for i, s in enumerate(cfg["layers"])]
+    ds = [to_device(L) for L in Ls]
+    outs = btc.GemvBatch([dict(x=d["x"], idx=btc.index_pack(d["idx"], L.spec.Kc), idx_bits=13, C_packed=d["Cp"], alpha=d["alpha"],
+                               v=L.spec.v, Kc=L.spec.Kc) for L, d in zip(Ls, ds)]).run()
+    torch.cuda.synchronize()
+    for L, y in zip(Ls, outs):
+        rel, fwd = errors(y, oracle_y(L), L)
+        assert rel <= TOL_GEMV and fwd <= TOL_GEMV, (L.spec, rel, fwd)
+    assert btc.device_status() == 0
