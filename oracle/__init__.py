@@ -120,6 +120,27 @@ def linear(x_f64, idx, C_pm1, alpha, mu=None, return_B: bool = False):
     return (y, B) if return_B else y
 
 
+def linear_terms(x_f64, N: int, terms) -> np.ndarray:
+    """y = x * W^T for a weight that is a SUM of codebook-binary terms, each covering a column range:
+        W^[n, k] = sum over terms t with k0_t <= k < k0_t + K_t of ( alpha_t[n] * B^_t[n, k - k0_t] + mu_t[n] ).
+    This is what a binariser with several scale groups per row emits (Eq. 1-2 applied per group of columns after the
+    columns are ordered by group: the split-point groups of Section 5's ablation) and what a residual binarisation of
+    salient columns emits (two terms over the same range, W ~ alpha_1 B_1 + alpha_2 B_2, Section 3).
+    terms: iterable of (k0, idx [N, K_t/v], C_pm1 [Kc, v], alpha [N], mu [N] or None).  Dense fp64 weight, then the naive
+    triple loop."""
+    x = np.ascontiguousarray(x_f64, dtype=np.float64)
+    M, K = x.shape
+    W = np.zeros((N, K), dtype=np.float64)
+    for (k0, idx, C_pm1, alpha, mu) in terms:
+        Wt = dense_weight(idx, C_pm1, alpha, mu)
+        if Wt.shape[0] != N or k0 < 0 or k0 + Wt.shape[1] > K:
+            raise ValueError("term outside the layer")
+        W[:, k0:k0 + Wt.shape[1]] += Wt
+    y = np.empty((M, N), dtype=np.float64)
+    _load().btc_oracle_matmul_nt(_p(x), _p(np.ascontiguousarray(W)), M, N, K, _p(y))
+    return y
+
+
 def lut_linear(x_f64, idx, C_pm1, alpha, mu=None, seg: int = 4) -> np.ndarray:
     """Same result through the paper's Stage-I / Stage-II lookup tables."""
     idx, C, al, m = _common(idx, C_pm1, alpha, mu)

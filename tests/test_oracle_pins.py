@@ -462,3 +462,44 @@ def test_index_packing_size_is_the_papers_storage_count():
         oracle.pack_indices(np.array([[4096]], dtype=np.uint16), 12)
     with pytest.raises(ValueError):
         oracle.pack_indices(np.zeros((1, 9), dtype=np.uint16), 12, pitch=13)
+
+
+# ------------------------------------------------------------------ several scale groups per row / residual terms
+
+def test_linear_terms_reduces_to_linear_and_adds_up():
+    """One term over all columns IS the plain layer; column groups with their own (alpha, mu) equal the sum of the plain
+    layer on each column slice; two terms over the same columns (residual binarisation) equal the sum of two layers;
+    and a brute-force element-by-element evaluation agrees."""
+    rng = np.random.default_rng(11)
+    N, K, v, Kc, M = 9, 96, 8, 21, 3
+    x = rng.standard_normal((M, K))
+    C = rng.choice(np.array([-1, 1], dtype=np.int8), size=(Kc, v))
+    idx = rng.integers(0, Kc, size=(N, K // v)).astype(np.uint16)
+    al = np.abs(rng.standard_normal(N)) * 0.02
+    mu = rng.standard_normal(N) * 0.002
+    one = oracle.linear_terms(x, N, [(0, idx, C, al, mu)])
+    assert np.allclose(one, oracle.linear(x, idx, C, al, mu), rtol=1e-13, atol=1e-15)
+    # three column groups (bounds in blocks), each with its own scales
+    bounds = [0, 4, 9, 12]
+    als = [np.abs(rng.standard_normal(N)) * 0.02 for _ in range(3)]
+    mus = [rng.standard_normal(N) * 0.002 for _ in range(3)]
+    terms = [(bounds[g] * v, idx[:, bounds[g]:bounds[g + 1]], C, als[g], mus[g]) for g in range(3)]
+    y = oracle.linear_terms(x, N, terms)
+    want = sum(oracle.linear(x[:, bounds[g] * v:bounds[g + 1] * v], idx[:, bounds[g]:bounds[g + 1]], C, als[g], mus[g]) for g in range(3))
+    assert np.allclose(y, want, rtol=1e-12, atol=1e-14)
+    # brute force, element by element
+    brute = np.zeros((M, N))
+    for m in range(M):
+        for n in range(N):
+            for k in range(K):
+                g = next(i for i in range(3) if bounds[i] * v <= k < bounds[i + 1] * v)
+                brute[m, n] += x[m, k] * (als[g][n] * C[idx[n, k // v], k % v] + mus[g][n])
+    assert np.allclose(y, brute, rtol=1e-12, atol=1e-14)
+    # residual: a second binary term over the first group's columns, with its own codebook and indices
+    C2 = rng.choice(np.array([-1, 1], dtype=np.int8), size=(5, v))
+    idx2 = rng.integers(0, 5, size=(N, 4)).astype(np.uint16)
+    al2 = np.abs(rng.standard_normal(N)) * 0.005
+    yr = oracle.linear_terms(x, N, terms + [(0, idx2, C2, al2, None)])
+    assert np.allclose(yr, y + oracle.linear(x[:, :4 * v], idx2, C2, al2), rtol=1e-12, atol=1e-14)
+    with pytest.raises(ValueError):
+        oracle.linear_terms(x, N, [(K - 8, idx, C, al, mu)])
