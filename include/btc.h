@@ -191,8 +191,27 @@ typedef struct {
     int x_dtype, y_dtype;
     int M, N, K, v, Kc;
     int idx_bits;          /* 0 or 16: uint16 containers; else btc_index_bits(Kc): dense-packed rows (see below) */
+    int x_stride;          /* elements from one row of x to the next; 0 = K.  A multiple of 8 (see btc_linear_gemv_sum) */
+    int idx_stride;        /* elements from one row of idx to the next; 0 = K/v.  A multiple of 8; uint16 containers only */
 } btc_linear_problem;
 BTC_API int btc_linear_gemv_batch(const btc_linear_problem *problems, int count, void *stream);
+
+/* ---- a layer whose weight is a SUM of codebook-binary terms (decode path, M <= 8) -----------------
+ *     y[m, n] = sum_t ( alpha_t[n] * sum_j <x[m, k0_t + j*v : k0_t + (j+1)*v], C_t[idx_t[n, j]]>  +  mu_t[n] * sum_k x[m, k0_t + k] )
+ * Two things the binariser of Section 3 emits have this form.  (1) Several scale groups per row: the non-salient
+ * columns are split by split points into groups with their own (alpha, mu) (Eq. 1-2 per group; the split-point
+ * ablation of Section 5) -- with the columns ordered by group, each group is a term over a column range.  (2) The
+ * residual binarisation of salient columns, W ~ alpha_1 B_1 + alpha_2 B_2: two terms over the same range.  The paper
+ * does not say how group membership is stored at inference; taken here: contiguous column ranges (a fixed column
+ * order is free: it folds into the activation transform).
+ * Each term is a btc_linear_problem whose x points at column k0_t of the activations (x_stride = the full K, in
+ * elements, when M > 1) and whose idx is either its own [N, K_t/v] matrix or a column range of a wider one
+ * (idx_stride).  k0_t, x_stride and idx_stride are multiples of 8 (16-byte alignment).  Every term names the same y,
+ * M and N; with more than one term y is fp32.  The terms run as `count` launches in order on `stream`: the first
+ * writes y, the others add to it (deterministic).  No transform argument.
+ * Errors: as btc_linear_gemv_batch; BTC_ERR_UNSUPPORTED when a term is outside what the decode kernel covers
+ * (v a multiple of 4 up to 20, K_t/v a multiple of 8). */
+BTC_API int btc_linear_gemv_sum(const btc_linear_problem *terms, int count, void *stream);
 
 /* ---- dense-packed indices ------------------------------------------------------------------
  * The paper's storage count gives an index ceil(log2 c) bits ("v*c + ceil(log2 c) * mn/v", Section 4.3): 12 bits for

@@ -22,7 +22,7 @@ EXPORTS = (
     "btc_codebook_pack", "btc_codebook_pack_host", "btc_linear_workspace_bytes", "btc_linear_gemv",
     "btc_linear_gemm", "btc_linear_gemv_batch", "btc_linear_gemm_static_scratch", "btc_decode_pm1", "btc_validate_indices", "btc_bits_per_weight", "btc_device_status", "btc_device_status_reset", "btc_selftest_bounded_wait",
     "btc_codebook_kmeans_workspace_bytes", "btc_codebook_kmeans",
-    "btc_index_bits", "btc_index_packed_row_bytes", "btc_index_pack", "btc_index_unpack", "btc_linear_gemv_packed",
+    "btc_index_bits", "btc_index_packed_row_bytes", "btc_index_pack", "btc_index_unpack", "btc_linear_gemv_packed", "btc_linear_gemv_sum",
 )
 
 
@@ -36,7 +36,7 @@ class BtcLinearProblem(ctypes.Structure):
                 ("alpha", ctypes.c_void_p), ("mu", ctypes.c_void_p), ("y", ctypes.c_void_p),
                 ("x_dtype", ctypes.c_int), ("y_dtype", ctypes.c_int),
                 ("M", ctypes.c_int), ("N", ctypes.c_int), ("K", ctypes.c_int), ("v", ctypes.c_int), ("Kc", ctypes.c_int),
-                ("idx_bits", ctypes.c_int)]
+                ("idx_bits", ctypes.c_int), ("x_stride", ctypes.c_int), ("idx_stride", ctypes.c_int)]
 
 
 class BtcError(RuntimeError):
@@ -70,6 +70,7 @@ def _load() -> ctypes.CDLL:
     L.btc_linear_gemv.argtypes = lin
     L.btc_linear_gemm.argtypes = lin
     L.btc_linear_gemv_batch.argtypes = [ctypes.POINTER(BtcLinearProblem), ci, vp]
+    L.btc_linear_gemv_sum.argtypes = [ctypes.POINTER(BtcLinearProblem), ci, vp]
     L.btc_linear_gemm_static_scratch.argtypes = lin[:14] + [vp]
     L.btc_decode_pm1.argtypes = [vp, vp, ci, ci, ci, ci, vp, vp]
     L.btc_validate_indices.argtypes = [vp, sz, ci, vp, vp]
@@ -235,7 +236,7 @@ class GemvBatch:
             if out is None:
                 out = torch.empty((M, N), dtype=torch.float32, device=x.device)
             arr[i] = BtcLinearProblem(x.data_ptr(), idx.data_ptr(), Cp.data_ptr(), alpha.data_ptr(), _ptr(mu),
-                                      out.data_ptr(), _DT[x.dtype], _DT[out.dtype], M, N, K, v, Kc, bits)
+                                      out.data_ptr(), _DT[x.dtype], _DT[out.dtype], M, N, K, v, Kc, bits, 0, 0)
             self.layers.append((x, idx, Cp, alpha, mu, out))          # keeps the tensors alive
         self._arr = arr
         self.outs = [t[5] for t in self.layers]
@@ -273,6 +274,35 @@ def linear_gemm_static_scratch(x, idx, C_packed, alpha, v, Kc, mu=None, out=None
                                             M, N, K, v, Kc, _stream())
     if st:
         raise BtcError(st, "btc_linear_gemm_static_scratch")
+    return out
+
+
+def linear_gemv_sum(x, terms, N: int, out=None):
+    """btc_linear_gemv_sum: y = sum of codebook-binary terms.  x: [M, K] activations; terms: list of dicts with k0 (first
+    column of the term), idx (16-bit [N, K_t/v], may be a column-range view of a wider matrix), C_packed, alpha, v, Kc
+    and optionally mu.  Returns fp32 [M, N]."""
+    _dev(x, "x")
+    M, K = x.shape
+    if out is None:
+        out = torch.empty((M, N), dtype=torch.float32, device=x.device)
+    arr = (BtcLinearProblem * len(terms))()
+    keep = []
+    for i, T in enumerate(terms):
+        idx, Cp, alpha, mu = T["idx"], T["C_packed"], T["alpha"], T.get("mu")
+        v, Kc, k0 = int(T["v"]), int(T["Kc"]), int(T["k0"])
+        if idx.dim() != 2 or idx.shape[0] != N or idx.stride(1) != 1 or idx.element_size() != 2:
+            raise ValueError("idx must be 16-bit [N, K_t/v] with unit column stride")
+        Kt = idx.shape[1] * v
+        if k0 < 0 or k0 + Kt > K or alpha.numel() != N:
+            raise ValueError("term outside the layer")
+        xt = x[:, k0:k0 + Kt]
+        arr[i] = BtcLinearProblem(xt.data_ptr(), idx.data_ptr(), Cp.data_ptr(), alpha.data_ptr(), _ptr(mu), out.data_ptr(),
+                                  _DT[x.dtype], _DT[out.dtype], M, N, Kt, v, Kc, 0,
+                                  0 if Kt == K else K, 0 if idx.stride(0) == idx.shape[1] else idx.stride(0))
+        keep.append((xt, idx, Cp, alpha, mu))
+    st = lib.btc_linear_gemv_sum(arr, len(terms), _stream())
+    if st:
+        raise BtcError(st, "btc_linear_gemv_sum")
     return out
 
 

@@ -146,7 +146,29 @@ extern "C" int btc_linear_gemm(const void *x, int x_dtype, const uint16_t *idx, 
                       workspace, workspace_bytes, stream);
 }
 
+namespace btc {
+static int run_batch(const btc_linear_problem *problems, int count, void *stream, int accumulate_from, int max_group);
+}
+
 extern "C" int btc_linear_gemv_batch(const btc_linear_problem *problems, int count, void *stream)
+{
+    return btc::run_batch(problems, count, stream, 0, IM_MAXP);
+}
+
+extern "C" int btc_linear_gemv_sum(const btc_linear_problem *terms, int count, void *stream)
+{
+    if (!terms) return BTC_ERR_NULL;
+    if (count < 1) return BTC_ERR_SHAPE;
+    for (int i = 1; i < count; ++i)
+        if (terms[i].y != terms[0].y || terms[i].M != terms[0].M || terms[i].N != terms[0].N || terms[i].y_dtype != terms[0].y_dtype)
+            return BTC_ERR_SHAPE;
+    if (count > 1 && terms[0].y_dtype != BTC_F32) return BTC_ERR_UNSUPPORTED;
+    // one launch per term, in order on the stream: the first writes y, every later one adds to it
+    return btc::run_batch(terms, count, stream, 1, 1);
+}
+
+// accumulate_from > 0: problems with index >= accumulate_from add to y; max_group: layers per launch
+static int btc::run_batch(const btc_linear_problem *problems, int count, void *stream, int accumulate_from, int max_group)
 {
     if (!problems) return BTC_ERR_NULL;
     if (count < 1) return BTC_ERR_SHAPE;
@@ -156,13 +178,13 @@ extern "C" int btc_linear_gemv_batch(const btc_linear_problem *problems, int cou
     while (i < count) {
         // longest run of layers (at most IM_MAXP) starting at i
         int n = 0;
-        for (; n < IM_MAXP && i + n < count; ++n) {
+        for (; n < max_group && i + n < count; ++n) {
             const btc_linear_problem &p = problems[i + n];
             int rc = validate(p.x, p.x_dtype, static_cast<const uint16_t *>(p.idx), p.C_packed, p.alpha, p.y, p.y_dtype, p.M, p.N, p.K, p.v, p.Kc);
             if (rc != BTC_OK) return rc;
             if (p.mu && !aligned(p.mu, 2)) return BTC_ERR_ALIGN;
             if (p.M > 8) return BTC_ERR_SHAPE;
-            if (debug_check_indices_enabled() && (p.idx_bits == 0 || p.idx_bits == 16)) {
+            if (debug_check_indices_enabled() && (p.idx_bits == 0 || p.idx_bits == 16) && p.idx_stride == 0) {
                 rc = launch_index_check(static_cast<const uint16_t *>(p.idx), (size_t)p.N * (p.K / p.v), p.Kc, s);
                 if (rc != BTC_OK) return rc;
             }
@@ -176,6 +198,7 @@ extern "C" int btc_linear_gemv_batch(const btc_linear_problem *problems, int cou
                 a.idx_pitch = btc_index_packed_row_bytes(p.K / p.v, p.Kc);
             }
             a.x = p.x; a.idx = static_cast<const uint16_t *>(p.idx); a.Cp = p.C_packed;
+            a.x_stride = p.x_stride; a.idx_stride = p.idx_stride; a.accumulate = accumulate_from > 0 && (i + n) >= accumulate_from ? 1 : 0;
             a.alpha = reinterpret_cast<const __half *>(p.alpha);
             a.mu = reinterpret_cast<const __half *>(p.mu);
             a.y = p.y; a.workspace = nullptr; a.workspace_bytes = 0;
@@ -187,7 +210,8 @@ extern "C" int btc_linear_gemv_batch(const btc_linear_problem *problems, int cou
             // some layer of the run is outside the fused kernel: one launch per layer instead
             for (int k = 0; k < n; ++k) {
                 rc = launch_gemv_imma(&group[k], 1, s);
-                if (rc == BTC_ERR_UNSUPPORTED && group[k].idx_bits) return rc;     // only the decode kernel reads dense indices
+                // only the decode kernel reads dense indices, column ranges of wider matrices, or adds to y
+                if (rc == BTC_ERR_UNSUPPORTED && (group[k].idx_bits || group[k].x_stride || group[k].idx_stride || group[k].accumulate)) return rc;
                 if (rc == BTC_ERR_UNSUPPORTED) rc = launch_gemv_decode(group[k], s);
                 if (rc == BTC_ERR_UNSUPPORTED) rc = launch_linear_generic(group[k], s);
                 if (rc != BTC_OK) return rc;
@@ -217,7 +241,7 @@ extern "C" int btc_linear_gemv_packed(const void *x, int x_dtype, const void *id
                                       const void *alpha, const void *mu, void *y, int y_dtype, int M, int N, int K,
                                       int v, int Kc, void *stream)
 {
-    btc_linear_problem p;
+    btc_linear_problem p = {};
     p.x = x; p.idx = idx_packed; p.C_packed = C_packed; p.alpha = alpha; p.mu = mu; p.y = y;
     p.x_dtype = x_dtype; p.y_dtype = y_dtype; p.M = M; p.N = N; p.K = K; p.v = v; p.Kc = Kc;
     p.idx_bits = btc_index_bits(Kc);

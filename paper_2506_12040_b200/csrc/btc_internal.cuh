@@ -23,6 +23,11 @@ struct LinearArgs {
     const void *idx_packed = nullptr;
     size_t idx_pitch = 0;
     int idx_bits = 0;
+    // a term of a sum of layers: x / idx may be column ranges of wider matrices (row strides in elements, 0 = dense),
+    // and the result may be added to y (fp32) instead of overwriting it
+    int x_stride = 0;
+    int idx_stride = 0;
+    int accumulate = 0;
 };
 
 // Records a CUDA error for btc_last_cuda_error() and maps it to BTC_ERR_CUDA.

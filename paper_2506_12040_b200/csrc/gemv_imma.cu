@@ -65,6 +65,8 @@ struct ImProblem {
     const __half *mu;         // may be nullptr
     void *y;
     int M, N, K, v, Kc, Kb;
+    int xs;                   // elements from one row of x to the next (K unless x is a column range of a wider matrix)
+    int acc;                  // 1: add to what y holds (a further term of a sum of layers); y is fp32 then
     int x_dt, y_dt;
     int parts;                // ceil(Kb / part width)
     int groups;               // tiles: ceil(N / 16)
@@ -478,7 +480,7 @@ gemv_imma_kernel(const __grid_constant__ ImBatch batch)
                     // ---- B fragments: lane (g = m, t) reads the activations of row m for its own BPL blocks
                     uint64_t breg[BPL][NCLS];
                     const bool has = wvalid && g < M;
-                    const unsigned char *xrow = reinterpret_cast<const unsigned char *>(P.x) + (size_t)g * K * xsz;
+                    const unsigned char *xrow = reinterpret_cast<const unsigned char *>(P.x) + (size_t)g * P.xs * xsz;
                     // 16-bit activations: all of this lane's loads are issued before anything uses them; with v = 16 a
                     // lane's four blocks are 128 contiguous bytes, read 16 bytes (two classes) at a time
                     uint2 raw[BPL][NCLS];
@@ -673,7 +675,9 @@ gemv_imma_kernel(const __grid_constant__ ImBatch batch)
                             }
                             if (n < P.N) {
                                 const float al = __half2float(__ushort_as_half(areg[q])), mu = __half2float(__ushort_as_half(mreg[q]));
-                                store_from_float(P.y, P.y_dt, (size_t)m * P.N + n, al * (2.0f * dot1 - sx) + mu * sx);
+                                float yv = al * (2.0f * dot1 - sx) + mu * sx;
+                                if (P.acc) yv += reinterpret_cast<const float *>(P.y)[(size_t)m * P.N + n];
+                                store_from_float(P.y, P.y_dt, (size_t)m * P.N + n, yv);
                             }
                         }
                     }
@@ -769,12 +773,12 @@ gemv_imma_kernel(const __grid_constant__ ImBatch batch)
                     }
 #pragma unroll 1
                     for (int m = 0; m < M; ++m) {
-                        const unsigned char *xrow = reinterpret_cast<const unsigned char *>(P.x) + (size_t)m * K * xsz;
+                        const unsigned char *xrow = reinterpret_cast<const unsigned char *>(P.x) + (size_t)m * P.xs * xsz;
                         float inv;
                         int xs = 0;
                         uint4 nxt0 = make_uint4(0u, 0u, 0u, 0u), nxt1 = nxt0;
                         if (pf16 && pin && m + 1 < M) {
-                            const uint4 *src = reinterpret_cast<const uint4 *>(reinterpret_cast<const uint16_t *>(P.x) + (size_t)(m + 1) * K + pk0);
+                            const uint4 *src = reinterpret_cast<const uint4 *>(reinterpret_cast<const uint16_t *>(P.x) + (size_t)(m + 1) * P.xs + pk0);
                             nxt0 = __ldg(src);
                             nxt1 = __ldg(src + 1);
                         }
@@ -1054,7 +1058,9 @@ gemv_imma_kernel(const __grid_constant__ ImBatch batch)
                             if (n < P.N) {
                                 const float al = __half2float(__ushort_as_half(areg[q])), mu = __half2float(__ushort_as_half(mreg[q]));
                                 const float dot = dot1 * unshift2 - sx;         // 2 * sum_{bit=1} x - sum x
-                                store_from_float(P.y, P.y_dt, (size_t)m * P.N + n, al * dot + mu * sx);
+                                float yv = al * dot + mu * sx;
+                                if (P.acc) yv += reinterpret_cast<const float *>(P.y)[(size_t)m * P.N + n];
+                                store_from_float(P.y, P.y_dt, (size_t)m * P.N + n, yv);
                             }
                         }
                     }
@@ -1097,17 +1103,17 @@ static im_encode_fn im_get_encode()
 // maps are kept per host thread, keyed by everything the encoding depends on.
 static bool im_tensor_map(im_encode_fn enc, const void *idx, int Kb, int N, int ib, size_t pitch, int box_words, CUtensorMap *out)
 {
-    struct Entry { const void *idx; int Kb, N, ib, box; CUtensorMap map; };
+    struct Entry { const void *idx; int Kb, N, ib, box; size_t pitch; CUtensorMap map; };
     constexpr int SLOTS = 64;
     thread_local Entry cache[SLOTS];
     thread_local int used = 0, next = 0;
     for (int i = 0; i < used; ++i)
-        if (cache[i].idx == idx && cache[i].Kb == Kb && cache[i].N == N && cache[i].ib == ib && cache[i].box == box_words) { *out = cache[i].map; return true; }
+        if (cache[i].idx == idx && cache[i].Kb == Kb && cache[i].N == N && cache[i].ib == ib && cache[i].box == box_words && cache[i].pitch == pitch) { *out = cache[i].map; return true; }
     const cuuint32_t estr[2] = {1, 1};
     CUtensorMap m;
     if (ib == 0) {
         const cuuint64_t dims[2] = {(cuuint64_t)Kb, (cuuint64_t)N};
-        const cuuint64_t strides[1] = {(cuuint64_t)Kb * 2};
+        const cuuint64_t strides[1] = {(cuuint64_t)pitch};          // bytes from row to row (Kb * 2 unless idx is a column range)
         const cuuint32_t box[2] = {(cuuint32_t)IM_BOX_COLS, 16u};
         if (enc(&m, CU_TENSOR_MAP_DATA_TYPE_UINT16, 2, const_cast<void *>(idx), dims, strides, box, estr,
                 CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -1124,7 +1130,7 @@ static bool im_tensor_map(im_encode_fn enc, const void *idx, int Kb, int N, int 
             return false;
     }
     Entry &e = cache[next];
-    e.idx = idx; e.Kb = Kb; e.N = N; e.ib = ib; e.box = box_words; e.map = m;
+    e.idx = idx; e.Kb = Kb; e.N = N; e.ib = ib; e.box = box_words; e.pitch = pitch; e.map = m;
     next = (next + 1) % SLOTS;
     if (used < SLOTS) ++used;
     *out = m;
@@ -1252,6 +1258,8 @@ int launch_gemv_imma(const LinearArgs *problems, int count, cudaStream_t s)
         // covered: M <= 8, v a multiple of 4 up to 20, K/v a multiple of 8 (16-byte rows for the bulk copies)
         if (a.M < 1 || a.M > 8 || a.v % 4 != 0 || a.v > 20 || a.Kb % 8 != 0 || a.K > (1 << 20)) return BTC_ERR_UNSUPPORTED;
         if (a.x_dt == BTC_F32 && a.K % 8 != 0) return BTC_ERR_UNSUPPORTED;
+        if (a.accumulate && a.y_dt != BTC_F32) return BTC_ERR_UNSUPPORTED;
+        if ((a.x_stride && a.x_stride % 8) || (a.idx_stride && (a.idx_stride % 8 || a.idx_bits))) return BTC_ERR_UNSUPPORTED;
         if (a.M > m_max) m_max = a.M;
         if (a.idx_bits != problems[0].idx_bits) return BTC_ERR_UNSUPPORTED;      // one index format per launch
     }
@@ -1268,11 +1276,13 @@ int launch_gemv_imma(const LinearArgs *problems, int count, cudaStream_t s)
         p.tab = a.Cp + (nm == 0 ? 1 : 2) * Kc4;      // fp16-layout words (fp16 form) or byte-lane words (integer form)
         p.tab16 = reinterpret_cast<const uint16_t *>(a.Cp + 3 * (size_t)Kc4);
         p.M = a.M; p.N = a.N; p.K = a.K; p.v = a.v; p.Kc = a.Kc; p.Kb = a.Kb;
+        p.xs = a.x_stride ? a.x_stride : a.K;
+        p.acc = a.accumulate ? 1 : 0;
         p.x_dt = a.x_dt; p.y_dt = a.y_dt;
         p.parts = (a.Kb + pw - 1) / pw;
         p.groups = (a.N + 15) / 16;
         p.ncls = a.v / 4;
-        if (!im_tensor_map(enc, p.idx, a.Kb, a.N, ib, a.idx_pitch, pw * ib / 32, &b.map[i]))
+        if (!im_tensor_map(enc, p.idx, a.Kb, a.N, ib, ib ? a.idx_pitch : (size_t)(a.idx_stride ? a.idx_stride : a.Kb) * 2, pw * ib / 32, &b.map[i]))
             return BTC_ERR_UNSUPPORTED;                     // shape the tensor map cannot describe: other kernels take it
         // a (tile, part) costs about the same whatever the part's width; rebuilding the activation fragments for a
         // part costs about as much as one and a half of them and is shared by the tiles a CTA walks with that part

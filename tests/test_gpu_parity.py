@@ -504,3 +504,40 @@ def test_fused_decode_step_on_packed_indices_full_size():
         rel, fwd = errors(y, oracle_y(L), L)
         assert rel <= TOL_GEMV and fwd <= TOL_GEMV, (L.spec, rel, fwd)
     assert btc.device_status() == 0
+
+
+# ------------------------------------------------------------------ scale groups per row / residual terms
+
+@pytest.mark.parametrize("M,N,K", [(1, 300, 4096), (2, 129, 2048), (8, 257, 4096)])
+def test_linear_sum_of_terms_groups_and_residual(M, N, K):
+    """Three column groups with their own (alpha, mu) over ONE index matrix (column-range views), plus a residual term
+    with its own codebook and indices over the first group's columns: btc_linear_gemv_sum against the oracle's dense sum."""
+    v, Kc = 16, 4096
+    L = wl.make_layer(_spec(N, K, v, Kc, with_mu=True, outlier_frac=0.01), M, seed=N + K + M)
+    d = to_device(L)
+    Kb = K // v
+    bounds = [0, Kb // 4, Kb // 4 + Kb // 2, Kb]                  # in blocks; multiples of 8
+    assert all(b % 8 == 0 for b in bounds)
+    rng = np.random.default_rng(N)
+    als = [(np.abs(rng.standard_normal(N)) * 0.02).astype(np.float16) for _ in range(3)]
+    mus = [(rng.standard_normal(N) * 0.002).astype(np.float16) for _ in range(3)]
+    L2 = wl.make_layer(_spec(N, bounds[1] * v, v, 300), M, seed=5 + N)       # the residual term's codebook / indices / scale
+    d2 = to_device(L2)
+    al2 = (L2.alpha.astype(np.float32) * 0.25).astype(np.float16)
+    dev = lambda a: torch.from_numpy(a.view(np.int16).copy()).cuda().view(torch.float16)
+    terms = [dict(k0=bounds[g] * v, idx=d["idx"][:, bounds[g]:bounds[g + 1]], C_packed=d["Cp"], alpha=dev(als[g]), mu=dev(mus[g]), v=v, Kc=Kc)
+             for g in range(3)]
+    terms.append(dict(k0=0, idx=d2["idx"], C_packed=d2["Cp"], alpha=dev(al2), v=v, Kc=300))
+    y = btc.linear_gemv_sum(d["x"], terms, N)
+    y2 = btc.linear_gemv_sum(d["x"], terms, N)
+    torch.cuda.synchronize()
+    assert torch.equal(y, y2)
+    oterms = [(bounds[g] * v, L.idx[:, bounds[g]:bounds[g + 1]], L.C_pm1, als[g], mus[g]) for g in range(3)]
+    oterms.append((0, L2.idx, L2.C_pm1, al2, None))
+    ref = oracle.linear_terms(L.x_f64(), N, oterms)
+    err = np.abs(y.double().cpu().numpy() - ref)
+    assert err.max() / np.abs(ref).max() <= TOL_GEMV
+    scale = np.outer(np.abs(L.x_f64()).sum(1), sum(np.abs(a.astype(np.float64)) for a in als) + np.abs(al2.astype(np.float64))
+                     + sum(np.abs(m_.astype(np.float64)) for m_ in mus))
+    assert (err / scale).max() <= TOL_GEMV
+    assert btc.device_status() == 0
