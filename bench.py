@@ -303,7 +303,7 @@ def run_gpu(args):
         details["isolated_step_us_M1"] = float(np.median(iso[2:]))
         del flush
         # ---- per shape, M in {1, 8}, each over its own rotating sets
-        def time_shape(i, M, reps=200):
+        def time_shape(i, M, reps=200, lut=False):
             s = specs[i]
             x = sets[0][i]["x"][:M].contiguous()
             outs = [torch.empty((M, s.N), dtype=torch.float32, device=dev) for _ in range(R)]
@@ -313,9 +313,15 @@ def run_gpu(args):
 
             ws1 = torch.empty(max(256, btc.linear_workspace_bytes(M, s.N, s.K, s.v, s.Kc)), dtype=torch.uint8, device=dev)
 
+            wsl = torch.empty(max(256, int(btc.lib.btc_linear_gemv_lut_workspace_bytes(M, s.N, s.K, s.v, s.Kc))), dtype=torch.uint8,
+                              device=dev) if lut else None
+
             def one(k):
                 d = sets[rr[k % R]][same[(k // R) % len(same)]]
-                btc.linear_gemv(x, d["idx"], d["Cp"], d["alpha"], s.v, s.Kc, out=outs[k % R], workspace=ws1)
+                if lut:      # the paper's two-stage lookup scheme (appendix "Binary codebook LUT-GEMM") on the same layer
+                    btc.linear_gemv_lut(x, d["idx"], d["Cp"], d["alpha"], s.v, s.Kc, out=outs[k % R], workspace=wsl)
+                else:
+                    btc.linear_gemv(x, d["idx"], d["Cp"], d["alpha"], s.v, s.Kc, out=outs[k % R], workspace=ws1)
             stream = torch.cuda.Stream(device=dev)
             with torch.cuda.stream(stream):
                 for k in range(5):
@@ -375,6 +381,7 @@ def run_gpu(args):
             for M in (1, 8):
                 details.setdefault(f"per_shape_M{M}", {})[f"{s.N}x{s.K}"] = time_shape(i, M)
             d1 = details["per_shape_M1"][f"{s.N}x{s.K}"]
+            d1["lut_scheme"] = time_shape(i, 1, lut=True)
             d1["dense_fp16_gemv"] = time_dense_fp16_gemv(i)
             d1["speedup_over_dense_fp16"] = d1["dense_fp16_gemv"]["us"] / d1["us"]
         torch.cuda.nvtx.range_pop()

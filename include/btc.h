@@ -213,6 +213,23 @@ BTC_API int btc_linear_gemv_batch(const btc_linear_problem *problems, int count,
  * (v a multiple of 4 up to 20, K_t/v a multiple of 8). */
 BTC_API int btc_linear_gemv_sum(const btc_linear_problem *terms, int count, void *stream);
 
+/* ---- the paper's own kernel scheme (alternative to btc_linear_gemv) ---------------------------------
+ * Same layer, same arguments (1 <= M <= 8, no transform), computed by the two-stage lookup of the appendix "Binary
+ * codebook LUT-GEMM": Stage I builds, per block of x, the signed sums LUT_{j,p}[s] of its P = v/mu segments (mu = 8
+ * when 8 divides v, else 4) over all 2^mu sign patterns; Stage II builds CBLUT_j[k] = sum_p LUT_{j,p}[key[k,p]] for
+ * every codeword (keys = bit fields of the packed codeword); the product is then one lookup and one add per
+ * (row, block).  Tables sit in shared memory, CBLUT entries in fp16 as the paper packs them (so an output carries an
+ * fp16 rounding per block: about 2^-12 of the block dots' magnitude), row sums in fp32.  K is cut into slices of 8
+ * blocks whose partial sums meet in `workspace` (btc_linear_gemv_lut_workspace_bytes(...) bytes, 16-byte aligned)
+ * and are added in slice order by a second kernel.  Needs v a multiple of 4, K/v a multiple of 8 and 16*Kc bytes of
+ * tables to fit shared memory (Kc up to about 13000); otherwise BTC_ERR_UNSUPPORTED.  Building CBLUT costs Kc*K/v*P
+ * lookups per CTA row chunk whatever N is, so this route pays only when N is much larger than Kc; it is kept for
+ * comparison (see the benchmark) and is not what btc_linear_gemv dispatches to. */
+BTC_API size_t btc_linear_gemv_lut_workspace_bytes(int M, int N, int K, int v, int Kc);
+BTC_API int btc_linear_gemv_lut(const void *x, int x_dtype, const uint16_t *idx, const uint32_t *C_packed,
+                    const void *alpha, const void *mu, void *y, int y_dtype, int M, int N, int K, int v, int Kc,
+                    void *workspace, size_t workspace_bytes, void *stream);
+
 /* ---- dense-packed indices ------------------------------------------------------------------
  * The paper's storage count gives an index ceil(log2 c) bits ("v*c + ceil(log2 c) * mn/v", Section 4.3): 12 bits for
  * 4096 centroids, 13 for 8192 (Table 3a pairs v = 16 with codebooks of that size), which is what makes v = 16 a

@@ -23,6 +23,7 @@ EXPORTS = (
     "btc_linear_gemm", "btc_linear_gemv_batch", "btc_linear_gemm_static_scratch", "btc_decode_pm1", "btc_validate_indices", "btc_bits_per_weight", "btc_device_status", "btc_device_status_reset", "btc_selftest_bounded_wait",
     "btc_codebook_kmeans_workspace_bytes", "btc_codebook_kmeans",
     "btc_index_bits", "btc_index_packed_row_bytes", "btc_index_pack", "btc_index_unpack", "btc_linear_gemv_packed", "btc_linear_gemv_sum",
+    "btc_linear_gemv_lut_workspace_bytes", "btc_linear_gemv_lut",
 )
 
 
@@ -85,6 +86,9 @@ def _load() -> ctypes.CDLL:
     L.btc_index_pack.argtypes = [vp, ci, ci, ci, vp, vp]
     L.btc_index_unpack.argtypes = [vp, ci, ci, ci, vp, vp]
     L.btc_linear_gemv_packed.argtypes = [vp, ci, vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, vp]
+    L.btc_linear_gemv_lut_workspace_bytes.restype = sz
+    L.btc_linear_gemv_lut_workspace_bytes.argtypes = [ci] * 5
+    L.btc_linear_gemv_lut.argtypes = [vp, ci, vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, vp, sz, vp]
     L.btc_bits_per_weight.restype = ctypes.c_double
     L.btc_bits_per_weight.argtypes = [ci] * 7
     return L
@@ -303,6 +307,26 @@ def linear_gemv_sum(x, terms, N: int, out=None):
     st = lib.btc_linear_gemv_sum(arr, len(terms), _stream())
     if st:
         raise BtcError(st, "btc_linear_gemv_sum")
+    return out
+
+
+def linear_gemv_lut(x, idx, C_packed, alpha, v, Kc, mu=None, out=None, workspace=None):
+    """btc_linear_gemv_lut: the layer through the paper's two-stage lookup tables (M <= 8)."""
+    for t, n in ((x, "x"), (idx, "idx"), (C_packed, "C_packed"), (alpha, "alpha")):
+        _dev(t, n)
+    M, K = x.shape
+    N, Kb = idx.shape
+    if Kb * v != K or alpha.numel() != N or C_packed.numel() != packed_words(Kc, v):
+        raise ValueError("shape mismatch between x, idx, v, alpha and C_packed")
+    if out is None:
+        out = torch.empty((M, N), dtype=torch.float32, device=x.device)
+    need = int(lib.btc_linear_gemv_lut_workspace_bytes(M, N, K, v, Kc))
+    if workspace is None:
+        workspace = torch.empty(max(need, 256), dtype=torch.uint8, device=x.device)
+    st = lib.btc_linear_gemv_lut(x.data_ptr(), _DT[x.dtype], idx.data_ptr(), C_packed.data_ptr(), alpha.data_ptr(), _ptr(mu),
+                                 out.data_ptr(), _DT[out.dtype], M, N, K, v, Kc, workspace.data_ptr(), workspace.numel(), _stream())
+    if st:
+        raise BtcError(st, "btc_linear_gemv_lut")
     return out
 
 

@@ -65,6 +65,10 @@ int launch_index_check(const uint16_t *idx, size_t count, int Kc, cudaStream_t s
 int index_status_read(int *out);
 int index_status_reset();
 
+// gemv_lut.cu: the paper's two-stage lookup scheme (alternative route, own entry point).
+int launch_gemv_lut(const LinearArgs &a, cudaStream_t s);
+size_t gemv_lut_workspace_bytes(int M, int N, int K, int v);
+
 // transform.cu: x' = x * D * (P1 (x) P2) into xt (same dtype/shape as x).
 int launch_transform(const void *x, int x_dt, const btc_transform &T, void *xt, int M, int K,
                      cudaStream_t s);

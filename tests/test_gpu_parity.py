@@ -541,3 +541,20 @@ def test_linear_sum_of_terms_groups_and_residual(M, N, K):
                      + sum(np.abs(m_.astype(np.float64)) for m_ in mus))
     assert (err / scale).max() <= TOL_GEMV
     assert btc.device_status() == 0
+
+
+# ------------------------------------------------------------------ the paper's two-stage lookup scheme as a kernel
+
+@pytest.mark.parametrize("N,K,v,Kc,M,mu", [(300, 1024, 16, 4096, 1, False), (4096, 4096, 16, 8192, 1, False), (129, 2048, 16, 300, 3, True),
+                                           (513, 640, 20, 5000, 2, True), (64, 768, 12, 777, 8, False), (11008, 4096, 16, 8192, 2, False)])
+def test_lut_scheme_kernel_matches_oracle(N, K, v, Kc, M, mu):
+    """btc_linear_gemv_lut (Stage-I activation tables, Stage-II codebook table in fp16, gather-accumulate) against the
+    oracle's dense product, at the decode tolerance; twice, bit for bit (slices are added in a fixed order)."""
+    L = wl.make_layer(_spec(N, K, v, Kc, with_mu=mu, outlier_frac=0.01), M, seed=N + K + M)
+    d = to_device(L)
+    y = btc.linear_gemv_lut(d["x"], d["idx"], d["Cp"], d["alpha"], v, Kc, mu=d["mu"])
+    y2 = btc.linear_gemv_lut(d["x"], d["idx"], d["Cp"], d["alpha"], v, Kc, mu=d["mu"])
+    torch.cuda.synchronize()
+    rel, fwd = errors(y, oracle_y(L), L)
+    assert rel <= TOL_GEMV and fwd <= TOL_GEMV, (rel, fwd)
+    assert torch.equal(y, y2)
