@@ -477,6 +477,46 @@ def run_gpu(args):
                                               "workspace_bytes": int(wsm.numel())}
         details["gemm_small_M"] = small
 
+        # ---- online activation transform (Section 4.2, X <- X T) in front of the layer: 4096 = 64 x 64, 11008 = 86 x 128
+        def time_transform(li, M, k1, k2, reps=40):
+            s = c4["layers"][li]
+            L = wl.make_layer(s, 1, c4["seed"], li)
+            d = dev_layer(L)
+            dt = torch.float16 if M <= 8 else torch.bfloat16
+            x = torch.randn(M, s.K, device=dev).to(dt)
+            g_ = torch.Generator(device="cpu"); g_.manual_seed(5)
+            P1 = torch.linalg.qr(torch.randn(k1, k1, generator=g_))[0].contiguous().to(dev)
+            P2 = torch.linalg.qr(torch.randn(k2, k2, generator=g_))[0].contiguous().to(dev)
+            sig = torch.randint(0, 2 ** 31 - 1, ((s.K + 31) // 32,), generator=g_, dtype=torch.int32).to(dev)
+            y = torch.empty((M, s.N), dtype=torch.float32, device=dev)
+            wsb = torch.empty(max(256, int(btc.lib.btc_linear_workspace_bytes_ex(M, s.N, s.K, s.v, s.Kc, 1))), dtype=torch.uint8, device=dev)
+            fn = btc.linear_gemv if M <= 8 else btc.linear_gemm
+            res = {}
+            for name, tr in (("layer", None), ("transform_and_layer", (sig, P1, P2))):
+                stream = torch.cuda.Stream(device=dev)
+                with torch.cuda.stream(stream):
+                    for _ in range(3):
+                        fn(x, d["idx"], d["Cp"], d["alpha"], s.v, s.Kc, out=y, workspace=wsb, transform=tr)
+                    stream.synchronize()
+                    g = torch.cuda.CUDAGraph()
+                    with torch.cuda.graph(g, stream=stream):
+                        for _ in range(reps):
+                            fn(x, d["idx"], d["Cp"], d["alpha"], s.v, s.Kc, out=y, workspace=wsb, transform=tr)
+                    g.replay()
+                    stream.synchronize()
+                    e0 = torch.cuda.Event(enable_timing=True)
+                    e1 = torch.cuda.Event(enable_timing=True)
+                    e0.record(stream)
+                    g.replay()
+                    e1.record(stream)
+                    stream.synchronize()
+                res[name + "_us"] = e0.elapsed_time(e1) * 1e3 / reps
+            res["transform_us"] = res["transform_and_layer_us"] - res["layer_us"]
+            res["note"] = "warm L2 (one weight copy): the difference is the transform kernel's share of the pair"
+            return res
+        details["transform"] = {f"M{M}_{c4['layers'][li].N}x{c4['layers'][li].K}": time_transform(li, M, k1, k2)
+                                for (li, k1, k2) in ((0, 64, 64), (2, 86, 128)) for M in (1, 512)}
+
         # ---- configs 1 and 3: single layers at M = 1 (config 3: v = 20, 65536 centroids gathered from L1/L2, Zipf indices)
         def time_single(spec, seed, lid, M, copies=24, reps=96):
             L = wl.make_layer(spec, M, seed, lid)

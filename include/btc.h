@@ -153,6 +153,10 @@ BTC_API int btc_codebook_kmeans(const uint32_t *vecs, size_t n, int v, int Kc, i
  * fails.  Both are asynchronous: a device-side failure shows up at the caller's next sync.
  */
 BTC_API size_t btc_linear_workspace_bytes(int M, int N, int K, int v, int Kc);
+/* The same plus, when has_transform != 0, the room for the transformed activations (a call with T != NULL needs this
+ * much): M*K fp32 values for the decode path (M <= 8, which then reads fp32 activations: no 16-bit rounding of x'),
+ * M*K values in the dtype of x otherwise. */
+BTC_API size_t btc_linear_workspace_bytes_ex(int M, int N, int K, int v, int Kc, int has_transform);
 
 BTC_API int btc_linear_gemv(const void *x, int x_dtype, const uint16_t *idx, const uint32_t *C_packed,
                     const void *alpha, const void *mu, const btc_transform *T, void *y, int y_dtype,

@@ -23,7 +23,7 @@ EXPORTS = (
     "btc_linear_gemm", "btc_linear_gemv_batch", "btc_linear_gemm_static_scratch", "btc_decode_pm1", "btc_validate_indices", "btc_bits_per_weight", "btc_device_status", "btc_device_status_reset", "btc_selftest_bounded_wait",
     "btc_codebook_kmeans_workspace_bytes", "btc_codebook_kmeans",
     "btc_index_bits", "btc_index_packed_row_bytes", "btc_index_pack", "btc_index_unpack", "btc_linear_gemv_packed", "btc_linear_gemv_sum",
-    "btc_linear_gemv_lut_workspace_bytes", "btc_linear_gemv_lut",
+    "btc_linear_gemv_lut_workspace_bytes", "btc_linear_gemv_lut", "btc_linear_workspace_bytes_ex",
 )
 
 
@@ -67,6 +67,8 @@ def _load() -> ctypes.CDLL:
     L.btc_codebook_pack_host.argtypes = [vp, ci, ci, vp]
     L.btc_linear_workspace_bytes.restype = sz
     L.btc_linear_workspace_bytes.argtypes = [ci] * 5
+    L.btc_linear_workspace_bytes_ex.restype = sz
+    L.btc_linear_workspace_bytes_ex.argtypes = [ci] * 6
     lin = [vp, ci, vp, vp, vp, vp, ctypes.POINTER(BtcTransform), vp, ci, ci, ci, ci, ci, ci, vp, sz, vp]
     L.btc_linear_gemv.argtypes = lin
     L.btc_linear_gemm.argtypes = lin
@@ -175,12 +177,10 @@ def _linear(fn, name, x, idx, C_packed, alpha, v, Kc, mu, out, out_dtype, worksp
         if tuple(out.shape) != (M, N):
             raise ValueError("out must be [M, N]")
     tr = None
-    extra = 0
     if transform is not None:
         sig, P1, P2 = transform
         tr = BtcTransform(sig.data_ptr(), P1.data_ptr(), P2.data_ptr(), P1.shape[0], P2.shape[0])
-        extra = (M * K * 2 + 255) // 256 * 256
-    need = linear_workspace_bytes(M, N, K, v, Kc) + extra
+    need = int(lib.btc_linear_workspace_bytes_ex(M, N, K, v, Kc, int(transform is not None)))
     ws_ptr, ws_bytes = None, 0
     if need:
         if workspace is None:

@@ -28,6 +28,13 @@ static int validate(const void *x, int x_dt, const uint16_t *idx, const uint32_t
 
 enum Path { PATH_GEMV, PATH_GEMM };
 
+// Room for the transformed activations at the front of the workspace (fp32 for the decode path, see run_linear).
+static size_t transform_bytes(int M, int K, int v)
+{
+    const bool f32 = M <= 8 && v % 4 == 0 && v <= 20 && (K / v) % 8 == 0 && K % 8 == 0;
+    return (((size_t)M * K * (f32 ? 4 : 2) + 255) / 256) * 256;
+}
+
 static int run_linear(Path path, const void *x, int x_dt, const uint16_t *idx, const uint32_t *Cp,
                       const void *alpha, const void *mu, const btc_transform *T, void *y, int y_dt, int M,
                       int N, int K, int v, int Kc, void *ws, size_t ws_bytes, void *stream)
@@ -40,7 +47,10 @@ static int run_linear(Path path, const void *x, int x_dt, const uint16_t *idx, c
     size_t need = (M <= 8) ? gemv_decode_workspace_bytes(M, N, K, v, Kc) : 0;
     if (gemm_tcgen05_workspace_min(M) > need) need = gemm_tcgen05_workspace_min(M);
     need = (need + 255) / 256 * 256;
-    const size_t xt_bytes = T ? (((size_t)M * K * 2 + 255) / 256) * 256 : 0;
+    // the transformed activations go to the front of the workspace: as fp32 where the decode kernel will read them (it
+    // quantises or rounds the activations itself), else in the dtype of x
+    const bool xt_f32 = T && M <= 8 && v % 4 == 0 && v <= 20 && (K / v) % 8 == 0 && K % 8 == 0;
+    const size_t xt_bytes = T ? transform_bytes(M, K, v) : 0;
     if (need + xt_bytes > 0) {
         if (!ws || ws_bytes < need + xt_bytes) return BTC_ERR_WORKSPACE;
         if (!aligned(ws, 256)) return BTC_ERR_ALIGN;
@@ -64,9 +74,10 @@ static int run_linear(Path path, const void *x, int x_dt, const uint16_t *idx, c
         // scratch follows.
         if (!T->sigma_bits || !T->P1 || !T->P2) return BTC_ERR_NULL;
         if (T->k1 < 1 || T->k2 < 1 || (long long)T->k1 * T->k2 != K) return BTC_ERR_SHAPE;
-        rc = launch_transform(x, x_dt, *T, ws, M, K, s);
+        rc = launch_transform(x, x_dt, *T, ws, xt_f32 ? BTC_F32 : x_dt, M, K, s);
         if (rc != BTC_OK) return rc;
         a.x = ws;
+        if (xt_f32) a.x_dt = BTC_F32;
         a.workspace = static_cast<char *>(ws) + xt_bytes;
         a.workspace_bytes = ws_bytes - xt_bytes;
     }
@@ -76,7 +87,7 @@ static int run_linear(Path path, const void *x, int x_dt, const uint16_t *idx, c
         // the decode kernel (integer form up to two rows of x, fp16 form above); for M = 5..8 with few row tiles and a
         // very long K the tensor-core launch with K split over the SMs, when the workspace has room for its partial
         // sums; the older fp16 kernel and the any-shape kernel take what the first does not cover
-        if (M > 2 && gemm_tcgen05_small_m_pays(M, N, K, v)) rc = launch_gemm_tcgen05(a, s, true);
+        if (M > 2 && a.x_dt != BTC_F32 && gemm_tcgen05_small_m_pays(M, N, K, v)) rc = launch_gemm_tcgen05(a, s, true);
         if (rc == BTC_ERR_UNSUPPORTED) rc = launch_gemv_imma(&a, 1, s);
         if (rc == BTC_ERR_UNSUPPORTED) rc = launch_gemv_decode(a, s);
     }
@@ -126,6 +137,12 @@ extern "C" size_t btc_linear_workspace_bytes(int M, int N, int K, int v, int Kc)
     size_t b = gemm_tcgen05_workspace_bytes(M, N, K, v, Kc);
     size_t w = a > b ? a : b;
     return (w + 255) / 256 * 256;
+}
+
+extern "C" size_t btc_linear_workspace_bytes_ex(int M, int N, int K, int v, int Kc, int has_transform)
+{
+    if (v < 1 || v > 32 || Kc < 1 || Kc > 65536 || M < 1 || N < 1 || K < 1 || K % v) return 0;
+    return btc_linear_workspace_bytes(M, N, K, v, Kc) + (has_transform ? transform_bytes(M, K, v) : 0);
 }
 
 extern "C" int btc_linear_gemv(const void *x, int x_dtype, const uint16_t *idx, const uint32_t *C_packed,

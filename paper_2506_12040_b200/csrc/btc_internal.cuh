@@ -69,8 +69,8 @@ int index_status_reset();
 int launch_gemv_lut(const LinearArgs &a, cudaStream_t s);
 size_t gemv_lut_workspace_bytes(int M, int N, int K, int v);
 
-// transform.cu: x' = x * D * (P1 (x) P2) into xt (same dtype/shape as x).
-int launch_transform(const void *x, int x_dt, const btc_transform &T, void *xt, int M, int K,
+// transform.cu: x' = x * D * (P1 (x) P2) into xt (same shape as x, dtype out_dt).
+int launch_transform(const void *x, int x_dt, const btc_transform &T, void *xt, int out_dt, int M, int K,
                      cudaStream_t s);
 
 // ---- small device helpers ------------------------------------------------------------------

@@ -326,10 +326,11 @@ def test_chained_decode_blocks_with_teacher_forcing(Kc, dist):
 
 # ------------------------------------------------------------------ online activation transform
 
-@pytest.mark.parametrize("path,M,k1,k2", [("gemv", 2, 32, 32), ("gemv", 1, 64, 64), ("gemm", 96, 16, 64), ("gemv", 8, 8, 40)])
+@pytest.mark.parametrize("path,M,k1,k2", [("gemv", 2, 32, 32), ("gemv", 1, 64, 64), ("gemm", 96, 16, 64), ("gemv", 8, 8, 40), ("gemv", 4, 64, 64), ("gemm", 300, 20, 72)])
 def test_online_transform_prologue(path, M, k1, k2):
     """x' = x * diag(sigma) * (P1 kron P2) before the layer (Section 4.2, applied on the fly): against the oracle's dense
-    K x K Kronecker form in fp64.  The kernel rounds x' to the activation dtype, hence the tensor-core tolerance."""
+    K x K Kronecker form in fp64.  On the decode path x' stays fp32 up to the layer kernel, so the decode tolerance holds;
+    on the tensor-core path x' is rounded to the activation dtype, as any activation is there."""
     K = k1 * k2
     v = 16 if K % 16 == 0 else 20
     L = wl.make_layer(_spec(272, K, v, 4096, x_dtype="f16" if path == "gemv" else "bf16"), M, seed=77 + k1)
@@ -348,9 +349,10 @@ def test_online_transform_prologue(path, M, k1, k2):
     xt = oracle.transform(L.x_f64(), sigma, P1.astype(np.float64), P2.astype(np.float64))
     ref = oracle.linear(xt, L.idx, L.C_pm1, L.alpha)
     err = np.abs(y.double().cpu().numpy() - ref)
-    assert err.max() / np.abs(ref).max() <= TOL_GEMM
+    tol = TOL_GEMV if path == "gemv" else TOL_GEMM
+    assert err.max() / np.abs(ref).max() <= tol
     scale = np.outer(np.abs(xt).sum(1), np.abs(L.alpha.astype(np.float64)))
-    assert (err / np.maximum(scale, 1e-300)).max() <= TOL_GEMM
+    assert (err / np.maximum(scale, 1e-300)).max() <= tol
 
 
 # ------------------------------------------------------------------ invariants through the production kernels
