@@ -39,31 +39,36 @@ lut_gemv_kernel(const LutParams p)
     const int r0 = blockIdx.y * p.rows_per_cta, r1 = min(p.N, r0 + p.rows_per_cta);
     const int nseg = 1 << p.mu;
     float *s_lut = reinterpret_cast<float *>(lut_smem);          // [LB][P][2^mu]
-    __half *s_cb = reinterpret_cast<__half *>(lut_smem + (size_t)LUT_LB * p.P * nseg * sizeof(float));   // [LB][Kc]
+    float *s_x = s_lut + (size_t)LUT_LB * p.P * nseg;            // [LB][v] activations of the slice
+    __half *s_cb = reinterpret_cast<__half *>(s_x + LUT_LB * 32);   // [LB][Kc]
     const uint32_t kmask = (uint32_t)nseg - 1u;
 
     for (int m = 0; m < p.M; ++m) {
-        // ---- Stage I: signed sums of every segment for every sign pattern
-        for (int e = tid; e < nb * p.P * nseg; e += LUT_THREADS) {
-            const int s = e & (nseg - 1), jp = e >> p.mu;        // jp = j * P + seg
-            const int j = jp / p.P, seg = jp - j * p.P;
-            const size_t k0 = (size_t)m * p.K + (size_t)(j0 + j) * p.v + (size_t)seg * p.mu;
-            float acc = 0.f;
-            for (int t = 0; t < p.mu; ++t) {
-                const float xv = load_as_float(p.x, p.x_dt, k0 + t);
-                acc += ((s >> t) & 1) ? xv : -xv;
+        // ---- Stage I: signed sums of every segment for every sign pattern (the slice's activations first go to shared
+        //      memory; entry s is built from entry s with its lowest set bit cleared: one add per entry)
+        for (int e = tid; e < nb * p.v; e += LUT_THREADS) s_x[e] = load_as_float(p.x, p.x_dt, (size_t)m * p.K + (size_t)j0 * p.v + e);
+        __syncthreads();
+        for (int jp = tid; jp < nb * p.P; jp += LUT_THREADS) {
+            const float *xs = s_x + (size_t)jp * p.mu;               // (block j, segment seg) = jp: mu consecutive activations
+            float *lut = s_lut + ((size_t)jp << p.mu);
+            float neg = 0.f;
+            for (int t = 0; t < p.mu; ++t) neg -= xs[t];
+            lut[0] = neg;                                            // all signs -1
+            for (int sp = 1; sp < nseg; ++sp) {
+                const int low = __ffs(sp) - 1;                       // lowest set bit: flipping it from -1 to +1 adds 2 x
+                lut[sp] = lut[sp & (sp - 1)] + 2.0f * xs[low];
             }
-            s_lut[e] = acc;
         }
         __syncthreads();
         // ---- Stage II: one entry per (block, codeword), P lookups each, rounded to fp16 as the paper stores it
-        for (int e = tid; e < nb * p.Kc; e += LUT_THREADS) {
-            const int j = e / p.Kc, k = e - j * p.Kc;
+        for (int k = tid; k < p.Kc; k += LUT_THREADS) {
             const uint32_t w = __ldg(p.Cp + k);
-            float acc = 0.f;
-            for (int seg = 0; seg < p.P; ++seg)
-                acc += s_lut[((j * p.P + seg) << p.mu) + ((w >> (seg * p.mu)) & kmask)];
-            s_cb[(size_t)j * p.Kc + k] = __float2half_rn(acc);
+            for (int j = 0; j < nb; ++j) {
+                float acc = 0.f;
+                for (int seg = 0; seg < p.P; ++seg)
+                    acc += s_lut[((j * p.P + seg) << p.mu) + ((w >> (seg * p.mu)) & kmask)];
+                s_cb[(size_t)j * p.Kc + k] = __float2half_rn(acc);
+            }
         }
         __syncthreads();
         // ---- gather: a thread per row, one lookup and one add per block
@@ -130,7 +135,7 @@ int launch_gemv_lut(const LinearArgs &a, cudaStream_t s)
     LutParams p;
     p.mu = (a.v % 8 == 0) ? 8 : 4;
     p.P = a.v / p.mu;
-    const size_t smem = (size_t)LUT_LB * p.P * (1u << p.mu) * sizeof(float) + (size_t)LUT_LB * a.Kc * sizeof(__half);
+    const size_t smem = ((size_t)LUT_LB * p.P * (1u << p.mu) + LUT_LB * 32) * sizeof(float) + (size_t)LUT_LB * a.Kc * sizeof(__half);
     if (smem > 227u * 1024u) return BTC_ERR_UNSUPPORTED;
     const size_t need = gemv_lut_workspace_bytes(a.M, a.N, a.K, a.v);
     if (!a.workspace || a.workspace_bytes < need) return BTC_ERR_WORKSPACE;
