@@ -39,7 +39,7 @@ CONFIG_ID = 2
 # profiles/decode_step_traffic.json, which also holds the SHA-256 of the kernel source it was taken on; when the source
 # has changed since, the figure no longer describes the kernel that is timed and `traffic` is reported as null.
 TRAFFIC_RECORD = os.path.join(ROOT, "profiles", "decode_step_traffic.json")
-KERNEL_SOURCE = os.path.join(ROOT, "paper_2506_12040_b200", "csrc", "gemv_imma.cu")
+KERNEL_SOURCE = os.path.join(ROOT, "paper_2506_12040_b200", "csrc", "gemv_imma_wide.cu")
 
 
 def kernel_source_sha256() -> str:
@@ -710,7 +710,7 @@ def run_gpu(args):
                 "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
                              "frac": achieved / peak, "traffic": traffic, "traffic_note": traffic_note,
                              "peak_source": f"of {peaks['source']}",
-                             "kernel": "gemv_imma_kernel (7 layers per launch)", "bytes_per_launch": bytes_per_launch,
+                             "kernel": "wide::gemv_imma_kernel<4,1,1> (integer form, one CTA per SM; 7 layers per launch)", "bytes_per_launch": bytes_per_launch,
                              "avg_launch_us": avg_launch_s * 1e6,
                              "per_layer_launches": details.get("per_layer_set_M1")},
                 "cpu_baseline": cpu, "details": details}

@@ -88,6 +88,7 @@ static int run_linear(Path path, const void *x, int x_dt, const uint16_t *idx, c
         // very long K the tensor-core launch with K split over the SMs, when the workspace has room for its partial
         // sums; the older fp16 kernel and the any-shape kernel take what the first does not cover
         if (M > 2 && a.x_dt != BTC_F32 && gemm_tcgen05_small_m_pays(M, N, K, v)) rc = launch_gemm_tcgen05(a, s, true);
+        if (rc == BTC_ERR_UNSUPPORTED && M <= 2) rc = launch_gemv_imma_wide(&a, 1, s);     // (plain launches at M <= 2: the faster geometry)
         if (rc == BTC_ERR_UNSUPPORTED) rc = launch_gemv_imma(&a, 1, s);
         if (rc == BTC_ERR_UNSUPPORTED) rc = launch_gemv_decode(a, s);
     }
@@ -222,11 +223,15 @@ static int btc::run_batch(const btc_linear_problem *problems, int count, void *s
             a.x_dt = p.x_dtype; a.y_dt = p.y_dtype;
             a.M = p.M; a.N = p.N; a.K = p.K; a.v = p.v; a.Kc = p.Kc; a.Kb = p.K / p.v;
         }
-        int rc = launch_gemv_imma(group, n, s);
+        // plain launches at M <= 2 take the one-CTA-per-SM geometry (it declines anything else); a sum of terms never does,
+        // so that all its terms share one arithmetic
+        int rc = accumulate_from > 0 ? BTC_ERR_UNSUPPORTED : launch_gemv_imma_wide(group, n, s);
+        if (rc == BTC_ERR_UNSUPPORTED) rc = launch_gemv_imma(group, n, s);
         if (rc == BTC_ERR_UNSUPPORTED) {
             // some layer of the run is outside the fused kernel: one launch per layer instead
             for (int k = 0; k < n; ++k) {
-                rc = launch_gemv_imma(&group[k], 1, s);
+                rc = accumulate_from > 0 ? BTC_ERR_UNSUPPORTED : launch_gemv_imma_wide(&group[k], 1, s);
+                if (rc == BTC_ERR_UNSUPPORTED) rc = launch_gemv_imma(&group[k], 1, s);
                 // only the decode kernel reads dense indices, column ranges of wider matrices, or adds to y
                 if (rc == BTC_ERR_UNSUPPORTED && (group[k].idx_bits || group[k].x_stride || group[k].idx_stride || group[k].accumulate)) return rc;
                 if (rc == BTC_ERR_UNSUPPORTED) rc = launch_gemv_decode(group[k], s);

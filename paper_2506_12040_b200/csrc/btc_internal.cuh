@@ -69,6 +69,11 @@ int index_status_reset();
 int launch_gemv_lut(const LinearArgs &a, cudaStream_t s);
 size_t gemv_lut_workspace_bytes(int M, int N, int K, int v);
 
+// gemv_imma_wide.cu: the integer form for M <= 2 in its one-CTA-per-SM geometry (plain launches only; UNSUPPORTED otherwise).
+int launch_gemv_imma_wide(const LinearArgs *problems, int count, cudaStream_t s);
+int wide_status_read(int *out);
+int wide_status_reset();
+
 // transform.cu: x' = x * D * (P1 (x) P2) into xt (same shape as x, dtype out_dt).
 int launch_transform(const void *x, int x_dt, const btc_transform &T, void *xt, int out_dt, int M, int K,
                      cudaStream_t s);

@@ -756,7 +756,9 @@ extern "C" BTC_API int btc_device_status_reset(void)
     const int zero = 0;
     cudaError_t e = cudaMemcpyToSymbol(btc::g_gemm_status, &zero, sizeof(int));
     if (e != cudaSuccess) return btc::cuda_fail(e);
-    const int rc = btc::index_status_reset();
+    int rc = btc::index_status_reset();
+    if (rc != BTC_OK) return rc;
+    rc = btc::wide_status_reset();
     if (rc != BTC_OK) return rc;
     return btc::imma_status_reset();
 }
@@ -778,7 +780,10 @@ extern "C" BTC_API int btc_device_status(int *status_host)
     int v3 = 0;
     const int rc3 = btc::index_status_read(&v3);
     if (rc3 != BTC_OK) return rc3;
-    *status_host = v ? v : (v2 ? v2 : v3);
+    int v4 = 0;
+    const int rc4 = btc::wide_status_read(&v4);
+    if (rc4 != BTC_OK) return rc4;
+    *status_host = v ? v : (v2 ? v2 : (v4 ? v4 : v3));
     return BTC_OK;
 }
 
