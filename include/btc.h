@@ -31,7 +31,9 @@
  *     mu must be complete in memory before the call is enqueued: they must not be
  *     written by a preceding kernel that itself triggers its dependents early (the
  *     library's own kernels that write them -- btc_codebook_pack,
- *     btc_codebook_kmeans -- do not).  x and y carry no such restriction.
+ *     btc_codebook_kmeans -- do not).  The same holds for the arrays of a
+ *     btc_transform (sigma_bits, P1, P2): the transform kernel stages them before
+ *     its predecessor has finished.  x and y carry no such restriction.
  *   - Ranges: 1 <= v <= 32, K % v == 0, 1 <= Kc <= 65536 (Kc need not be a power
  *     of two), N >= 1, M >= 1.
  *   - Alignment: x, idx, y and C_packed 16-byte aligned; alpha / mu 2-byte.

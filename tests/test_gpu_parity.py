@@ -326,11 +326,14 @@ def test_chained_decode_blocks_with_teacher_forcing(Kc, dist):
 
 # ------------------------------------------------------------------ online activation transform
 
-@pytest.mark.parametrize("path,M,k1,k2", [("gemv", 2, 32, 32), ("gemv", 1, 64, 64), ("gemm", 96, 16, 64), ("gemv", 8, 8, 40), ("gemv", 4, 64, 64), ("gemm", 300, 20, 72)])
+@pytest.mark.parametrize("path,M,k1,k2", [("gemv", 2, 32, 32), ("gemv", 1, 64, 64), ("gemm", 96, 16, 64), ("gemv", 8, 8, 40), ("gemv", 4, 64, 64), ("gemm", 300, 20, 72),
+                                           ("gemm", 200, 64, 64), ("gemm", 130, 48, 96), ("gemm", 64, 100, 32), ("gemm", 70, 40, 48)])
 def test_online_transform_prologue(path, M, k1, k2):
     """x' = x * diag(sigma) * (P1 kron P2) before the layer (Section 4.2, applied on the fly): against the oracle's dense
     K x K Kronecker form in fp64.  On the decode path x' stays fp32 up to the layer kernel, so the decode tolerance holds;
-    on the tensor-core path x' is rounded to the activation dtype, as any activation is there."""
+    on the tensor-core path x' is rounded to the activation dtype, as any activation is there.  From 64 rows on, with k2 a
+    multiple of 16, the two products run on the warp-level tensor cores (tf32): the last four cases, with k1 that is and is
+    not a multiple of 16 and of 8, and k2 on both bank phases."""
     K = k1 * k2
     v = 16 if K % 16 == 0 else 20
     L = wl.make_layer(_spec(272, K, v, 4096, x_dtype="f16" if path == "gemv" else "bf16"), M, seed=77 + k1)
