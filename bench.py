@@ -477,30 +477,30 @@ def run_gpu(args):
                                               "workspace_bytes": int(wsm.numel())}
         details["gemm_small_M"] = small
 
-        # ---- tensor-core path for v = 20 (config 3 shapes): the any-v kernel (both operands through shared memory), M = 512
+        # ---- tensor-core path for v = 20 (config 3 shapes; weights through tensor memory as for v = 16), M = 512 and 2048
         gv = {}
         c3g = wl.CONFIGS[3]
         for li in (0, 4):                                             # 5120 x 5120 and 13824 x 5120
             s = c3g["layers"][li]
             d = dev_layer(wl.make_layer(s, 1, c3g["seed"], li))
-            M = 512
-            xb = torch.from_numpy(wl.make_x(M, s.K, "bf16", c3g["seed"], 16 * li + 7).view(np.int16)).to(dev).view(torch.bfloat16)
-            y = torch.empty((M, s.N), dtype=torch.float32, device=dev)
-            for _ in range(3):
-                btc.linear_gemm(xb, d["idx"], d["Cp"], d["alpha"], s.v, s.Kc, out=y, workspace=ws)
-            ts = []
-            for _ in range(7):
-                flush.zero_()
-                e0 = torch.cuda.Event(enable_timing=True)
-                e1 = torch.cuda.Event(enable_timing=True)
-                e0.record()
-                btc.linear_gemm(xb, d["idx"], d["Cp"], d["alpha"], s.v, s.Kc, out=y, workspace=ws)
-                e1.record()
-                torch.cuda.synchronize()
-                ts.append(e0.elapsed_time(e1) * 1e3)
-            us = float(np.median(ts))
-            gv[f"M{M}_{s.N}x{s.K}"] = {"us": us, "TFLOPs": 2.0 * M * s.N * s.K / us * 1e-6,
-                                       "frac_bf16_peak_measured": 2.0 * M * s.N * s.K / us * 1e-6 / peaks["bf16_tflops"]}
+            for M in (512, 2048):
+                xb = torch.from_numpy(wl.make_x(M, s.K, "bf16", c3g["seed"], 16 * li + 7).view(np.int16)).to(dev).view(torch.bfloat16)
+                y = torch.empty((M, s.N), dtype=torch.float32, device=dev)
+                for _ in range(3):
+                    btc.linear_gemm(xb, d["idx"], d["Cp"], d["alpha"], s.v, s.Kc, out=y, workspace=ws)
+                ts = []
+                for _ in range(7):
+                    flush.zero_()
+                    e0 = torch.cuda.Event(enable_timing=True)
+                    e1 = torch.cuda.Event(enable_timing=True)
+                    e0.record()
+                    btc.linear_gemm(xb, d["idx"], d["Cp"], d["alpha"], s.v, s.Kc, out=y, workspace=ws)
+                    e1.record()
+                    torch.cuda.synchronize()
+                    ts.append(e0.elapsed_time(e1) * 1e3)
+                us = float(np.median(ts))
+                gv[f"M{M}_{s.N}x{s.K}"] = {"us": us, "TFLOPs": 2.0 * M * s.N * s.K / us * 1e-6,
+                                           "frac_bf16_peak_measured": 2.0 * M * s.N * s.K / us * 1e-6 / peaks["bf16_tflops"]}
         details["gemm_v20"] = gv
 
         # ---- online activation transform (Section 4.2, X <- X T) in front of the layer: 4096 = 64 x 64, 11008 = 86 x 128

@@ -314,7 +314,7 @@ __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void *src, uint32_t
                  ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
 }
 
-// ------------------------------------------------------------------------------------ v = 16, weights in tensor memory
+// ------------------------------------------------------------------------------------ v = 16 and v = 20, weights in tensor memory
 // With both operands in shared memory the kernel above is bound by shared-memory bandwidth: per 64-wide k step the
 // tensor core reads the A and B tiles while the decode warps write 16 KB of A and TMA writes the x tile, more than
 // the 128 bytes per clock an SM's shared memory delivers (66 % of the MMA rate at best with 256-row x tiles, 50 % with
@@ -349,13 +349,30 @@ __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.
 
 // SPLIT: the CTAs of a tile share K along grid.z and leave raw partial sums in p.part (a separate instantiation, so
 // that the unsplit kernel carries none of it).
-template <int BM, int STAGES, int KS, bool SPLIT>
+// v = 20: the 64 weights of step S of a super-block are the weight pairs 2 S .. 2 S + 31 of its four blocks (ten pairs each);
+// in the fp16-layout word of a 20-bit codeword pair j sits at bits (2 + j, 18 + j).
+template <int S>
+__device__ __forceinline__ void expand_v20(const uint32_t (&w)[4], uint32_t one2, uint32_t (&regs)[32])
+{
+#pragma unroll
+    for (int i = 0; i < 32; ++i) {
+        const int q = 2 * S + i, c = q / 10, j = q - 10 * c;
+        regs[i] = ((w[c] << (13 - j)) & 0x80008000u) | one2;
+    }
+}
+
+template <int BM, int STAGES, int KS, bool SPLIT, int V>
 __global__ void __launch_bounds__(G2_THREADS, 1)
 gemm_v16t_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_i, const Gemm2Params p, const SplitArgs sp)
 {
     constexpr uint32_t B_BYTES = BM * G_BK * 2;                    // one x tile (64 k); a stage holds KS of them
     constexpr uint32_t STAGE_BYTES = KS * B_BYTES;
     constexpr int ACOLS = 32 * KS;                                 // tensor-memory columns of a stage's A tile
+    // An index tile of 64 blocks covers 64 * V weights = V k steps: 16 for v = 16 (four whole blocks per step); 20 for
+    // v = 20, where a step takes 64 weights out of four consecutive blocks, starting 0, 4, 8, 12 or 16 weights into the
+    // first (five steps = sixteen blocks, then the pattern repeats).
+    constexpr int KPT = V;
+    static_assert(V == 16 || V == 20, "index tiles of 64 blocks and whole k steps");
     // With 128-row x tiles an MMA runs for 64 clk, less than it takes one thread to issue it next to sixteen busy decode
     // warps; then two threads issue (warp 1: even stages into accumulator 0; warp 3: odd stages into accumulator 1 in
     // columns [128, 256)) and the epilogue adds the two accumulators.
@@ -370,7 +387,7 @@ gemm_v16t_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
     // One ring of STAGES stages holds both operands of a k step: the x tile in shared memory and the A tile in tensor
     // memory.  full[s]: the TMA arrival (with its bytes) plus the four decode warps; empty[s]: the MMAs' commit.
     // bars: [0,S) full, [S,2S) empty, accum, full_i[2], empty_i[2], tab_full
-    static_assert(STAGES % 4 == 0 && STAGES * ACOLS <= 512 - G4_A_COL0 && 16 % KS == 0, "a decode group must meet a stage in consecutive phases");
+    static_assert(STAGES % 4 == 0 && STAGES * ACOLS <= 512 - G4_A_COL0 && KPT % KS == 0, "a decode group must meet a stage in consecutive phases");
     constexpr int NB = 2 * STAGES + 6;
     uint32_t *s_tmem = reinterpret_cast<uint32_t *>(bars + NB);
     volatile int *s_abort = reinterpret_cast<volatile int *>(s_tmem + 1);
@@ -413,11 +430,11 @@ gemm_v16t_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
             }
             for (int ks = 0; ks < NS; ++ks) {
                 const int kt0 = ks * KS;
-                if ((kt0 & 15) == 0) {
-                    const int it = kt0 >> 4, ib = it & 1;
+                if (kt0 % KPT == 0) {
+                    const int it = kt0 / KPT, ib = it & 1;
                     if (it >= 2 && !mbar_wait(bar_empty_i(ib), ((it >> 1) & 1) ^ 1, s_abort)) break;
                     mbar_expect_tx(bar_full_i(ib), G2_IDX_BYTES);
-                    tma_load_2d(smem_u32(s_idx + (size_t)ib * G2_IDX_BYTES), &tmap_i, (kt_first >> 4) * 64 + it * 64, n0, bar_full_i(ib));
+                    tma_load_2d(smem_u32(s_idx + (size_t)ib * G2_IDX_BYTES), &tmap_i, (kt_first / KPT) * 64 + it * 64, n0, bar_full_i(ib));
                 }
                 const int s = ks % STAGES;
                 if (ks >= STAGES && !mbar_wait(bar_empty(s), ((ks / STAGES) & 1) ^ 1, s_abort)) break;
@@ -461,24 +478,38 @@ gemm_v16t_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
         int cur_it = -1;
         for (int ks = grp; ks < NS && ok; ks += 4) {
             const int kt0 = ks * KS;
-            const int it = kt0 >> 4, ib = it & 1;
+            const int it = kt0 / KPT, ib = it & 1;
             if (it != cur_it) {
                 if (!mbar_wait(bar_full_i(ib), (it >> 1) & 1, s_abort)) { ok = false; break; }
                 cur_it = it;
             }
-            // the four indices per k step of this row: columns (kt % 16) * 4 .. + 3 of the index tile (8 bytes each)
+            // the four indices per k step of this row.  v = 16: columns (kt % 16) * 4 .. + 3 of the index tile (8 bytes);
+            // v = 20: step s of super-block q (16 blocks) starts in block 16 q + 3 s
             uint32_t w[KS][4];
+            int spos[KS];
 #pragma unroll
             for (int j = 0; j < KS; ++j) {
-                const int boff = ((kt0 + j) & 15) * 8;
-                const uint2 quad = *reinterpret_cast<const uint2 *>(
-                    s_idx + (size_t)ib * G2_IDX_BYTES + (size_t)r * 128 + ((((boff >> 4) & 7) ^ (r & 7)) << 4) + (boff & 15));
-                w[j][0] = ~(tab_smem ? s_tab[quad.x & 0xffffu] : __ldg(p.tab + (quad.x & 0xffffu)));
-                w[j][1] = ~(tab_smem ? s_tab[quad.x >> 16] : __ldg(p.tab + (quad.x >> 16)));
-                w[j][2] = ~(tab_smem ? s_tab[quad.y & 0xffffu] : __ldg(p.tab + (quad.y & 0xffffu)));
-                w[j][3] = ~(tab_smem ? s_tab[quad.y >> 16] : __ldg(p.tab + (quad.y >> 16)));
+                const int ktl = (kt0 + j) % KPT;
+                const unsigned char *irow_s = s_idx + (size_t)ib * G2_IDX_BYTES + (size_t)r * 128;
+                uint32_t i4[4];
+                if (V == 16) {
+                    const int boff = ktl * 8;
+                    const uint2 quad = *reinterpret_cast<const uint2 *>(irow_s + ((((boff >> 4) & 7) ^ (r & 7)) << 4) + (boff & 15));
+                    i4[0] = quad.x & 0xffffu; i4[1] = quad.x >> 16; i4[2] = quad.y & 0xffffu; i4[3] = quad.y >> 16;
+                    spos[j] = 0;
+                } else {
+                    const int sb = ktl / 5, sp5 = ktl - 5 * sb;
+                    spos[j] = sp5;
+#pragma unroll
+                    for (int b = 0; b < 4; ++b) {
+                        const int boff = (16 * sb + 3 * sp5 + b) * 2;
+                        i4[b] = *reinterpret_cast<const uint16_t *>(irow_s + ((((boff >> 4) & 7) ^ (r & 7)) << 4) + (boff & 15));
+                    }
+                }
+#pragma unroll
+                for (int b = 0; b < 4; ++b) w[j][b] = ~(tab_smem ? s_tab[i4[b]] : __ldg(p.tab + i4[b]));
             }
-            if ((((ks + 4) * KS) >> 4) != it || ks + 4 >= NS) {     // this group's last stage in the index tile
+            if (((ks + 4) * KS) / KPT != it || ks + 4 >= NS) {     // this group's last stage in the index tile
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar_empty_i(ib));
             }
@@ -489,10 +520,20 @@ gemm_v16t_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
             for (int j = 0; j < KS; ++j) {
                 // register i holds the weights 2i, 2i+1 of the k step (K elements 2i, 2i+1 of this row of A)
                 uint32_t regs[32];
+                if (V == 16) {
 #pragma unroll
-                for (int b = 0; b < 4; ++b)
+                    for (int b = 0; b < 4; ++b)
 #pragma unroll
-                    for (int i = 0; i < 8; ++i) regs[8 * b + i] = ((w[j][b] << (11 - i)) & 0x80008000u) | one2;
+                        for (int i = 0; i < 8; ++i) regs[8 * b + i] = ((w[j][b] << (11 - i)) & 0x80008000u) | one2;
+                } else {
+                    switch (spos[j]) {
+                    case 0: expand_v20<0>(w[j], one2, regs); break;
+                    case 1: expand_v20<1>(w[j], one2, regs); break;
+                    case 2: expand_v20<2>(w[j], one2, regs); break;
+                    case 3: expand_v20<3>(w[j], one2, regs); break;
+                    default: expand_v20<4>(w[j], one2, regs); break;
+                    }
+                }
                 tmem_st32(tmem_d + lane_base + G4_A_COL0 + sa * ACOLS + 32 * j, regs);
             }
             tmem_st_wait();
@@ -597,12 +638,12 @@ static int launch_cfg(const CUtensorMap &tm, const GemmParams &p, cudaStream_t s
     return cuda_check_launch();
 }
 
-template <int BM, int STAGES, int KS, bool SPLIT>
+template <int BM, int STAGES, int KS, bool SPLIT, int V = 16>
 static int launch_v16t(const CUtensorMap &tm, const CUtensorMap &ti, const Gemm2Params &p, const SplitArgs &sp, cudaStream_t s)
 {
     const size_t smem = (size_t)STAGES * KS * (BM * G_BK * 2) + 1024 + 2 * G2_IDX_BYTES + ((p.tab_bytes + 15) & ~15) +
                         (2 * STAGES + 6) * 8 + 16;
-    auto kern = gemm_v16t_kernel<BM, STAGES, KS, SPLIT>;
+    auto kern = gemm_v16t_kernel<BM, STAGES, KS, SPLIT, V>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return cuda_fail(e);
     dim3 grid((p.a.N + G_BN - 1) / G_BN, (p.a.M + BM - 1) / BM, SPLIT ? (p.k_tiles + sp.split_tiles - 1) / sp.split_tiles : 1);
@@ -697,8 +738,9 @@ int launch_gemm_tcgen05(const LinearArgs &a, cudaStream_t s, bool small_m)
         if (rc != BTC_OK) return rc;
         p.sumx = sx;
     }
-    if (a.v == 16 && a.Kb % 8 == 0) {
-        // v = 16: index tiles by TMA, table in shared memory when it fits, weights through tensor memory
+    if ((a.v == 16 && a.Kb % 8 == 0) || (a.v == 20 && a.Kb % 16 == 0)) {
+        // v = 16, and v = 20 with K a multiple of 320: index tiles by TMA, table in shared memory when it fits, weights
+        // through tensor memory
         CUtensorMap ti;
         const cuuint64_t idims[2] = {(cuuint64_t)a.Kb, (cuuint64_t)a.N};
         const cuuint64_t istr[1] = {(cuuint64_t)a.Kb * 2};
@@ -716,7 +758,9 @@ int launch_gemm_tcgen05(const LinearArgs &a, cudaStream_t s, bool small_m)
             // few tiles and a long K: split K over the idle SMs when the caller's workspace has room for the partial sums
             SplitArgs sp = {q.k_tiles, nullptr};
             int splits = 1;
-            const int per = splitk_tiles(((a.N + 127) / 128) * ((a.M + BM - 1) / BM), q.k_tiles, &splits);
+            const int per = a.v == 16 ? splitk_tiles(((a.N + 127) / 128) * ((a.M + BM - 1) / BM), q.k_tiles, &splits) : q.k_tiles;
+            if (a.v == 20)                                         // (no K split here: its index tiles are 20 k steps)
+                return (BM == 256) ? launch_v16t<256, 4, 1, false, 20>(tm, ti, q, sp, s) : launch_v16t<128, 4, 2, false, 20>(tm, ti, q, sp, s);
             if (splits > 1) {
                 const size_t off = ((size_t)a.M * sizeof(float) + 255) & ~(size_t)255;   // (row sums of x come first)
                 const size_t need = off + (size_t)splits * a.M * a.N * sizeof(float);

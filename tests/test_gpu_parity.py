@@ -141,6 +141,11 @@ GEMM_SMALL = [
     (130, 640, 20, 65536, 300, "bf16", False),
     (1000, 512, 8, 85, 9, "bf16", True),
     (512, 2048, 16, 7132, 1024, "bf16", False),
+    # v = 20 with K a multiple of 320 (weights through tensor memory): one index tile exactly; a K that ends inside an
+    # index tile with the table in shared memory; 256-row x tiles
+    (300, 1280, 20, 65536, 130, "f16", True),
+    (260, 2240, 20, 5000, 600, "bf16", False),
+    (7680, 640, 20, 4096, 512, "bf16", False),
 ]
 
 
