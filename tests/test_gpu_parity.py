@@ -1,6 +1,8 @@
 """GPU parity: the CUDA path (through the C ABI) against the fp64 CPU oracle, element by element,
 on the same seeded inputs.  Tolerances: decode bit-exact; outputs max-rel-err <= 2e-3 for the
 decode path (fp32 accumulate, M <= 8) and <= 1e-2 for the tensor-core path."""
+from dataclasses import replace
+
 import numpy as np
 import pytest
 import torch
@@ -187,6 +189,25 @@ def test_gemm_parity_benchmark_config_M2048():
             sub = wl.LayerData(spec, len(rows), L.C_pm1, L.idx, L.alpha, L.x_bits[rows].copy(), L.mu)
             rel, fwd = errors(y[torch.from_numpy(rows).cuda()], oracle_y(sub), sub)
         assert rel <= TOL_GEMM and fwd <= TOL_GEMM, (spec, M, rel, fwd)
+    assert btc.device_status() == 0
+
+
+def test_gemm_parity_config3_shapes_v20_M512():
+    """The tensor-core path on the config-3 layers (v = 20, 65536 centroids, Zipf indices; K = 5120 = 16 x 320, so the
+    weights go through tensor memory in the five-phase expansion) at M = 512, bf16 activations as on that path: one row
+    of x out of every 128-row tile plus the first and last rows, all N columns of each, against the oracle."""
+    cfg = wl.CONFIGS[3]
+    M = 512
+    for lid in (0, 4):
+        spec = replace(cfg["layers"][lid], x_dtype="bf16")
+        L = wl.make_layer(spec, M, cfg["seed"], lid)
+        y, _ = run_layer(L, "gemm")
+        assert bool(torch.isfinite(y).all())
+        tiles = np.arange(M // 128)
+        rows = np.unique(np.concatenate([[0, 1, 127, 128, 255, 256, M - 1], tiles * 128 + (tiles * 37 + 11) % 128]))
+        sub = wl.LayerData(spec, len(rows), L.C_pm1, L.idx, L.alpha, L.x_bits[rows].copy(), L.mu)
+        rel, fwd = errors(y[torch.from_numpy(rows).cuda()], oracle_y(sub), sub)
+        assert rel <= TOL_GEMM and fwd <= TOL_GEMM, (spec, rel, fwd)
     assert btc.device_status() == 0
 
 
