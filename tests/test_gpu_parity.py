@@ -384,6 +384,35 @@ def test_online_transform_prologue(path, M, k1, k2):
     assert (err / np.maximum(scale, 1e-300)).max() <= tol
 
 
+def test_online_transform_full_size_M512():
+    """The transform in front of the 4096 x 4096 config-4 layer at M = 512 (K = 64 x 64: the tensor-core form of the
+    transform, then the tensor-core layer kernel), as the benchmark times it: six rows of x spread over the row tiles,
+    all N columns of each, against the oracle's dense Kronecker form followed by the oracle layer."""
+    cfg = wl.CONFIGS[4]
+    spec, M, k1, k2 = cfg["layers"][0], 512, 64, 64
+    L = wl.make_layer(spec, M, cfg["seed"], 0)
+    rng = np.random.default_rng(11)
+    sigma = rng.choice(np.array([-1, 1], dtype=np.int8), size=spec.K)
+    P1 = np.linalg.qr(rng.standard_normal((k1, k1)))[0].astype(np.float32)
+    P2 = np.linalg.qr(rng.standard_normal((k2, k2)))[0].astype(np.float32)
+    bits = np.zeros((spec.K + 31) // 32, dtype=np.uint32)
+    for i in np.nonzero(sigma < 0)[0]:
+        bits[i >> 5] |= np.uint32(1) << np.uint32(i & 31)
+    d = to_device(L)
+    tr = (torch.from_numpy(bits.view(np.int32)).cuda(), torch.from_numpy(P1).cuda(), torch.from_numpy(P2).cuda())
+    y = btc.linear_gemm(d["x"], d["idx"], d["Cp"], d["alpha"], spec.v, spec.Kc, transform=tr)
+    torch.cuda.synchronize()
+    assert bool(torch.isfinite(y).all())
+    rows = np.array([0, 127, 128, 300, 383, M - 1])
+    xt = oracle.transform(L.x_f64()[rows], sigma, P1.astype(np.float64), P2.astype(np.float64))
+    ref = oracle.linear(xt, L.idx, L.C_pm1, L.alpha)
+    err = np.abs(y[torch.from_numpy(rows).cuda()].double().cpu().numpy() - ref)
+    assert err.max() / np.abs(ref).max() <= TOL_GEMM
+    scale = np.outer(np.abs(xt).sum(1), np.abs(L.alpha.astype(np.float64)))
+    assert (err / np.maximum(scale, 1e-300)).max() <= TOL_GEMM
+    assert btc.device_status() == 0
+
+
 # ------------------------------------------------------------------ invariants through the production kernels
 
 @pytest.mark.parametrize("path,M", [("gemv", 1), ("gemv", 6), ("gemm", 72)])
