@@ -35,6 +35,7 @@ import workloads as wl  # noqa: E402
 METRIC = "effective HBM GB/s at M=1 (us/layer and TFLOP/s at M=2048 in details)"
 UNIT = "GB/s"
 CONFIG_ID = 2
+WORKLOAD = "config 2: LLaMA-2-7B decode layer set (7 projections, v=16, Kc=8192), M=1"
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the fused step kernel come from the ncu capture recorded in
 # profiles/decode_step_traffic.json, which also holds the SHA-256 of the kernel source it was taken on; when the source
 # has changed since, the figure no longer describes the kernel that is timed and `traffic` is reported as null.
@@ -153,7 +154,7 @@ def run_reference(args):
     line = {"impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": "config 2: LLaMA-2-7B decode layer set, M=1, 7 projections per step"},
+            "config": {"workload": WORKLOAD},
             "cpu_baseline": {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle",
                              "sample": f"{args.steps} steps, each the first 1/{REF_ROW_FRACTION} of the output rows of the 7 layers "
                                        "(fp64 dense decode + naive matmul)"},
@@ -192,8 +193,12 @@ def run_gpu(args):
     torch.cuda.set_device(local)
     dev = torch.device("cuda", local)
     peaks = measured_peaks()
-    cfg = wl.CONFIGS[CONFIG_ID]
+    cfg = dict(wl.CONFIGS[args.config])
+    if args.seed is not None:
+        cfg["seed"] = args.seed
     specs = cfg["layers"]
+    custom = args.config != CONFIG_ID or args.M != 1 or args.seed is not None
+    HM = args.M                                    # rows of x in the headline step
 
     def dev_layer(L):
         dt = torch.float16 if L.spec.x_dtype == "f16" else torch.bfloat16
@@ -259,10 +264,10 @@ def run_gpu(args):
             torch.cuda.synchronize()
         return sorted(ts)
 
-    # ---- headline: M = 1
-    step1, outs1, xs1 = make_runner(1)
-    bytes_step = sum(algorithmic_bytes(s, 1) for s in specs)
-    torch.cuda.nvtx.range_push("headline: fused decode step, M=1")
+    # ---- headline: M = 1 (unless --M says otherwise)
+    step1, outs1, xs1 = make_runner(HM)
+    bytes_step = sum(algorithmic_bytes(s, HM) for s in specs)
+    torch.cuda.nvtx.range_push(f"headline: fused decode step, M={HM}")
     with ClockSampler(local) as clk:
         replays = time_steps(step1, args.steps, args.warmup)
         # keep the sampler busy for at least a few samples on very short runs
@@ -662,13 +667,13 @@ def run_gpu(args):
         noff = np.cumsum([0] + [s.N for s in specs])
         xh_all = torch.cat([x.reshape(-1) for x in xs1]).cpu().pin_memory()
         xd_all = torch.empty_like(xh_all, device=dev)
-        yd_all = [torch.empty(int(noff[-1]), dtype=torch.float32, device=dev) for _ in range(R)]
-        yh_all = torch.empty(int(noff[-1]), dtype=torch.float32).pin_memory()
+        yd_all = [torch.empty(HM * int(noff[-1]), dtype=torch.float32, device=dev) for _ in range(R)]
+        yh_all = torch.empty(HM * int(noff[-1]), dtype=torch.float32).pin_memory()
         stream = torch.cuda.Stream(device=dev)
         n_e2e = max(20, min(args.steps, 200))
-        e2e_batches = [btc.GemvBatch([dict(x=xd_all[int(koff[i]):int(koff[i + 1])].view(1, s.K), idx=sets[r][i]["idx"], C_packed=sets[r][i]["Cp"],
+        e2e_batches = [btc.GemvBatch([dict(x=xd_all[HM * int(koff[i]):HM * int(koff[i + 1])].view(HM, s.K), idx=sets[r][i]["idx"], C_packed=sets[r][i]["Cp"],
                                            alpha=sets[r][i]["alpha"], v=s.v, Kc=s.Kc,
-                                           out=yd_all[r][int(noff[i]):int(noff[i + 1])].view(1, s.N)) for i, s in enumerate(specs)])
+                                           out=yd_all[r][HM * int(noff[i]):HM * int(noff[i + 1])].view(HM, s.N)) for i, s in enumerate(specs)])
                        for r in range(R)]
 
         def e2e_step(r):
@@ -708,7 +713,7 @@ def run_gpu(args):
     cpu = None
     if rank == 0 and world == 1:
         import oracle
-        layers = [wl.make_layer(s, 1, cfg["seed"], i) for i, s in enumerate(specs)]
+        layers = [wl.make_layer(s, HM, cfg["seed"], i) for i, s in enumerate(specs)]
         xs64 = [L.x_f64() for L in layers]
         oracle.linear(xs64[0], layers[0].idx, layers[0].C_pm1, layers[0].alpha)
         n_rep, t0 = 0, time.perf_counter()
@@ -720,15 +725,22 @@ def run_gpu(args):
                 break
         dt = (time.perf_counter() - t0) / n_rep
         cpu = {"value": bytes_step / dt * 1e-9, "unit": UNIT, "cores": oracle.threads(), "kind": "oracle",
-               "sample": f"{n_rep} full M=1 steps (7 layers each), fp64 dense decode + naive matmul"}
+               "sample": f"{n_rep} full M={HM} steps ({len(specs)} layers each), fp64 dense decode + naive matmul"}
 
     if rank == 0:
         peak = peaks["hbm_gbs"]
         traffic, traffic_note = recorded_traffic()
+        workload = WORKLOAD
+        kernel_name = "wide::gemv_imma_kernel<4,1,1> (integer form, one CTA per SM; 7 layers per launch)"
+        if custom:
+            traffic, traffic_note = None, "no counters were taken for this workload"
+            workload = (f"config {args.config}: {len(specs)} layers, v={specs[0].v}, Kc={specs[0].Kc}, M={HM}, base seed {cfg['seed']}"
+                        " (not the metric's workload: flags --config / --M / --seed)")
+            kernel_name = "decode kernel chosen by btc_linear_gemv_batch for this workload (one launch per step)"
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
                 "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
                 "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-                "config": {"workload": "config 2: LLaMA-2-7B decode layer set (7 projections, v=16, Kc=8192), M=1",
+                "config": {"workload": workload,
                            "cold_l2": f"inputs larger than L2: {R} weight sets x {step_idx_bytes / 1e6:.1f} MB of indices",
                            "timing": "one CUDA graph of all steps replayed 25 times, CUDA events on the launching stream around every replay, median replay",
                            "multi_gpu": "replicas only"},
@@ -736,7 +748,7 @@ def run_gpu(args):
                 "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
                              "frac": achieved / peak, "traffic": traffic, "traffic_note": traffic_note,
                              "peak_source": f"of {peaks['source']}",
-                             "kernel": "wide::gemv_imma_kernel<4,1,1> (integer form, one CTA per SM; 7 layers per launch)", "bytes_per_launch": bytes_per_launch,
+                             "kernel": kernel_name, "bytes_per_launch": bytes_per_launch,
                              "avg_launch_us": avg_launch_s * 1e6,
                              "per_layer_launches": details.get("per_layer_set_M1")},
                 "cpu_baseline": cpu, "details": details}
@@ -753,7 +765,13 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="btc", choices=["btc", "reference"])
     ap.add_argument("--quick", action="store_true", help="headline only (skip per-shape and GEMM details)")
+    ap.add_argument("--config", type=int, default=CONFIG_ID, choices=[1, 2, 3],
+                    help="decode layer set of the headline (2 = the metric's workload; others imply --quick)")
+    ap.add_argument("--M", type=int, default=1, choices=list(range(1, 9)), help="rows of x in the headline step (default 1; others imply --quick)")
+    ap.add_argument("--seed", type=int, default=None, help="base seed of the synthetic inputs (default: the config's own; implies --quick)")
     args = ap.parse_args()
+    if args.config != CONFIG_ID or args.M != 1 or args.seed is not None:
+        args.quick = True
     if args.impl == "reference":
         if int(os.environ.get("RANK", "0")) == 0:
             run_reference(args)
