@@ -72,6 +72,23 @@ def e_step(B_pm1: np.ndarray, C_pm1: np.ndarray) -> np.ndarray:
     return z_u[inverse]
 
 
+def e_step_per_vector(B_pm1: np.ndarray, C_pm1: np.ndarray) -> np.ndarray:
+    """The E-step exactly as Section 4.1 (2) words it, one vector at a time and every vector on its own:
+    z_i = argmin_k ||b_i - c_k||^2, smallest k among equals.  Slow; e_step above must agree with it on every input
+    (identical vectors have identical distances, which is all that e_step's evaluation per distinct vector uses)."""
+    B = np.asarray(B_pm1, dtype=np.int64)
+    C = np.asarray(C_pm1, dtype=np.int64)
+    z = np.empty(B.shape[0], dtype=np.int64)
+    for i in range(B.shape[0]):
+        best, best_d = 0, None
+        for k in range(C.shape[0]):
+            d = int(((B[i] - C[k]) ** 2).sum())
+            if best_d is None or d < best_d:
+                best, best_d = k, d
+        z[i] = best
+    return z
+
+
 def m_step(B_pm1: np.ndarray, z: np.ndarray, C_pm1: np.ndarray) -> np.ndarray:
     C = np.array(C_pm1, dtype=np.int8, copy=True)
     B = np.asarray(B_pm1, dtype=np.int64)

@@ -391,6 +391,19 @@ def test_kmeans_e_step_equals_hamming_argmin_on_packed_words():
         assert ((B[i].astype(int) - C[z[i]].astype(int)) ** 2).sum() == 4 * min(d)
 
 
+def test_kmeans_e_step_per_distinct_vector_equals_the_per_vector_definition():
+    """e_step evaluates every distinct vector once; the definition (Section 4.1 (2)) visits every vector.  Inputs with
+    many repeated vectors, ties between centroids and duplicated centroids: the two must agree everywhere."""
+    from oracle import codebook_kmeans as km
+    rng = np.random.default_rng(16)
+    for v, n, c in ((6, 500, 9), (12, 800, 40), (3, 200, 8)):
+        proto = np.where(rng.random((30, v)) < 0.5, 1, -1).astype(np.int8)
+        B = proto[rng.integers(0, 30, n)]
+        C = np.where(rng.random((c, v)) < 0.5, 1, -1).astype(np.int8)
+        C[c - 1] = C[0]                              # a duplicated centroid: the smaller index must win
+        assert np.array_equal(km.e_step(B, C), km.e_step_per_vector(B, C))
+
+
 def test_kmeans_objective_never_increases_and_few_distinct_vectors_are_kept_exactly():
     from oracle import codebook_kmeans as km
     rng = np.random.default_rng(7)
