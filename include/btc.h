@@ -183,7 +183,9 @@ BTC_API int btc_linear_gemm(const void *x, int x_dtype, const uint16_t *idx, con
  * cover are run by further launches on the same stream, so the call never fails for that reason.
  *   problems  HOST array of `count` descriptors; it is read before the call returns.  Every pointer
  *             inside a descriptor is a DEVICE pointer with the layout, alignment and ranges stated
- *             for btc_linear_gemv; 1 <= M <= 8 for every layer.  No transform argument.
+ *             for btc_linear_gemv; 1 <= M <= 8 for every layer.  No transform argument: transform the shared
+ *             input once with btc_activation_transform.  x_dtype may also be BTC_F32 (what that call hands over)
+ *             for layers with v a multiple of 4 up to 20 and K/v a multiple of 8 (BTC_ERR_UNSUPPORTED otherwise).
  *   The layers must be independent: no y_i may alias an x_j, idx_j or another y_j of the same call.
  * Errors: as btc_linear_gemv; the first failing layer's status is returned and later layers of the
  * list may not have been enqueued.
@@ -203,6 +205,17 @@ typedef struct {
     int idx_stride;        /* elements from one row of idx to the next; 0 = K/v.  A multiple of 8; uint16 containers only */
 } btc_linear_problem;
 BTC_API int btc_linear_gemv_batch(const btc_linear_problem *problems, int count, void *stream);
+
+/* ---- the activation transform on its own ------------------------------------------------------------
+ * xt = x * D * (P1 (x) P2) for M rows (see btc_transform; Section 4.2, X <- X T), for layers that share their
+ * input: in a decode block q/k/v read one transformed activation vector and gate/up another, so the transform runs
+ * once per distinct input and the layers follow as ONE btc_linear_gemv_batch call on xt.  xt_dtype is BTC_F32 (no
+ * 16-bit rounding of x'; btc_linear_gemv_batch accepts such activations, see there) or the dtype of x.  x and xt are
+ * [M, K] row-major, 16-byte aligned, and must not overlap.  Asynchronous on `stream`; no workspace.
+ * Errors: NULL / SHAPE (k1 * k2 != K) / ALIGN / UNSUPPORTED (x not fp16 / bf16; xt neither fp32 nor the dtype of x; or
+ * factors that do not fit shared memory: K above about 40000 for the few-row form). */
+BTC_API int btc_activation_transform(const void *x, int x_dtype, const btc_transform *T, void *xt, int xt_dtype, int M, int K,
+                                     void *stream);
 
 /* ---- a layer whose weight is a SUM of codebook-binary terms (decode path, M <= 8) -----------------
  *     y[m, n] = sum_t ( alpha_t[n] * sum_j <x[m, k0_t + j*v : k0_t + (j+1)*v], C_t[idx_t[n, j]]>  +  mu_t[n] * sum_k x[m, k0_t + k] )

@@ -24,6 +24,7 @@ EXPORTS = (
     "btc_codebook_kmeans_workspace_bytes", "btc_codebook_kmeans",
     "btc_index_bits", "btc_index_packed_row_bytes", "btc_index_pack", "btc_index_unpack", "btc_linear_gemv_packed", "btc_linear_gemv_sum",
     "btc_linear_gemv_lut_workspace_bytes", "btc_linear_gemv_lut", "btc_linear_workspace_bytes_ex",
+    "btc_activation_transform",
 )
 
 
@@ -91,6 +92,7 @@ def _load() -> ctypes.CDLL:
     L.btc_linear_gemv_lut_workspace_bytes.restype = sz
     L.btc_linear_gemv_lut_workspace_bytes.argtypes = [ci] * 5
     L.btc_linear_gemv_lut.argtypes = [vp, ci, vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, vp, sz, vp]
+    L.btc_activation_transform.argtypes = [vp, ci, ctypes.POINTER(BtcTransform), vp, ci, ci, ci, vp]
     L.btc_bits_per_weight.restype = ctypes.c_double
     L.btc_bits_per_weight.argtypes = [ci] * 7
     return L
@@ -233,8 +235,8 @@ class GemvBatch:
                     raise ValueError("idx is not the buffer index_pack wrote for this (K/v, Kc)")
             if Kb * v != K or alpha.numel() != N or Cp.numel() != packed_words(Kc, v):
                 raise ValueError("shape mismatch between x, idx, v, alpha and C_packed")
-            if x.dtype not in (torch.float16, torch.bfloat16) or alpha.dtype != torch.float16:
-                raise ValueError("x must be fp16/bf16, alpha fp16")
+            if x.dtype not in (torch.float16, torch.bfloat16, torch.float32) or alpha.dtype != torch.float16:
+                raise ValueError("x must be fp16/bf16 (or fp32 from activation_transform), alpha fp16")
             mu = L.get("mu")
             out = L.get("out")
             if out is None:
@@ -250,6 +252,23 @@ class GemvBatch:
         if st:
             raise BtcError(st, "btc_linear_gemv_batch")
         return self.outs
+
+
+def activation_transform(x, transform, out_dtype=torch.float32, out=None):
+    """x' = x * diag(sigma) * (P1 kron P2) for the rows of x (fp16 / bf16 [M, K]); transform = (sigma_bits int32
+    [ceil(K/32)], P1 fp32 [k1, k1], P2 fp32 [k2, k2]).  out_dtype: torch.float32 or the dtype of x."""
+    _dev(x, "x")
+    sig, P1, P2 = transform
+    for t, n in ((sig, "sigma_bits"), (P1, "P1"), (P2, "P2")):
+        _dev(t, n)
+    M, K = x.shape
+    if out is None:
+        out = torch.empty((M, K), dtype=out_dtype, device=x.device)
+    T = BtcTransform(sig.data_ptr(), P1.data_ptr(), P2.data_ptr(), P1.shape[0], P2.shape[0])
+    st = lib.btc_activation_transform(x.data_ptr(), _DT[x.dtype], ctypes.byref(T), out.data_ptr(), _DT[out.dtype], M, K, _stream())
+    if st:
+        raise BtcError(st, "btc_activation_transform")
+    return out
 
 
 def linear_gemv_batch(layers):

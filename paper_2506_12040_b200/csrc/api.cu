@@ -198,7 +198,12 @@ static int btc::run_batch(const btc_linear_problem *problems, int count, void *s
         int n = 0;
         for (; n < max_group && i + n < count; ++n) {
             const btc_linear_problem &p = problems[i + n];
-            int rc = validate(p.x, p.x_dtype, static_cast<const uint16_t *>(p.idx), p.C_packed, p.alpha, p.y, p.y_dtype, p.M, p.N, p.K, p.v, p.Kc);
+            // fp32 activations (what btc_activation_transform hands over) are the decode kernel's alone: they are
+            // accepted where that kernel covers the layer
+            const bool x_f32 = p.x_dtype == BTC_F32;
+            if (x_f32 && !(p.v >= 4 && p.v % 4 == 0 && p.v <= 20 && p.K % p.v == 0 && (p.K / p.v) % 8 == 0 && p.K % 8 == 0 && p.M <= 8))
+                return BTC_ERR_UNSUPPORTED;
+            int rc = validate(p.x, x_f32 ? (int)BTC_F16 : p.x_dtype, static_cast<const uint16_t *>(p.idx), p.C_packed, p.alpha, p.y, p.y_dtype, p.M, p.N, p.K, p.v, p.Kc);
             if (rc != BTC_OK) return rc;
             if (p.mu && !aligned(p.mu, 2)) return BTC_ERR_ALIGN;
             if (p.M > 8) return BTC_ERR_SHAPE;
@@ -232,8 +237,9 @@ static int btc::run_batch(const btc_linear_problem *problems, int count, void *s
             for (int k = 0; k < n; ++k) {
                 rc = accumulate_from > 0 ? BTC_ERR_UNSUPPORTED : launch_gemv_imma_wide(&group[k], 1, s);
                 if (rc == BTC_ERR_UNSUPPORTED) rc = launch_gemv_imma(&group[k], 1, s);
-                // only the decode kernel reads dense indices, column ranges of wider matrices, or adds to y
-                if (rc == BTC_ERR_UNSUPPORTED && (group[k].idx_bits || group[k].x_stride || group[k].idx_stride || group[k].accumulate)) return rc;
+                // only the decode kernel reads dense indices, fp32 activations, column ranges of wider matrices, or adds to y
+                if (rc == BTC_ERR_UNSUPPORTED && (group[k].idx_bits || group[k].x_stride || group[k].idx_stride || group[k].accumulate ||
+                                                  group[k].x_dt == BTC_F32)) return rc;
                 if (rc == BTC_ERR_UNSUPPORTED) rc = launch_gemv_decode(group[k], s);
                 if (rc == BTC_ERR_UNSUPPORTED) rc = launch_linear_generic(group[k], s);
                 if (rc != BTC_OK) return rc;
@@ -244,6 +250,17 @@ static int btc::run_batch(const btc_linear_problem *problems, int count, void *s
         i += n;
     }
     return BTC_OK;
+}
+
+extern "C" int btc_activation_transform(const void *x, int x_dtype, const btc_transform *T, void *xt, int xt_dtype, int M, int K,
+                                       void *stream)
+{
+    if (!x || !T || !xt || !T->sigma_bits || !T->P1 || !T->P2) return BTC_ERR_NULL;
+    if (M < 1 || K < 1 || T->k1 < 1 || T->k2 < 1 || (long long)T->k1 * T->k2 != K) return BTC_ERR_SHAPE;
+    if (x_dtype != BTC_F16 && x_dtype != BTC_BF16) return BTC_ERR_UNSUPPORTED;
+    if (xt_dtype != BTC_F32 && xt_dtype != x_dtype) return BTC_ERR_UNSUPPORTED;
+    if (!aligned(x, 16) || !aligned(xt, 16)) return BTC_ERR_ALIGN;
+    return launch_transform(x, x_dtype, *T, xt, xt_dtype, M, K, (cudaStream_t)stream);
 }
 
 extern "C" double btc_bits_per_weight(int N, int K, int v, int Kc, int scale_bits_per_row, int mode,

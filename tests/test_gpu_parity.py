@@ -384,6 +384,44 @@ def test_online_transform_prologue(path, M, k1, k2):
     assert (err / np.maximum(scale, 1e-300)).max() <= tol
 
 
+@pytest.mark.parametrize("M,k1,k2,xdt", [(1, 64, 64, "f16"), (2, 32, 40, "bf16"), (4, 64, 64, "f16")])
+def test_shared_transform_then_fused_layers(M, k1, k2, xdt):
+    """Layers that share their input (q / k / v of a block): btc_activation_transform once, fp32 x' out, then ONE
+    btc_linear_gemv_batch call over the three layers on x'.  x' itself against the oracle's dense Kronecker form (fp32
+    products of fp32 factors: 1e-5 of the row's largest |x'|; rounded to the 16-bit dtype: half an ulp more), every
+    output of every layer against oracle.linear on the oracle's x' at the decode tolerance."""
+    K = k1 * k2
+    Ls = [wl.make_layer(_spec(N, K, 16, 4096, x_dtype=xdt), M, seed=91 + i, layer_id=i) for i, N in enumerate((272, 520, 272))]
+    rng = np.random.default_rng(3 + k1)
+    sigma = rng.choice(np.array([-1, 1], dtype=np.int8), size=K)
+    P1 = np.linalg.qr(rng.standard_normal((k1, k1)))[0].astype(np.float32)
+    P2 = np.linalg.qr(rng.standard_normal((k2, k2)))[0].astype(np.float32)
+    bits = np.zeros((K + 31) // 32, dtype=np.uint32)
+    for i in np.nonzero(sigma < 0)[0]:
+        bits[i >> 5] |= np.uint32(1) << np.uint32(i & 31)
+    tr = (torch.from_numpy(bits.view(np.int32)).cuda(), torch.from_numpy(P1).cuda(), torch.from_numpy(P2).cuda())
+    ds = [to_device(L) for L in Ls]
+    x = ds[0]["x"]                                           # the shared input: layer 0's activations
+    x64 = Ls[0].x_f64()
+    xt_ref = oracle.transform(x64, sigma, P1.astype(np.float64), P2.astype(np.float64))
+    xt = btc.activation_transform(x, tr)
+    xt16 = btc.activation_transform(x, tr, out_dtype=x.dtype)
+    torch.cuda.synchronize()
+    big = np.abs(xt_ref).max(axis=1, keepdims=True)
+    assert (np.abs(xt.double().cpu().numpy() - xt_ref) <= 1e-5 * big).all()
+    ulp = 2.0 ** -11 if xdt == "f16" else 2.0 ** -8
+    assert (np.abs(xt16.double().cpu().numpy() - xt_ref) <= 1e-5 * big + ulp * np.abs(xt_ref)).all()
+    outs = btc.linear_gemv_batch([dict(x=xt, idx=d["idx"], C_packed=d["Cp"], alpha=d["alpha"], v=16, Kc=4096) for d in ds])
+    torch.cuda.synchronize()
+    for L, y in zip(Ls, outs):
+        ref = oracle.linear(xt_ref, L.idx, L.C_pm1, L.alpha)
+        err = np.abs(y.double().cpu().numpy() - ref)
+        assert err.max() / np.abs(ref).max() <= TOL_GEMV
+        scale = np.outer(np.abs(xt_ref).sum(1), np.abs(L.alpha.astype(np.float64)))
+        assert (err / np.maximum(scale, 1e-300)).max() <= TOL_GEMV
+    assert btc.device_status() == 0
+
+
 def test_online_transform_full_size_M512():
     """The transform in front of the 4096 x 4096 config-4 layer at M = 512 (K = 64 x 64: the tensor-core form of the
     transform, then the tensor-core layer kernel), as the benchmark times it: six rows of x spread over the row tiles,
