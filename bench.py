@@ -548,6 +548,49 @@ def run_gpu(args):
         details["transform"] = {f"M{M}_{c4['layers'][li].N}x{c4['layers'][li].K}": time_transform(li, M, k1, k2)
                                 for (li, k1, k2) in ((0, 64, 64), (2, 86, 128)) for M in (1, 512)}
 
+        # ---- the transform shared by the layers that read one input: q / k / v of config 2 at M = 1, one
+        #      btc_activation_transform (fp32 x') and ONE fused launch over the three layers, against the fused launch alone
+        def time_shared_transform(reps=40):
+            g_ = torch.Generator(device="cpu"); g_.manual_seed(6)
+            k1 = k2 = 64
+            P1 = torch.linalg.qr(torch.randn(k1, k1, generator=g_))[0].contiguous().to(dev)
+            P2 = torch.linalg.qr(torch.randn(k2, k2, generator=g_))[0].contiguous().to(dev)
+            sig = torch.randint(0, 2 ** 31 - 1, ((4096 + 31) // 32,), generator=g_, dtype=torch.int32).to(dev)
+            x = xs1[0]
+            xt = torch.empty((1, 4096), dtype=torch.float32, device=dev)
+            outs3 = [torch.empty((1, specs[i].N), dtype=torch.float32, device=dev) for i in range(3)]
+            plain = btc.GemvBatch([dict(x=x, idx=sets[0][i]["idx"], C_packed=sets[0][i]["Cp"], alpha=sets[0][i]["alpha"],
+                                        v=specs[i].v, Kc=specs[i].Kc, out=outs3[i]) for i in range(3)])
+            onxt = btc.GemvBatch([dict(x=xt, idx=sets[0][i]["idx"], C_packed=sets[0][i]["Cp"], alpha=sets[0][i]["alpha"],
+                                       v=specs[i].v, Kc=specs[i].Kc, out=outs3[i]) for i in range(3)])
+
+            def with_t():
+                btc.activation_transform(x, (sig, P1, P2), out=xt)
+                onxt.run()
+            res = {}
+            for name, fn in (("qkv_us", plain.run), ("transform_and_qkv_us", with_t)):
+                stream = torch.cuda.Stream(device=dev)
+                with torch.cuda.stream(stream):
+                    for _ in range(3):
+                        fn()
+                    stream.synchronize()
+                    g = torch.cuda.CUDAGraph()
+                    with torch.cuda.graph(g, stream=stream):
+                        for _ in range(reps):
+                            fn()
+                    g.replay()
+                    stream.synchronize()
+                    e0 = torch.cuda.Event(enable_timing=True)
+                    e1 = torch.cuda.Event(enable_timing=True)
+                    e0.record(stream)
+                    g.replay()
+                    e1.record(stream)
+                    stream.synchronize()
+                res[name] = e0.elapsed_time(e1) * 1e3 / reps
+            res["note"] = "warm L2 (one weight set); the second figure runs the three layers on fp32 activations (two-CTA geometry of the decode kernel)"
+            return res
+        details["transform"]["shared_qkv_M1"] = time_shared_transform()
+
         # ---- configs 1 and 3: single layers at M = 1 (config 3: v = 20, 65536 centroids gathered from L1/L2, Zipf indices)
         def time_single(spec, seed, lid, M, copies=24, reps=96):
             L = wl.make_layer(spec, M, seed, lid)
