@@ -70,6 +70,21 @@ def test_argument_validation_returns_codes():
     assert btc.lib.btc_codebook_pack(0x100, 4, 40, 0x200, None) == 2
     assert btc.lib.btc_decode_pm1(0x100, 0x200, 4, 10, 4, 4, 0x300, None) == 2
     assert btc.lib.btc_validate_indices(None, 4, 4, 0x100, None) == 1
+    # the transform on its own: NULL, factor sizes, dtypes, alignment -- all decided on the host
+    import ctypes
+    from paper_2506_12040_b200.binding import BtcLinearProblem, BtcTransform
+    T = BtcTransform(0x1000, 0x2000, 0x3000, 4, 8)
+    at = btc.lib.btc_activation_transform
+    assert at(None, 0, ctypes.byref(T), 0x5000, 2, 1, 32, None) == 1
+    assert at(0x4000, 0, None, 0x5000, 2, 1, 32, None) == 1
+    assert at(0x4000, 0, ctypes.byref(T), 0x5000, 2, 1, 40, None) == 2      # k1 * k2 != K
+    assert at(0x4000, 2, ctypes.byref(T), 0x5000, 2, 1, 32, None) == 4      # fp32 input
+    assert at(0x4000, 0, ctypes.byref(T), 0x5000, 1, 1, 32, None) == 4      # fp16 in, bf16 out
+    assert at(0x4008, 0, ctypes.byref(T), 0x5000, 2, 1, 32, None) == 3
+    # fp32 activations in a batch call only where the decode kernel covers the layer (v = 10 is not a multiple of 4)
+    P = (BtcLinearProblem * 1)()
+    P[0] = BtcLinearProblem(0x4000, 0x6000, 0x7000, 0x8000, None, 0x9000, 2, 2, 1, 16, 80, 10, 64, 0, 0, 0)
+    assert btc.lib.btc_linear_gemv_batch(P, 1, None) == 4
 
 
 def test_accounting_matches_closed_forms():
