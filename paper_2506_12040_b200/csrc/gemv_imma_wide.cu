@@ -130,6 +130,19 @@ __device__ __forceinline__ void im_mma_u8s8(int (&c)[4], uint32_t a0, uint32_t a
         : "+r"(c[0]), "+r"(c[1]), "+r"(c[2]), "+r"(c[3])
         : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
+// Two 16-bit indices packed in one word -> the shared addresses base + 4 * index of both.
+__device__ __forceinline__ void im_pair_addr(uint32_t pair, uint32_t base, uint32_t &lo, uint32_t &hi) {
+    asm("{\n\t.reg .u16 l, h;\n\t"
+        "mov.b32 {l, h}, %2;\n\t"
+        "mad.wide.u16 %0, l, 4, %3;\n\t"
+        "mad.wide.u16 %1, h, 4, %3;\n\t}"
+        : "=r"(lo), "=r"(hi) : "r"(pair), "r"(base));
+}
+__device__ __forceinline__ uint32_t im_lds32(uint32_t addr) {
+    uint32_t v;
+    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(addr));
+    return v;
+}
 __device__ __forceinline__ void im_named_bar(int id, int threads) {
     asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
 }
@@ -623,21 +636,33 @@ gemv_imma_kernel(const __grid_constant__ ImBatch batch)
 #pragma unroll
                             for (int e4 = 0; e4 < BPL; e4 += 4) {
                                 uint32_t w0[4], w1[4];
+                                if (TAB_MODE == 1) {
+                                    // whole table in shared memory: one multiply-add per index gives its address
+                                    const uint32_t tb = im_smem_u32(s_tab);
 #pragma unroll
-                                for (int e = 0; e < 4; ++e) {
-                                    const uint32_t pa = ia[(e4 + e) >> 1], pb = ib[(e4 + e) >> 1];
-                                    const uint32_t i0 = (e & 1) ? (pa >> 16) : (pa & 0xffffu);
-                                    const uint32_t i1 = (e & 1) ? (pb >> 16) : (pb & 0xffffu);
-                                    if (TAB_MODE == 1) { w0[e] = s_tab[i0]; w1[e] = s_tab[i1]; }
-                                    else if (TAB_MODE == 3) {
-                                        const uint32_t h0 = reinterpret_cast<const uint16_t *>(s_tab)[i0];
-                                        const uint32_t h1 = reinterpret_cast<const uint16_t *>(s_tab)[i1];
-                                        w0[e] = h0 | (h0 << 12); w1[e] = h1 | (h1 << 12);
+                                    for (int ep = 0; ep < 2; ++ep) {
+                                        uint32_t a0, a1, b0, b1;
+                                        im_pair_addr(ia[(e4 >> 1) + ep], tb, a0, a1);
+                                        im_pair_addr(ib[(e4 >> 1) + ep], tb, b0, b1);
+                                        w0[2 * ep] = im_lds32(a0); w0[2 * ep + 1] = im_lds32(a1);
+                                        w1[2 * ep] = im_lds32(b0); w1[2 * ep + 1] = im_lds32(b1);
                                     }
-                                    else if (TAB_MODE == 0) { w0[e] = __ldg(gtab + i0); w1[e] = __ldg(gtab + i1); }
-                                    else {
-                                        w0[e] = i0 < tab_head ? s_tab[i0] : __ldg(gtab + i0);
-                                        w1[e] = i1 < tab_head ? s_tab[i1] : __ldg(gtab + i1);
+                                } else {
+#pragma unroll
+                                    for (int e = 0; e < 4; ++e) {
+                                        const uint32_t pa = ia[(e4 + e) >> 1], pb = ib[(e4 + e) >> 1];
+                                        const uint32_t i0 = (e & 1) ? (pa >> 16) : (pa & 0xffffu);
+                                        const uint32_t i1 = (e & 1) ? (pb >> 16) : (pb & 0xffffu);
+                                        if (TAB_MODE == 3) {
+                                            const uint32_t h0 = reinterpret_cast<const uint16_t *>(s_tab)[i0];
+                                            const uint32_t h1 = reinterpret_cast<const uint16_t *>(s_tab)[i1];
+                                            w0[e] = h0 | (h0 << 12); w1[e] = h1 | (h1 << 12);
+                                        }
+                                        else if (TAB_MODE == 0) { w0[e] = __ldg(gtab + i0); w1[e] = __ldg(gtab + i1); }
+                                        else {
+                                            w0[e] = i0 < tab_head ? s_tab[i0] : __ldg(gtab + i0);
+                                            w1[e] = i1 < tab_head ? s_tab[i1] : __ldg(gtab + i1);
+                                        }
                                     }
                                 }
 #pragma unroll
