@@ -29,64 +29,104 @@ struct LutParams {
     int rows_per_cta, slices;
 };
 
+// TMU / TP: segment length and segments per block as compile-time constants (0: taken from the parameters), so that
+// the table-build loops unroll with immediate offsets.
+template <int TMU, int TP>
 __global__ void __launch_bounds__(LUT_THREADS, 1)
 lut_gemv_kernel(const LutParams p)
 {
+    const int mu = TMU ? TMU : p.mu, P = TP ? TP : p.P;
     extern __shared__ __align__(16) unsigned char lut_smem[];
     const int tid = threadIdx.x;
     const int slice = blockIdx.x, j0 = slice * LUT_LB;
     const int nb = min(LUT_LB, p.Kb - j0);                       // blocks of this slice
     const int r0 = blockIdx.y * p.rows_per_cta, r1 = min(p.N, r0 + p.rows_per_cta);
-    const int nseg = 1 << p.mu;
+    const int nseg = 1 << mu;
     float *s_lut = reinterpret_cast<float *>(lut_smem);          // [LB][P][2^mu]
-    float *s_x = s_lut + (size_t)LUT_LB * p.P * nseg;            // [LB][v] activations of the slice
+    float *s_x = s_lut + (size_t)LUT_LB * P * nseg;            // [LB][v] activations of the slice
     __half *s_cb = reinterpret_cast<__half *>(s_x + LUT_LB * 32);   // [LB][Kc]
     const uint32_t kmask = (uint32_t)nseg - 1u;
 
     for (int m = 0; m < p.M; ++m) {
         // ---- Stage I: signed sums of every segment for every sign pattern (the slice's activations first go to shared
-        //      memory; entry s is built from entry s with its lowest set bit cleared: one add per entry)
+        //      memory; one thread per table entry)
         for (int e = tid; e < nb * p.v; e += LUT_THREADS) s_x[e] = load_as_float(p.x, p.x_dt, (size_t)m * p.K + (size_t)j0 * p.v + e);
         __syncthreads();
-        for (int jp = tid; jp < nb * p.P; jp += LUT_THREADS) {
-            const float *xs = s_x + (size_t)jp * p.mu;               // (block j, segment seg) = jp: mu consecutive activations
-            float *lut = s_lut + ((size_t)jp << p.mu);
-            float neg = 0.f;
-            for (int t = 0; t < p.mu; ++t) neg -= xs[t];
-            lut[0] = neg;                                            // all signs -1
-            for (int sp = 1; sp < nseg; ++sp) {
-                const int low = __ffs(sp) - 1;                       // lowest set bit: flipping it from -1 to +1 adds 2 x
-                lut[sp] = lut[sp & (sp - 1)] + 2.0f * xs[low];
-            }
+        for (int e = tid; e < (nb * P) << mu; e += LUT_THREADS) {
+            // entry sp of the table of (block j, segment seg) = jp: the signed sum of its mu activations (bit t of sp set <=> +)
+            const int jp = e >> mu, sp = e & (nseg - 1);
+            const float *xs = s_x + (size_t)jp * mu;
+            float acc = 0.f;
+            for (int t = 0; t < mu; ++t) acc += ((sp >> t) & 1) ? xs[t] : -xs[t];
+            s_lut[e] = acc;
         }
         __syncthreads();
-        // ---- Stage II: one entry per (block, codeword), P lookups each, rounded to fp16 as the paper stores it
-        for (int k = tid; k < p.Kc; k += LUT_THREADS) {
-            const uint32_t w = __ldg(p.Cp + k);
-            for (int j = 0; j < nb; ++j) {
-                float acc = 0.f;
-                for (int seg = 0; seg < p.P; ++seg)
-                    acc += s_lut[((j * p.P + seg) << p.mu) + ((w >> (seg * p.mu)) & kmask)];
-                s_cb[(size_t)j * p.Kc + k] = __float2half_rn(acc);
+        // ---- Stage II: one entry per (block, codeword), P lookups each, rounded to fp16 as the paper stores it.  The
+        //      codeword words go out eight loads at a time before any is used.
+        for (int k0 = tid; k0 < p.Kc; k0 += 8 * LUT_THREADS) {
+            uint32_t wv[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const int k = k0 + u * LUT_THREADS;
+                wv[u] = k < p.Kc ? __ldg(p.Cp + k) : 0u;
+            }
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const int k = k0 + u * LUT_THREADS;
+                if (k < p.Kc) {
+                    if (TMU && nb == LUT_LB) {
+#pragma unroll
+                        for (int j = 0; j < LUT_LB; ++j) {
+                            float acc = 0.f;
+#pragma unroll
+                            for (int seg = 0; seg < (TP ? TP : 1); ++seg)
+                                acc += s_lut[((j * P + seg) << mu) + ((wv[u] >> (seg * mu)) & kmask)];
+                            s_cb[(size_t)j * p.Kc + k] = __float2half_rn(acc);
+                        }
+                    } else {
+                        for (int j = 0; j < nb; ++j) {
+                            float acc = 0.f;
+                            for (int seg = 0; seg < P; ++seg)
+                                acc += s_lut[((j * P + seg) << mu) + ((wv[u] >> (seg * mu)) & kmask)];
+                            s_cb[(size_t)j * p.Kc + k] = __float2half_rn(acc);
+                        }
+                    }
+                }
             }
         }
         __syncthreads();
         // ---- gather: a thread per row, one lookup and one add per block
-        for (int n = r0 + tid; n < r1; n += LUT_THREADS) {
-            const uint16_t *row = p.idx + (size_t)n * p.Kb + j0;
-            float acc = 0.f;
-            if (nb == LUT_LB) {
-                const uint4 q = __ldg(reinterpret_cast<const uint4 *>(row));     // K/v is a multiple of 8: 16-byte aligned
-                const uint32_t wd[4] = {q.x, q.y, q.z, q.w};
+        if (nb == LUT_LB) {
+            // whole slices: 16 bytes of indices per row (K/v is a multiple of 8: aligned), four rows' loads in flight
+            for (int n0 = r0 + tid; n0 < r1; n0 += 4 * LUT_THREADS) {
+                uint4 q[4];
 #pragma unroll
-                for (int j = 0; j < LUT_LB; ++j) {
-                    const uint32_t i = (j & 1) ? (wd[j >> 1] >> 16) : (wd[j >> 1] & 0xffffu);
-                    acc += __half2float(s_cb[(size_t)j * p.Kc + i]);
+                for (int u = 0; u < 4; ++u) {
+                    const int n = n0 + u * LUT_THREADS;
+                    q[u] = n < r1 ? __ldg(reinterpret_cast<const uint4 *>(p.idx + (size_t)n * p.Kb + j0)) : make_uint4(0u, 0u, 0u, 0u);
                 }
-            } else {
-                for (int j = 0; j < nb; ++j) acc += __half2float(s_cb[(size_t)j * p.Kc + row[j]]);
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const int n = n0 + u * LUT_THREADS;
+                    if (n < r1) {
+                        const uint32_t wd[4] = {q[u].x, q[u].y, q[u].z, q[u].w};
+                        float acc = 0.f;
+#pragma unroll
+                        for (int j = 0; j < LUT_LB; ++j) {
+                            const uint32_t i = (j & 1) ? (wd[j >> 1] >> 16) : (wd[j >> 1] & 0xffffu);
+                            acc += __half2float(s_cb[(size_t)j * p.Kc + i]);
+                        }
+                        p.part[((size_t)slice * p.M + m) * p.N + n] = acc;
+                    }
+                }
             }
-            p.part[((size_t)slice * p.M + m) * p.N + n] = acc;
+        } else {
+            for (int n = r0 + tid; n < r1; n += LUT_THREADS) {
+                const uint16_t *row = p.idx + (size_t)n * p.Kb + j0;
+                float acc = 0.f;
+                for (int j = 0; j < nb; ++j) acc += __half2float(s_cb[(size_t)j * p.Kc + row[j]]);
+                p.part[((size_t)slice * p.M + m) * p.N + n] = acc;
+            }
         }
         __syncthreads();
     }
@@ -142,16 +182,20 @@ int launch_gemv_lut(const LinearArgs &a, cudaStream_t s)
     p.x = a.x; p.idx = a.idx; p.Cp = a.Cp; p.part = reinterpret_cast<float *>(a.workspace);
     p.M = a.M; p.N = a.N; p.K = a.K; p.v = a.v; p.Kc = a.Kc; p.Kb = a.Kb; p.x_dt = a.x_dt;
     p.slices = (a.Kb + LUT_LB - 1) / LUT_LB;
-    // row chunks: enough CTAs to fill the SMs once, no more (every CTA of a K-slice rebuilds that slice's tables)
+    // row chunks: as many CTAs as fit the SMs in one round, no more (every CTA of a K-slice rebuilds that slice's tables)
     int dev = 0, sms = 148;
     if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    int chunks = (sms + p.slices - 1) / p.slices;
+    int chunks = sms / p.slices;                 // (rounded down: a second round of CTAs would cost a whole table build)
     if (chunks < 1) chunks = 1;
     p.rows_per_cta = (a.N + chunks - 1) / chunks;
     chunks = (a.N + p.rows_per_cta - 1) / p.rows_per_cta;
-    cudaError_t e = cudaFuncSetAttribute(lut_gemv_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    void (*kern)(const LutParams) = lut_gemv_kernel<0, 0>;
+    if (p.mu == 8 && p.P == 2) kern = lut_gemv_kernel<8, 2>;          // v = 16
+    else if (p.mu == 8 && p.P == 1) kern = lut_gemv_kernel<8, 1>;     // v = 8
+    else if (p.mu == 4 && p.P == 5) kern = lut_gemv_kernel<4, 5>;     // v = 20
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return cuda_fail(e);
-    lut_gemv_kernel<<<dim3((unsigned)p.slices, (unsigned)chunks), LUT_THREADS, smem, s>>>(p);
+    kern<<<dim3((unsigned)p.slices, (unsigned)chunks), LUT_THREADS, smem, s>>>(p);
     int rc = cuda_check_launch();
     if (rc != BTC_OK) return rc;
     lut_reduce_kernel<<<dim3((unsigned)((a.N + 255) / 256), (unsigned)a.M), 256, 0, s>>>(p.part, p.slices, a.M, a.N, a.K, a.x, a.x_dt,
