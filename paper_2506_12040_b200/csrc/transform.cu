@@ -165,30 +165,33 @@ __host__ __device__ inline TmLayout tm_layout(int k1, int k2)
     return L;
 }
 
-template <int MT>                           // 16-row tiles of k1
+// MT: 16-row tiles of k1.  TK1 / TK2: the factor sizes as compile-time constants (0: taken from the arguments), so
+// that the pitches and loop bounds of the common shapes fold into immediates.
+template <int MT, int TK1, int TK2>
 __global__ void __launch_bounds__(TM_THREADS, 1)
 transform_mma_kernel(const void *__restrict__ x, int x_dt, const uint32_t *__restrict__ sigma_bits, const float *__restrict__ P1,
-                     const float *__restrict__ P2, int k1, int k2, void *__restrict__ xt, int out_dt, int M)
+                     const float *__restrict__ P2, int k1_arg, int k2_arg, void *__restrict__ xt, int out_dt, int M)
 {
     extern __shared__ __align__(16) uint32_t tm_smem[];
+    const int k1 = TK1 ? TK1 : k1_arg, k2 = TK2 ? TK2 : k2_arg;
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const TmLayout L = tm_layout(k1, k2);
     uint32_t *Xs = tm_smem + L.x_off, *Ys = tm_smem + L.y_off, *P1s = tm_smem + L.p1_off, *P2s = tm_smem + L.p2_off;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
     const int K = k1 * k2;
     // the factors, once per CTA, zero-padded to whole tiles; so are the pad rows of X and Y.  Loads go out in batches
-    // of eight before any of them is used (a loop of load-convert-store would wait for each trip to L2 in turn)
+    // of eight or sixteen before any of them is used (a loop of load-convert-store would wait for each trip to L2 in turn)
     {
         const int n1 = L.k1k * L.p1p, n2 = k2 * L.p2p;
-        for (int i0 = tid; i0 < n1; i0 += 8 * TM_THREADS) {
-            float f[8];
+        for (int i0 = tid; i0 < n1; i0 += 16 * TM_THREADS) {
+            float f[16];
 #pragma unroll
-            for (int u = 0; u < 8; ++u) {
+            for (int u = 0; u < 16; ++u) {
                 const int i = i0 + u * TM_THREADS, a = i / L.p1p, c = i - a * L.p1p;
                 f[u] = (i < n1 && a < k1 && c < k1) ? __ldg(P1 + (size_t)a * k1 + c) : 0.f;
             }
 #pragma unroll
-            for (int u = 0; u < 8; ++u) {
+            for (int u = 0; u < 16; ++u) {
                 const int i = i0 + u * TM_THREADS;
                 if (i < n1) P1s[i] = tm_tf32(f[u]);
             }
@@ -234,44 +237,46 @@ transform_mma_kernel(const void *__restrict__ x, int x_dt, const uint32_t *__res
     asm volatile("griddepcontrol.wait;" ::: "memory");
     const int npairs = k2 / 16;             // pairs of 8-column tiles of d
     constexpr int MG = (MT + 1) / 2;        // a warp's work item: half of the a (or c) tiles x one pair of d tiles
+    // a row of x: eight 16-bit activations per load (k2 is a multiple of 16: they share a row a of X); the loads of the
+    // next row are in flight while this row's products run
+    constexpr int NQ = 8;                   // loads per thread: K <= 8 * NQ * TM_THREADS
+    const int nvec = K / 8;
+    uint4 q[NQ];
+    auto load_row = [&](int m) {
+        const uint4 *src = reinterpret_cast<const uint4 *>(reinterpret_cast<const uint16_t *>(x) + (size_t)m * K);
+#pragma unroll
+        for (int u = 0; u < NQ; ++u) {
+            const int i = tid + u * TM_THREADS;
+            q[u] = i < nvec ? __ldg(src + i) : make_uint4(0u, 0u, 0u, 0u);
+        }
+    };
+    if ((int)blockIdx.x < M) load_row(blockIdx.x);
     for (int m = blockIdx.x; m < M; m += gridDim.x) {
         const size_t row = (size_t)m * K;
         __syncthreads();                    // (the previous row's X and Y are no longer read; pads and factors are in place)
-        {
-            // eight 16-bit activations per load (k2 is a multiple of 16: they share a row a of X), four loads in flight
-            const uint4 *src = reinterpret_cast<const uint4 *>(reinterpret_cast<const uint16_t *>(x) + row);
-            const int nvec = K / 8;
-            for (int i0 = tid; i0 < nvec; i0 += 4 * TM_THREADS) {
-                uint4 q[4];
 #pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    const int i = i0 + u * TM_THREADS;
-                    q[u] = i < nvec ? __ldg(src + i) : make_uint4(0u, 0u, 0u, 0u);
+        for (int u = 0; u < NQ; ++u) {
+            const int i = tid + u * TM_THREADS;
+            if (i < nvec) {
+                const int k = 8 * i, a = k / k2, bcol = k - a * k2;
+                const uint32_t sg = __ldg(sigma_bits + (k >> 5)) >> (k & 31);
+                const uint32_t w[4] = {q[u].x, q[u].y, q[u].z, q[u].w};
+                uint32_t o[8];
+#pragma unroll
+                for (int h = 0; h < 4; ++h) {
+                    float lo, hi;
+                    if (x_dt == BTC_F16) { const float2 f = __half22float2(*reinterpret_cast<const __half2 *>(&w[h])); lo = f.x; hi = f.y; }
+                    else { lo = __uint_as_float(w[h] << 16); hi = __uint_as_float(w[h] & 0xffff0000u); }
+                    if ((sg >> (2 * h)) & 1u) lo = -lo;
+                    if ((sg >> (2 * h + 1)) & 1u) hi = -hi;
+                    o[2 * h] = tm_tf32(lo); o[2 * h + 1] = tm_tf32(hi);
                 }
-#pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    const int i = i0 + u * TM_THREADS;
-                    if (i < nvec) {
-                        const int k = 8 * i, a = k / k2, bcol = k - a * k2;
-                        const uint32_t sg = __ldg(sigma_bits + (k >> 5)) >> (k & 31);
-                        const uint32_t w[4] = {q[u].x, q[u].y, q[u].z, q[u].w};
-                        uint32_t o[8];
-#pragma unroll
-                        for (int h = 0; h < 4; ++h) {
-                            float lo, hi;
-                            if (x_dt == BTC_F16) { const float2 f = __half22float2(*reinterpret_cast<const __half2 *>(&w[h])); lo = f.x; hi = f.y; }
-                            else { lo = __uint_as_float(w[h] << 16); hi = __uint_as_float(w[h] & 0xffff0000u); }
-                            if ((sg >> (2 * h)) & 1u) lo = -lo;
-                            if ((sg >> (2 * h + 1)) & 1u) hi = -hi;
-                            o[2 * h] = tm_tf32(lo); o[2 * h + 1] = tm_tf32(hi);
-                        }
-                        uint4 *dst = reinterpret_cast<uint4 *>(Xs + (size_t)a * L.xp + bcol);
-                        dst[0] = make_uint4(o[0], o[1], o[2], o[3]);
-                        dst[1] = make_uint4(o[4], o[5], o[6], o[7]);
-                    }
-                }
+                uint4 *dst = reinterpret_cast<uint4 *>(Xs + (size_t)a * L.xp + bcol);
+                dst[0] = make_uint4(o[0], o[1], o[2], o[3]);
+                dst[1] = make_uint4(o[4], o[5], o[6], o[7]);
             }
         }
+        if (m + (int)gridDim.x < M) load_row(m + gridDim.x);
         __syncthreads();
         // ---- Y[a][d] = sum_b X[a][b] P2[b][d]
         for (int item = warp; item < 2 * npairs; item += TM_WARPS) {
@@ -358,10 +363,10 @@ transform_mma_kernel(const void *__restrict__ x, int x_dt, const uint32_t *__res
     }
 }
 
-template <int MT>
+template <int MT, int TK1 = 0, int TK2 = 0>
 static int launch_transform_mma(const void *x, int x_dt, const btc_transform &T, void *xt, int out_dt, int M, size_t smem, cudaStream_t s)
 {
-    auto kern = transform_mma_kernel<MT>;
+    auto kern = transform_mma_kernel<MT, TK1, TK2>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return cuda_fail(e);
     int dev = 0, sms = 148;
@@ -384,10 +389,13 @@ int launch_transform(const void *x, int x_dt, const btc_transform &T, void *xt, 
 {
     if ((long long)T.k1 * T.k2 != K) return BTC_ERR_SHAPE;
     // many rows: the tensor-core form, when the factors fit shared memory beside one row (k2 a multiple of 16)
-    if (M >= 64 && x_dt != BTC_F32 && T.k2 % 16 == 0 && T.k1 <= 128) {
+    if (M >= 64 && x_dt != BTC_F32 && T.k2 % 16 == 0 && T.k1 <= 128 && K <= 8 * 8 * TM_THREADS) {
         const size_t bytes = tm_layout(T.k1, T.k2).words * sizeof(uint32_t);
         if (bytes <= 227u * 1024u) {
             const int mt = (T.k1 + 15) / 16;
+            // the factor shapes of the LLaMA-2-7B widths (4096 = 64 x 64, 11008 = 86 x 128) have instantiations of their own
+            if (T.k1 == 64 && T.k2 == 64) return launch_transform_mma<4, 64, 64>(x, x_dt, T, xt, out_dt, M, bytes, s);
+            if (T.k1 == 86 && T.k2 == 128) return launch_transform_mma<6, 86, 128>(x, x_dt, T, xt, out_dt, M, bytes, s);
             switch (mt) {
             case 1: return launch_transform_mma<1>(x, x_dt, T, xt, out_dt, M, bytes, s);
             case 2: return launch_transform_mma<2>(x, x_dt, T, xt, out_dt, M, bytes, s);
