@@ -422,6 +422,39 @@ def test_shared_transform_then_fused_layers(M, k1, k2, xdt):
     assert btc.device_status() == 0
 
 
+@pytest.mark.parametrize("M,k1,k2,xdt", [(96, 48, 96, "f16"), (64, 86, 128, "bf16"), (130, 64, 64, "bf16")])
+def test_activation_transform_many_rows(M, k1, k2, xdt):
+    """btc_activation_transform from 64 rows on (the tf32 tensor-core form; 86 x 128 and 64 x 64 are the shapes with
+    compile-time sizes) against the oracle's dense Kronecker form, on sampled rows where K is large: fp32 output within
+    2^-9 of the row's largest |x'| (two tf32 roundings per product term, random signs), 16-bit output half an ulp more."""
+    K = k1 * k2
+    rng = np.random.default_rng(9 + k1)
+    x_bits = wl.make_x(M, K, xdt, 4242, 3)
+    x64 = (x_bits.view(np.float16).astype(np.float64) if xdt == "f16"
+           else wl.bf16_bits_to_f32(x_bits).astype(np.float64)).reshape(M, K)
+    sigma = rng.choice(np.array([-1, 1], dtype=np.int8), size=K)
+    P1 = np.linalg.qr(rng.standard_normal((k1, k1)))[0].astype(np.float32)
+    P2 = np.linalg.qr(rng.standard_normal((k2, k2)))[0].astype(np.float32)
+    bits = np.zeros((K + 31) // 32, dtype=np.uint32)
+    for i in np.nonzero(sigma < 0)[0]:
+        bits[i >> 5] |= np.uint32(1) << np.uint32(i & 31)
+    tr = (torch.from_numpy(bits.view(np.int32)).cuda(), torch.from_numpy(P1).cuda(), torch.from_numpy(P2).cuda())
+    dt = torch.float16 if xdt == "f16" else torch.bfloat16
+    x = torch.from_numpy(x_bits.view(np.int16).reshape(M, K).copy()).cuda().view(dt)
+    xt = btc.activation_transform(x, tr)
+    xt16 = btc.activation_transform(x, tr, out_dtype=dt)
+    torch.cuda.synchronize()
+    rows = np.arange(M) if K <= 4608 else np.array([0, 1, M // 2, M - 1])
+    ref = oracle.transform(x64[rows], sigma, P1.astype(np.float64), P2.astype(np.float64))
+    big = np.abs(ref).max(axis=1, keepdims=True)
+    got = xt[torch.from_numpy(rows).cuda()].double().cpu().numpy()
+    assert (np.abs(got - ref) <= 2.0 ** -9 * big).all(), float((np.abs(got - ref) / big).max())
+    got16 = xt16[torch.from_numpy(rows).cuda()].double().cpu().numpy()
+    ulp = 2.0 ** -11 if xdt == "f16" else 2.0 ** -8
+    assert (np.abs(got16 - ref) <= 2.0 ** -9 * big + ulp * np.abs(ref)).all()
+    assert btc.device_status() == 0
+
+
 def test_online_transform_full_size_M512():
     """The transform in front of the 4096 x 4096 config-4 layer at M = 512 (K = 64 x 64: the tensor-core form of the
     transform, then the tensor-core layer kernel), as the benchmark times it: six rows of x spread over the row tiles,
