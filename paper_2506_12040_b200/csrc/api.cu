@@ -84,10 +84,14 @@ static int run_linear(Path path, const void *x, int x_dt, const uint16_t *idx, c
 
     rc = BTC_ERR_UNSUPPORTED;
     if (path == PATH_GEMV || M <= 8) {
-        // the decode kernel (integer form up to two rows of x, fp16 form above); for M = 5..8 with few row tiles and a
+        // the decode kernel (integer form up to two rows of x, fp16 form above; the older fp16 kernel where the table
+        // does not fit shared memory); for M = 5..8 with few row tiles and a
         // very long K the tensor-core launch with K split over the SMs, when the workspace has room for its partial
         // sums; the older fp16 kernel and the any-shape kernel take what the first does not cover
         if (M > 2 && a.x_dt != BTC_F32 && gemm_tcgen05_small_m_pays(M, N, K, v)) rc = launch_gemm_tcgen05(a, s, true);
+        // M = 3..8 with a codeword table too large for shared memory (65536 centroids): the older fp16 kernel, which
+        // gathers the whole table from L1/L2, is the faster one (measured 13.8 against 19.6 us for 5120 x 5120, v = 20, M = 4)
+        if (rc == BTC_ERR_UNSUPPORTED && M > 2 && (size_t)Kc * 4 > 96u * 1024u && a.x_dt != BTC_F32) rc = launch_gemv_decode(a, s);
         if (rc == BTC_ERR_UNSUPPORTED && M <= 2) rc = launch_gemv_imma_wide(&a, 1, s);     // (plain launches at M <= 2: the faster geometry)
         if (rc == BTC_ERR_UNSUPPORTED) rc = launch_gemv_imma(&a, 1, s);
         if (rc == BTC_ERR_UNSUPPORTED) rc = launch_gemv_decode(a, s);
