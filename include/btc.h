@@ -145,8 +145,8 @@ BTC_API int btc_codebook_kmeans(const uint32_t *vecs, size_t n, int v, int Kc, i
  *   M <= 2: x is quantised per K-slice to a block-fixed-point integer (2^-20 of the slice's largest magnitude
  *   for v = 16), the sums over set bits are exact integer sums on the warp-level int8 MMA, recombined and added
  *   over the slices in fp32.  M = 3..8: masked codeword bits act as fp16 numbers on the warp-level fp16 MMA with
- *   fp32 accumulation (an older kernel of the same arithmetic where the codeword table is too large for shared
- *   memory).  With v = 16, at most 74 tiles of 128 rows and a workspace of the size
+ *   fp32 accumulation (one layer per call runs on an older kernel of the same arithmetic, a CTA per row tile; the
+ *   fused multi-layer launch of btc_linear_gemv_batch on a newer one).  With v = 16, at most 74 tiles of 128 rows and a workspace of the size
  *   btc_linear_workspace_bytes asks for, M = 5..8 at K >= 8192 and M = 6..8 at K >= 4096 go to the tensor-core launch
  *   of btc_linear_gemm with K split over the SMs instead (it is the faster one there).  All stay well inside a
  *   relative error of 2e-3 against the exact product.  Shapes outside what these kernels cover (v not a multiple

@@ -89,9 +89,10 @@ static int run_linear(Path path, const void *x, int x_dt, const uint16_t *idx, c
         // very long K the tensor-core launch with K split over the SMs, when the workspace has room for its partial
         // sums; the older fp16 kernel and the any-shape kernel take what the first does not cover
         if (M > 2 && a.x_dt != BTC_F32 && gemm_tcgen05_small_m_pays(M, N, K, v)) rc = launch_gemm_tcgen05(a, s, true);
-        // M = 3..8 with a codeword table too large for shared memory (65536 centroids): the older fp16 kernel, which
-        // gathers the whole table from L1/L2, is the faster one (measured 13.8 against 19.6 us for 5120 x 5120, v = 20, M = 4)
-        if (rc == BTC_ERR_UNSUPPORTED && M > 2 && (size_t)Kc * 4 > 96u * 1024u && a.x_dt != BTC_F32) rc = launch_gemv_decode(a, s);
+        // M = 3..8, one layer per call: the older fp16 kernel (a CTA per row tile over the whole K) is the faster one --
+        // 8.5 against 10.1 us for 4096 x 4096 at M = 3, 15.8 against 24.6 us for 4096 x 11008, 13.8 against 19.6 us for
+        // 5120 x 5120 with 65536 centroids at M = 4; the newer fp16 form earns its keep in the fused multi-layer launch
+        if (rc == BTC_ERR_UNSUPPORTED && M > 2 && a.x_dt != BTC_F32) rc = launch_gemv_decode(a, s);
         if (rc == BTC_ERR_UNSUPPORTED && M <= 2) rc = launch_gemv_imma_wide(&a, 1, s);     // (plain launches at M <= 2: the faster geometry)
         if (rc == BTC_ERR_UNSUPPORTED) rc = launch_gemv_imma(&a, 1, s);
         if (rc == BTC_ERR_UNSUPPORTED) rc = launch_gemv_decode(a, s);
@@ -235,6 +236,10 @@ static int btc::run_batch(const btc_linear_problem *problems, int count, void *s
         // plain launches at M <= 2 take the one-CTA-per-SM geometry (it declines anything else); a sum of terms never does,
         // so that all its terms share one arithmetic
         int rc = accumulate_from > 0 ? BTC_ERR_UNSUPPORTED : launch_gemv_imma_wide(group, n, s);
+        // a run of one plain layer at M = 3..8: the older fp16 kernel, as in btc_linear_gemv
+        if (rc == BTC_ERR_UNSUPPORTED && n == 1 && accumulate_from == 0 && group[0].M > 2 && group[0].x_dt != BTC_F32 &&
+            !group[0].idx_bits && !group[0].x_stride && !group[0].idx_stride)
+            rc = launch_gemv_decode(group[0], s);
         if (rc == BTC_ERR_UNSUPPORTED) rc = launch_gemv_imma(group, n, s);
         if (rc == BTC_ERR_UNSUPPORTED) {
             // some layer of the run is outside the fused kernel: one launch per layer instead
